@@ -1,0 +1,218 @@
+/*
+ * specblock.h -- C ABI of the SpecBlock draft-and-verify hot path for NVIDIA B200 (sm_100a).
+ *
+ * One verifier iteration of SpecBlock (Algorithm 1) grows a draft tree by block
+ * expansions, scores every tree node with one parallel target forward, commits the
+ * longest accepted root-to-node path plus one bonus token, and keeps the committed
+ * positions' keys/values in the cache.  This library holds the device steps of that
+ * iteration that do not need model weights:
+ *
+ *   sb_tree_ancestors  ancestor bitmask / depth of every tree node      (Sec. 3.1, App. A.2, Fig. 4)
+ *   sb_tree_attention  tree-masked attention over prefix KV + ancestors (Sec. 3.1, App. A.2, Alg. 1 "verify")
+ *   sb_tree_expand     per-row top-k + bucket-driven branching          (Sec. 3.2, App. A.5, Alg. 1 "attach")
+ *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
+ *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
+ *
+ * Conventions that hold for every call
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
+ *     The library never allocates or frees device memory, keeps no state between calls,
+ *     enqueues its kernels on `stream` (a cudaStream_t passed as void*, NULL = legacy default
+ *     stream) and returns without synchronising.
+ *   - The return value reports what the host can see (null pointers, unsupported shapes,
+ *     a workspace that is too small, a failed launch).  Data-dependent problems (a parent
+ *     index that is not smaller than its child, a prefix longer than the cache, a page id
+ *     outside the pool) are written to the caller's `status` device array, one int32 per
+ *     sequence (0 = ok, else an sb_status value); the outputs of such a sequence are
+ *     zero-filled.  No kernel traps, spins without bound or reads outside the described arrays.
+ *   - bf16 = IEEE-754 binary32 truncated to its upper 16 bits (round-to-nearest-even on
+ *     conversion).  All accumulation is fp32.
+ *   - Tree node i of sequence b lives at logical cache position prefix_len[b] + i: the
+ *     forward that produced the tree's K/V appended them behind the prefix in node order.
+ */
+#ifndef SPECBLOCK_H_
+#define SPECBLOCK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SB_MAX_NODES 128 /* nodes per tree: one 128-bit ancestor mask per node            */
+#define SB_MAX_DEPTH 32  /* longest accepted path (drafted tokens) handled by accept/compact */
+#define SB_KMAX 16       /* widest per-row top-k kept by sb_tree_expand (paper's widest map entry is 10) */
+
+typedef enum sb_status {
+  SB_OK = 0,
+  SB_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, Hq % Hkv != 0 ...        */
+  SB_ERR_UNSUPPORTED = 2,  /* head_dim / page_size / limits outside what is built        */
+  SB_ERR_WORKSPACE = 3,    /* workspace smaller than the *_workspace_bytes query         */
+  SB_ERR_INVALID_TREE = 4, /* per-sequence: parent[i] not in {-1} U [0,i), too many nodes */
+  SB_ERR_BOUNDS = 5,       /* per-sequence: prefix+nodes beyond cache, page id outside pool */
+  SB_ERR_CUDA = 6          /* a CUDA runtime call or launch failed                       */
+} sb_status;
+
+typedef enum sb_dtype { SB_BF16 = 0, SB_F32 = 1 } sb_dtype;
+
+/*
+ * A ragged batch of draft trees over ONE layer's KV cache.
+ *
+ * Cache layouts (bf16, K and V separate, same shape):
+ *   page_size == 0 : contiguous  [batch][kv_capacity][n_kv_heads][head_dim]
+ *   page_size  > 0 : paged pool  [num_pages][page_size][n_kv_heads][head_dim]; logical position
+ *                    j of sequence b is row (j % page_size) of pool page
+ *                    page_table[b*max_pages + j / page_size].
+ * Tree: node_offsets is the exclusive scan of the per-sequence node counts N_b (N_b <=
+ * SB_MAX_NODES); parent[node_offsets[b] + i] is the LOCAL index of node i's parent, -1 when the
+ * node hangs directly off the prefix.  A valid tree has parent[i] in {-1} U [0, i).
+ * The three host integers at the end only size grids and bound loops; the kernels re-check
+ * the device values against them and flag SB_ERR_INVALID_TREE / SB_ERR_BOUNDS instead of
+ * trusting them.
+ */
+typedef struct sb_tree_batch {
+  int32_t batch;      /* B >= 1                                                     */
+  int32_t n_q_heads;  /* Hq                                                         */
+  int32_t n_kv_heads; /* Hkv, Hq % Hkv == 0, group size G = Hq/Hkv <= 16            */
+  int32_t head_dim;   /* D in {64, 128}                                             */
+  const void* k_cache;
+  const void* v_cache;
+  int32_t page_size;         /* 0 = contiguous, else a power of two >= 16           */
+  int32_t max_pages;         /* paged: row length of page_table                     */
+  int64_t kv_capacity;       /* contiguous: positions per sequence                  */
+  int32_t num_pages;         /* paged: pages in the pool                            */
+  int32_t total_nodes;       /* host copy of node_offsets[B]                        */
+  const int32_t* page_table; /* [B][max_pages], paged only                          */
+  const int32_t* prefix_len; /* [B]  P_b >= 0                                       */
+  const int32_t* node_offsets; /* [B+1]                                             */
+  const int32_t* parent;     /* [total_nodes]                                       */
+  int32_t max_nodes;         /* host upper bound on N_b (<= SB_MAX_NODES)           */
+  int32_t max_kv_len;        /* host upper bound on P_b + N_b                       */
+} sb_tree_batch;
+
+/*
+ * sb_tree_ancestors -- ancestor set and depth of every node (App. A.2; Fig. 4).
+ *   anc(i) = {i} U anc(parent[i]), anc(-1) = {}; depth(i) = |anc(i)| - 1.  Bit a of the 128-bit
+ *   mask anc_mask[node][4] (little-endian 32-bit words) is set iff a is in anc(i).  The
+ *   position id the figure prints for a node is prefix_len + depth.
+ *   node_offsets [B+1], parent [total]; outputs anc_mask uint32 [total][4], depth int32 [total],
+ *   status int32 [B].  anc_mask or depth may be NULL.  Invalid trees: status = SB_ERR_INVALID_TREE,
+ *   that sequence's outputs zero.
+ */
+sb_status sb_tree_ancestors(int32_t batch, const int32_t* node_offsets, const int32_t* parent,
+                            int32_t max_nodes, uint32_t* anc_mask, int32_t* depth,
+                            int32_t* status, void* stream);
+
+/*
+ * sb_tree_attention -- tree-masked attention of one layer (Sec. 3.1 "within-block
+ * dependence"; App. A.2: prefix fully visible, earlier draft positions visible only along
+ * the branch path, causal inside the block; Alg. 1 line "verify").
+ *
+ *   For sequence b, query node i in [q_node_begin[b], N_b), query head h (KV head g = h / G):
+ *     visible keys = {0..P_b-1} U {P_b + a : a in anc(i)}
+ *     s_j = scale * <q[i,h,:], k[j,g,:]>,  lse = ln sum_j exp(s_j),
+ *     out[i,h,:] = sum_j exp(s_j - lse) v[j,g,:]
+ *
+ *   q, out : bf16 [total_q][Hq][D]; sequence b's first query row is q_offsets[b] (NULL: the
+ *            rows follow node_offsets, which requires q_node_begin == NULL).
+ *   q_node_begin : [B] first node that has a query row (earlier nodes are cached context
+ *            only, e.g. blocks drafted by an earlier forward), or NULL = 0.
+ *   lse    : fp32 [total_q][Hq] natural-log sum-exp, or NULL.
+ *   scale  : 0 means 1/sqrt(D).
+ *   num_splits : how many KV chunks each (sequence, KV head, query tile) is cut into;
+ *            0 = chosen from the grid size.  Chunks are merged by log-sum-exp; a chunk in which
+ *            a row sees no key contributes nothing.
+ *   workspace : scratch of at least sb_tree_attention_workspace_bytes(...) bytes, 256-byte
+ *            aligned; contents need no initialisation and are garbage afterwards.  Calls
+ *            that may overlap on the GPU need distinct workspaces.
+ *   status : int32 [B].
+ */
+sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q_node_begin,
+                            const int32_t* q_offsets, int32_t total_q, const void* q, void* out,
+                            float* lse, float scale, int32_t num_splits, void* workspace,
+                            size_t workspace_bytes, int32_t* status, void* stream);
+
+/* Bytes of workspace sb_tree_attention needs for this batch / num_splits (0 = auto). Host only. */
+size_t sb_tree_attention_workspace_bytes(const sb_tree_batch* tb, int32_t total_q,
+                                         int32_t num_splits);
+
+/*
+ * sb_tree_expand -- attach candidates of one batched drafter forward to the tree
+ * (Sec. 3.2 "bucket-driven branching"; App. A.5 maps b(.); Alg. 1 lines "for each starting
+ * point i and position k: attach the top-b(bkt) tokens").
+ *
+ *   Rows r = i*block_k + k (start i, position k), scores fp32 [n_rows][row_stride >= vocab].
+ *   (1) per row the SB_KMAX best ids by (score descending, id ascending; NaN counts as -inf)
+ *       -> topk_tok int32 [n_rows][SB_KMAX], topk_val fp32 [n_rows][SB_KMAX] (ranks beyond vocab: -1 / -inf);
+ *   (2) b_r = bmap[bucket[r]] (bucket in 0..3; bmap host array of 4 entries, each 0..SB_KMAX);
+ *   (3) rows in order: row (i,0) attaches under start_parent[i] (an existing node id, or -1);
+ *       row (i,k>0) attaches under the rank-0 node created for row (i,k-1); when that node does
+ *       not exist the row and the rest of its block emit nothing;
+ *   (4) ranks 0..b_r-1 become nodes n_nodes, n_nodes+1, ... with tok, parent,
+ *       depth = depth[parent]+1 (0 under -1), node_row = r, node_rank = rank, until
+ *       node_budget nodes exist (emission stops for good).
+ *   n_nodes : device int32 scalar, in = nodes already in the arrays, out = new count.
+ *   tok/parent/depth/node_row/node_rank : int32 arrays of capacity node_budget.
+ *   workspace : sb_tree_expand_workspace_bytes(n_rows, vocab) bytes.
+ *   status : int32 [1].
+ */
+sb_status sb_tree_expand(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                         int32_t block_k, const uint8_t* bucket, const int32_t* bmap /*host[4]*/,
+                         const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
+                         int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
+                         int32_t* node_rank, int32_t* topk_tok, float* topk_val, void* workspace,
+                         size_t workspace_bytes, int32_t* status, void* stream);
+size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab);
+
+/*
+ * sb_verify_accept -- greedy (temperature 0) verification (App. A.5 "the longest accepted
+ * prefix is committed"; Alg. 1 "(prefix, bonus) <- verify(tree)"; case study: accepted
+ * tokens plus one bonus token are committed).
+ *
+ *   logits [total_nodes][row_stride >= vocab] (bf16 or fp32): the target's next-token scores
+ *   at every tree node.  amax[i] = smallest id attaining the row maximum (NaN counts as -inf).
+ *   Node 0 of each sequence is the root (last committed token, parent -1; any other parent of
+ *   -1 is SB_ERR_INVALID_TREE).  Node i>0 is accepted iff tok[i] == amax[parent[i]] and its
+ *   parent is accepted.  best = accepted node of greatest depth (ties: smallest index).
+ *   accept_len[b] = depth(best) (drafted tokens accepted; the committed count is accept_len+1);
+ *   path_nodes[b][0..accept_len] = root..best (rest -1); out_tokens[b][0..accept_len-1] = their
+ *   tokens (root excluded), out_tokens[b][accept_len] = bonus[b] = amax[best] (rest -1).
+ *   Row length of path_nodes/out_tokens is max_depth+1, max_depth <= SB_MAX_DEPTH; a deeper
+ *   accepted path is cut at max_depth.
+ *   workspace : sb_verify_accept_workspace_bytes(total_nodes, vocab) bytes.
+ */
+sb_status sb_verify_accept(const void* logits, sb_dtype dtype, int64_t row_stride, int32_t vocab,
+                           int32_t batch, int32_t total_nodes, const int32_t* node_offsets,
+                           const int32_t* parent, const int32_t* tok, int32_t max_depth,
+                           int32_t* amax, int32_t* accept_len, int32_t* path_nodes,
+                           int32_t* out_tokens, int32_t* bonus, void* workspace,
+                           size_t workspace_bytes, int32_t* status, void* stream);
+size_t sb_verify_accept_workspace_bytes(int32_t total_nodes, int32_t vocab);
+
+/*
+ * sb_kv_compact -- keep the committed positions' K/V, drop the rest (Sec. 3.1 / App. A.2: later
+ * forwards see every committed position's cached keys and values as the verified prefix).
+ *
+ *   For every layer l < n_layers (layer l's cache starts layer_stride_elems bf16 elements after
+ *   layer l-1's; tb->k_cache / v_cache are layer 0), K and V, sequence b, j = 0..accept_len[b]:
+ *       cache[P_b + j] <- cache[P_b + path_nodes[b][j]]          (in place)
+ *   new_len[b] = P_b + accept_len[b] + 1.  Positions >= new_len[b] are unspecified afterwards.
+ *   path_nodes int32 [B][max_depth+1] and accept_len int32 [B] as written by sb_verify_accept.
+ *   A path that is not strictly increasing from node 0, or leaves the tree, sets
+ *   SB_ERR_INVALID_TREE for that sequence and moves nothing.
+ */
+sb_status sb_kv_compact(const sb_tree_batch* tb, int32_t n_layers, int64_t layer_stride_elems,
+                        const int32_t* path_nodes, const int32_t* accept_len, int32_t max_depth,
+                        int32_t* new_len, int32_t* status, void* stream);
+
+/* Text for a status code (static storage). */
+const char* sb_status_string(sb_status s);
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t sb_version(void);
+/* Kernels launched by this library in this process since load (host counter, for benchmarks). */
+int64_t sb_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECBLOCK_H_ */

@@ -1,0 +1,211 @@
+"""ctypes loader for specblock_oracle.c -- TEST INFRASTRUCTURE ONLY.
+
+Thin numpy marshalling around the C oracle; no arithmetic of the method lives here.
+bf16 data travels as uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "specblock_oracle.c")
+_LIB = os.path.join(_HERE, "libspecblock_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+KMAX = 16
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (fp64, OpenMP only to spread rows over cores)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            _lib = C.CDLL(build())
+            _lib.sbo_num_threads.restype = C.c_int
+            for name in ("sbo_tree_ancestors", "sbo_tree_attention", "sbo_accept_from_amax",
+                         "sbo_tree_expand"):
+                getattr(_lib, name).restype = C.c_int
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _i32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.int32)
+
+
+def num_threads() -> int:
+    return int(_load().sbo_num_threads())
+
+
+def tree_ancestors(parent):
+    """-> (anc_mask uint32 [n,4], depth int32 [n], rc)."""
+    parent = _i32(parent)
+    n = parent.shape[0]
+    anc = np.zeros((n, 4), np.uint32)
+    depth = np.zeros(n, np.int32)
+    rc = _load().sbo_tree_ancestors(_p(parent), C.c_int(n), _p(anc), _p(depth))
+    return anc, depth, int(rc)
+
+
+def tree_attention(*, n_q_heads, n_kv_heads, head_dim, k, v, page_size=0, max_pages=0,
+                   num_pages=0, kv_capacity=0, page_table=None, prefix_len, node_offsets, parent,
+                   q, q_node_begin=None, q_offsets=None, scale=0.0, sel=None):
+    """k, v, q: uint16 bf16 bit patterns.  -> (out f64, lse f64, status int32 [B]).
+
+    sel=None: out [total_q, Hq, D], lse [total_q, Hq]; else sel int32 [n,3] of (b, node, head)
+    and out [n, D], lse [n].
+    """
+    k = np.ascontiguousarray(k, np.uint16)
+    v = np.ascontiguousarray(v, np.uint16)
+    q = np.ascontiguousarray(q, np.uint16)
+    prefix_len, node_offsets, parent = _i32(prefix_len), _i32(node_offsets), _i32(parent)
+    q_node_begin, q_offsets, page_table = _i32(q_node_begin), _i32(q_offsets), _i32(page_table)
+    batch = prefix_len.shape[0]
+    total_q = q.size // (n_q_heads * head_dim)
+    if sel is None:
+        n_sel = 0
+        out = np.zeros((total_q, n_q_heads, head_dim), np.float64)
+        lse = np.zeros((total_q, n_q_heads), np.float64)
+    else:
+        sel = _i32(sel).reshape(-1, 3)
+        n_sel = sel.shape[0]
+        out = np.zeros((n_sel, head_dim), np.float64)
+        lse = np.zeros(n_sel, np.float64)
+    status = np.zeros(batch, np.int32)
+    _load().sbo_tree_attention(
+        C.c_int(batch), C.c_int(n_q_heads), C.c_int(n_kv_heads), C.c_int(head_dim), _p(k), _p(v),
+        C.c_int(page_size), C.c_int(max_pages), C.c_int(num_pages), C.c_int64(kv_capacity),
+        _p(page_table), _p(prefix_len), _p(node_offsets), _p(parent), _p(q_node_begin),
+        _p(q_offsets), _p(q), C.c_double(scale), C.c_int64(n_sel), _p(sel), _p(out), _p(lse),
+        _p(status))
+    return out, lse, status
+
+
+def _logits_arg(logits):
+    if logits.dtype == np.uint16:
+        return np.ascontiguousarray(logits), 0
+    if logits.dtype == np.float32:
+        return np.ascontiguousarray(logits), 1
+    raise TypeError("logits must be uint16 (bf16 bits) or float32")
+
+
+def row_argmax(logits, vocab=None):
+    logits, dt = _logits_arg(logits)
+    n_rows, stride = logits.shape
+    vocab = stride if vocab is None else vocab
+    amax = np.zeros(n_rows, np.int32)
+    _load().sbo_row_argmax(_p(logits), C.c_int(dt), C.c_int64(stride), C.c_int(vocab),
+                           C.c_int64(n_rows), _p(amax))
+    return amax
+
+
+def row_topk(scores, vocab=None):
+    scores = np.ascontiguousarray(scores, np.float32)
+    n_rows, stride = scores.shape
+    vocab = stride if vocab is None else vocab
+    tok = np.zeros((n_rows, KMAX), np.int32)
+    val = np.zeros((n_rows, KMAX), np.float32)
+    _load().sbo_row_topk(_p(scores), C.c_int64(stride), C.c_int(n_rows), C.c_int(vocab), _p(tok),
+                         _p(val))
+    return tok, val
+
+
+def verify_accept(logits, node_offsets, parent, tok, max_depth, vocab=None):
+    """-> dict(amax, accept_len, path_nodes, out_tokens, bonus, status)."""
+    logits, dt = _logits_arg(logits)
+    node_offsets, parent, tok = _i32(node_offsets), _i32(parent), _i32(tok)
+    batch = node_offsets.shape[0] - 1
+    total, stride = logits.shape
+    vocab = stride if vocab is None else vocab
+    r = dict(amax=np.zeros(total, np.int32), accept_len=np.zeros(batch, np.int32),
+             path_nodes=np.zeros((batch, max_depth + 1), np.int32),
+             out_tokens=np.zeros((batch, max_depth + 1), np.int32),
+             bonus=np.zeros(batch, np.int32), status=np.zeros(batch, np.int32))
+    _load().sbo_verify_accept(_p(logits), C.c_int(dt), C.c_int64(stride), C.c_int(vocab),
+                              C.c_int(batch), _p(node_offsets), _p(parent), _p(tok),
+                              C.c_int(max_depth), _p(r["amax"]), _p(r["accept_len"]),
+                              _p(r["path_nodes"]), _p(r["out_tokens"]), _p(r["bonus"]),
+                              _p(r["status"]))
+    return r
+
+
+def accept_from_amax(parent, tok, amax, max_depth):
+    parent, tok, amax = _i32(parent), _i32(tok), _i32(amax)
+    n = parent.shape[0]
+    accept_len = np.zeros(1, np.int32)
+    bonus = np.zeros(1, np.int32)
+    path = np.zeros(max_depth + 1, np.int32)
+    out = np.zeros(max_depth + 1, np.int32)
+    rc = _load().sbo_accept_from_amax(C.c_int(n), _p(parent), _p(tok), _p(amax),
+                                      C.c_int(max_depth), _p(accept_len), _p(path), _p(out),
+                                      _p(bonus))
+    return dict(accept_len=int(accept_len[0]), path_nodes=path, out_tokens=out,
+                bonus=int(bonus[0]), status=int(rc))
+
+
+def kv_compact(*, n_kv_heads, head_dim, cache, n_layers, layer_stride_elems, page_size=0,
+               max_pages=0, num_pages=0, kv_capacity=0, page_table=None, prefix_len,
+               node_offsets, path_nodes, accept_len, max_depth):
+    """cache: uint16 flat array holding all layers.  -> (new_cache, new_len, status)."""
+    cache = np.ascontiguousarray(cache, np.uint16)
+    new = cache.copy()
+    prefix_len, node_offsets = _i32(prefix_len), _i32(node_offsets)
+    path_nodes, accept_len, page_table = _i32(path_nodes), _i32(accept_len), _i32(page_table)
+    batch = prefix_len.shape[0]
+    new_len = np.zeros(batch, np.int32)
+    status = np.zeros(batch, np.int32)
+    _load().sbo_kv_compact(C.c_int(batch), C.c_int(n_kv_heads), C.c_int(head_dim), _p(cache),
+                           _p(new), C.c_int(n_layers), C.c_int64(layer_stride_elems),
+                           C.c_int(page_size), C.c_int(max_pages), C.c_int(num_pages),
+                           C.c_int64(kv_capacity), _p(page_table), _p(prefix_len),
+                           _p(node_offsets), _p(path_nodes), _p(accept_len), C.c_int(max_depth),
+                           _p(new_len), _p(status))
+    return new, new_len, status
+
+
+def tree_expand(scores, block_k, bucket, bmap, start_parent, node_budget, tree=None, vocab=None):
+    """tree: optional dict(tok, parent, depth, node_row, node_rank) of existing nodes.
+
+    -> dict(n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val, status).
+    """
+    scores = np.ascontiguousarray(scores, np.float32)
+    n_rows, stride = scores.shape
+    vocab = stride if vocab is None else vocab
+    bucket = np.ascontiguousarray(bucket, np.uint8)
+    bmap, start_parent = _i32(bmap), _i32(start_parent)
+    arrs = {k: np.full(node_budget, -1, np.int32)
+            for k in ("tok", "parent", "depth", "node_row", "node_rank")}
+    n0 = 0
+    if tree is not None:
+        n0 = len(tree["tok"])
+        for k in arrs:
+            arrs[k][:n0] = tree[k]
+    n_nodes = np.array([n0], np.int32)
+    topk_tok = np.zeros((n_rows, KMAX), np.int32)
+    topk_val = np.zeros((n_rows, KMAX), np.float32)
+    rc = _load().sbo_tree_expand(_p(scores), C.c_int64(stride), C.c_int(n_rows), C.c_int(vocab),
+                                 C.c_int(block_k), _p(bucket), _p(bmap), _p(start_parent),
+                                 C.c_int(node_budget), _p(n_nodes), _p(arrs["tok"]),
+                                 _p(arrs["parent"]), _p(arrs["depth"]), _p(arrs["node_row"]),
+                                 _p(arrs["node_rank"]), _p(topk_tok), _p(topk_val))
+    return dict(n_nodes=int(n_nodes[0]), topk_tok=topk_tok, topk_val=topk_val, status=int(rc),
+                **arrs)

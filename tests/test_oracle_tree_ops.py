@@ -1,0 +1,342 @@
+"""Pins of the CPU oracle's integer steps (argmax, acceptance, compaction, top-k, branching) to
+library routines, independent algorithms on exhaustive small inputs, planted constructions and
+the paper's printed examples."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2605_07243_b200 import workloads as W
+
+
+# ---- argmax / top-k against numpy -------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("vocab", [7, 1000, 32000])
+def test_row_argmax_matches_numpy_first_maximum(dtype, vocab):
+    rng = W.rng_for(21)
+    x = rng.standard_normal((9, vocab), dtype=np.float32) * 2
+    x[3] = np.round(x[3])                      # many exact ties
+    x[4, :] = -np.inf
+    x[5, 2] = np.nan
+    x[5, 5] = np.inf
+    if dtype == "bf16":
+        bits = W.f32_to_bf16_bits(np.nan_to_num(x, nan=0.0, posinf=3e38, neginf=-3e38))
+        ref = np.argmax(W.bf16_bits_to_f32(bits), axis=1)       # numpy: first maximal index
+        got = oracle.row_argmax(bits)
+    else:
+        ref = np.argmax(np.where(np.isnan(x), -np.inf, x), axis=1)
+        got = oracle.row_argmax(x)
+    np.testing.assert_array_equal(got, ref)
+
+
+def test_row_argmax_all_nan_row_and_signed_zero():
+    x = np.full((2, 5), np.nan, np.float32)
+    x[1] = [-0.0, 0.0, -1.0, 0.0, -0.0]        # +0 == -0: the first one wins
+    np.testing.assert_array_equal(oracle.row_argmax(x), [0, 0])
+
+
+@pytest.mark.parametrize("vocab", [5, 16, 1000, 32000])
+def test_row_topk_matches_numpy_stable_sort(vocab):
+    rng = W.rng_for(22)
+    x = rng.standard_normal((6, vocab), dtype=np.float32) * 2
+    x[1] = np.round(x[1] * 2) / 2              # ties
+    x[2, ::3] = np.nan
+    tok, val = oracle.row_topk(x)
+    clean = np.where(np.isnan(x), -np.inf, x)
+    order = np.argsort(-clean, axis=1, kind="stable")           # value desc, id asc
+    k = min(16, vocab)
+    np.testing.assert_array_equal(tok[:, :k], order[:, :k])
+    np.testing.assert_array_equal(val[:, :k], np.take_along_axis(clean, order[:, :k], 1))
+    assert (tok[:, k:] == -1).all() and np.isneginf(val[:, k:]).all()
+    np.testing.assert_array_equal(tok[:, 0], oracle.row_argmax(x))   # k = 1 is the argmax
+
+
+# ---- acceptance ------------------------------------------------------------------------------------
+
+def _accept_by_recurrence(parent, tok, amax, max_depth):
+    """Independent algorithm: acc[i] = acc[parent] and tok[i] == amax[parent], in index order."""
+    n = len(parent)
+    acc = [False] * n
+    depth = [0] * n
+    acc[0] = True
+    best = 0
+    for i in range(1, n):
+        p = parent[i]
+        depth[i] = depth[p] + 1
+        acc[i] = acc[p] and tok[i] == amax[p] and depth[i] <= max_depth
+        if acc[i] and depth[i] > depth[best]:
+            best = i
+    path = [best]
+    while parent[path[-1]] >= 0:
+        path.append(parent[path[-1]])
+    path = path[::-1]
+    return depth[best], path, [tok[i] for i in path[1:]] + [amax[best]]
+
+
+def _all_trees(n):
+    """Every parent array with parent[0] = -1 and parent[i] in [0, i)."""
+    for rest in itertools.product(*[range(i) for i in range(1, n)]):
+        yield [-1] + list(rest)
+
+
+def test_accept_exhaustive_small_trees():
+    """All trees with up to 5 nodes x all token/choice assignments over a 2-letter alphabet
+    (plus 6-node trees on a sample): path enumeration equals the recurrence."""
+    rng = W.rng_for(23)
+    checked = 0
+    for n in range(1, 7):
+        for parent in _all_trees(n):
+            assigns = itertools.product(range(2), repeat=2 * n - 1)
+            if n == 6:
+                assigns = [tuple(rng.integers(0, 3, 2 * n - 1)) for _ in range(4)]
+            for a in assigns:
+                tok = [7] + list(a[: n - 1])
+                amax = list(a[n - 1:])
+                r = oracle.accept_from_amax(parent, tok, amax, max_depth=8)
+                ln, path, toks = _accept_by_recurrence(parent, tok, amax, 8)
+                assert r["status"] == 0 and r["accept_len"] == ln
+                assert list(r["path_nodes"][: ln + 1]) == path
+                assert list(r["out_tokens"][: ln + 1]) == toks
+                assert (r["path_nodes"][ln + 1:] == -1).all()
+                checked += 1
+    assert checked > 5000
+
+
+def test_accept_random_trees_with_duplicates_and_depth_cut():
+    rng = W.rng_for(24)
+    for _ in range(300):
+        n = int(rng.integers(1, 16))
+        parent = W.random_tree(rng, n, 6)
+        tok = rng.integers(0, 3, n)            # tiny alphabet: duplicate siblings, many matches
+        amax = rng.integers(0, 3, n)
+        md = int(rng.integers(1, 7))
+        r = oracle.accept_from_amax(parent, tok, amax, md)
+        ln, path, toks = _accept_by_recurrence(list(parent), list(tok), list(amax), md)
+        assert r["accept_len"] == ln and list(r["path_nodes"][: ln + 1]) == path
+        assert list(r["out_tokens"][: ln + 1]) == toks and r["bonus"] == toks[-1]
+
+
+def test_accept_chain_is_longest_matching_prefix():
+    """A chain tree is textbook greedy speculative verification of one draft sequence."""
+    rng = W.rng_for(25)
+    for _ in range(50):
+        n = int(rng.integers(2, 12))
+        tok = rng.integers(0, 2, n)
+        amax = rng.integers(0, 2, n)
+        matched = 0
+        while matched < n - 1 and tok[matched + 1] == amax[matched]:
+            matched += 1
+        r = oracle.accept_from_amax(W.chain_tree(n), tok, amax, 16)
+        assert r["accept_len"] == matched and r["bonus"] == amax[matched]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_accept_planted_path_is_recovered(dtype):
+    rng = W.rng_for(26)
+    parents = [W.random_tree(rng, int(n), 6) for n in (15, 1, 40, 9)]
+    case = W.make_verify_case(rng, parents=parents, vocab=777, dtype=dtype)
+    r = oracle.verify_accept(case.logits, case.node_offsets, case.parent, case.tok,
+                             case.max_depth)
+    assert not r["status"].any()
+    np.testing.assert_array_equal(r["accept_len"], case.planted_len)
+    np.testing.assert_array_equal(r["bonus"], case.planted_bonus)
+    for b, path in enumerate(case.planted_path):
+        assert list(r["path_nodes"][b, : len(path)]) == path
+
+
+def test_accept_case_study_tree(golden_dir):
+    """Case study, tree (b): the K=4 chain is accepted and a bonus follows -> five tokens."""
+    nodes, expect = [], {}
+    for line in open(os.path.join(golden_dir, "case_study_tree.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("expect_"):
+            key, *vals = line.split()
+            expect[key] = [int(t) for t in vals]
+        else:
+            nodes.append([int(t) for t in line.split()])
+    nodes = np.asarray(nodes)
+    r = oracle.accept_from_amax(nodes[:, 1], nodes[:, 2], nodes[:, 3], 8)
+    a = expect["expect_accept_len"][0]
+    assert r["accept_len"] == a and a + 1 == 5
+    assert list(r["out_tokens"][: a + 1]) == expect["expect_tokens"]
+
+
+def test_accept_rejects_second_root_and_bad_parent():
+    assert oracle.accept_from_amax([-1, -1], [1, 2], [2, 2], 4)["status"] == 4
+    assert oracle.accept_from_amax([-1, 1], [1, 2], [2, 2], 4)["status"] == 4
+
+
+# ---- compaction ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("page_size", [0, 16])
+def test_kv_compact_equals_numpy_gather(page_size):
+    rng = W.rng_for(27)
+    parents = [W.random_tree(rng, 20, 6), W.random_tree(rng, 9, 4)]
+    L = 3
+    case = W.make_attn_case(rng, parents=parents, prefix_lens=[19, 33], n_q_heads=4,
+                            n_kv_heads=2, head_dim=16, page_size=page_size)
+    layers = np.stack([rng.integers(0, 65536, case.k.shape).astype(np.uint16) for _ in range(L)])
+    paths = np.full((2, 7), -1, np.int32)
+    paths[0, :4] = [0, 2, 5, 11]
+    paths[1, :1] = [0]
+    alen = np.asarray([3, 0], np.int32)
+    new, new_len, st = oracle.kv_compact(
+        n_kv_heads=2, head_dim=16, cache=layers.reshape(-1), n_layers=L,
+        layer_stride_elems=layers[0].size, page_size=page_size, max_pages=case.max_pages,
+        num_pages=case.num_pages, kv_capacity=case.kv_capacity, page_table=case.page_table,
+        prefix_len=case.prefix_len, node_offsets=case.node_offsets, path_nodes=paths,
+        accept_len=alen, max_depth=6)
+    assert not st.any()
+    np.testing.assert_array_equal(new_len, case.prefix_len + alen + 1)
+    new = new.reshape(layers.shape)
+    ref = layers.copy()
+    for b in range(2):
+        P = int(case.prefix_len[b])
+        src = [W.kv_slot(case, b, P + int(p)) for p in paths[b, : alen[b] + 1]]
+        dst = [W.kv_slot(case, b, P + j) for j in range(alen[b] + 1)]
+        si, sj = zip(*src)
+        di, dj = zip(*dst)
+        ref[:, list(di), list(dj)] = layers[:, list(si), list(sj)]     # numpy fancy-index gather
+    np.testing.assert_array_equal(new, ref)
+
+
+def test_compaction_then_chain_attention_equals_tree_attention_of_last_path_node():
+    """After compaction the accepted path is an ordinary prefix: a new token attending to the
+    compacted cache sees exactly what the path's last node saw (plus itself)."""
+    rng = W.rng_for(28)
+    par = W.random_tree(rng, 12, 5)
+    case = W.make_attn_case(rng, parents=[par], prefix_lens=[23], n_q_heads=2, n_kv_heads=1,
+                            head_dim=32, capacity_pad=4)
+    end = 11
+    path = [end]
+    while par[path[-1]] >= 0:
+        path.append(int(par[path[-1]]))
+    path = path[::-1]
+    a = len(path) - 1
+    paths = np.full((1, 8), -1, np.int32)
+    paths[0, : a + 1] = path
+    out_tree, lse_tree, _ = oracle.tree_attention(**case.oracle_kwargs())
+    new = {}
+    for name in ("k", "v"):
+        arr = getattr(case, name)
+        new[name], new_len, st = oracle.kv_compact(
+            n_kv_heads=1, head_dim=32, cache=arr.reshape(-1), n_layers=1, layer_stride_elems=0,
+            kv_capacity=case.kv_capacity, prefix_len=case.prefix_len,
+            node_offsets=case.node_offsets, path_nodes=paths, accept_len=[a], max_depth=7)
+        new[name] = new[name].reshape(arr.shape)
+    # the path's last node, re-asked as a single node whose own K/V sit at the new prefix end
+    P2 = int(new_len[0]) - 1
+    kw = case.oracle_kwargs()
+    kw.update(k=new["k"], v=new["v"], prefix_len=[P2], node_offsets=[0, 1], parent=[-1],
+              q=case.q[end:end + 1])
+    out2, lse2, st2 = oracle.tree_attention(**kw)
+    np.testing.assert_allclose(out2[0], out_tree[end], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(lse2[0], lse_tree[end], rtol=1e-13)
+
+
+def test_kv_compact_flags_bad_paths():
+    rng = W.rng_for(29)
+    case = W.make_attn_case(rng, parents=[W.chain_tree(5)], prefix_lens=[4], n_q_heads=1,
+                            n_kv_heads=1, head_dim=16)
+    for bad in ([1, 2, -1], [0, 3, 2], [0, 2, 7]):
+        _n, new_len, st = oracle.kv_compact(
+            n_kv_heads=1, head_dim=16, cache=case.k.reshape(-1), n_layers=1, layer_stride_elems=0,
+            kv_capacity=case.kv_capacity, prefix_len=case.prefix_len,
+            node_offsets=case.node_offsets, path_nodes=np.asarray([bad], np.int32),
+            accept_len=[2], max_depth=2)
+        assert st[0] == 4 and new_len[0] == 4
+
+
+# ---- branching ---------------------------------------------------------------------------------------------
+
+def _read_expand_examples(golden_dir):
+    ex, cur = {}, None
+    for line in open(os.path.join(golden_dir, "expand_examples.txt")):
+        t = line.split()
+        if not t or t[0] == "#" or t[0].startswith("#"):
+            continue
+        if t[0] == "example":
+            cur = dict(nodes=[])
+            ex[t[1]] = cur
+        elif t[0] == "node":
+            cur["nodes"].append([int(x) for x in t[1:]])
+        elif t[0] == "existing":
+            cur["existing"] = t[1]
+        elif t[0] != "end":
+            cur[t[0]] = [int(x) for x in t[1:]]
+    return ex
+
+
+def _scores_with_known_ranking(rng, n_rows, vocab):
+    """Row r ranks the ids of a random permutation: its j-th entry gets the j-th largest score."""
+    ranking = np.stack([rng.permutation(vocab) for _ in range(n_rows)])
+    scores = np.zeros((n_rows, vocab), np.float32)
+    for r in range(n_rows):
+        scores[r, ranking[r]] = 100.0 - np.arange(vocab, dtype=np.float32)
+    return scores, ranking
+
+
+def test_expand_hand_derived_examples(golden_dir):
+    """The two printed branching maps on hand-worked blocks, incl. a width-0 bucket that ends a
+    block, a second block level, and the node budget cutting a row."""
+    ex = _read_expand_examples(golden_dir)
+    rng = W.rng_for(30)
+    results = {}
+    for name in ("A", "B", "C"):
+        e = ex[name]
+        n_rows = len(e["bucket"])
+        scores, ranking = _scores_with_known_ranking(rng, n_rows, 50)
+        tree = None if e["existing"] == "0" else results[e["existing"]]
+        n0 = 0 if tree is None else len(tree["tok"])
+        r = oracle.tree_expand(scores, e["block_k"][0], e["bucket"], e["bmap"], e["start_parent"],
+                               e["budget"][0], tree=tree)
+        assert r["status"] == 0
+        want = np.asarray(e["nodes"])
+        assert r["n_nodes"] == n0 + len(want)
+        new = slice(n0, r["n_nodes"])
+        np.testing.assert_array_equal(r["parent"][new], want[:, 0])
+        np.testing.assert_array_equal(r["depth"][new], want[:, 1])
+        np.testing.assert_array_equal(r["node_row"][new], want[:, 2])
+        np.testing.assert_array_equal(r["node_rank"][new], want[:, 3])
+        np.testing.assert_array_equal(r["tok"][new], ranking[want[:, 2], want[:, 3]])
+        results[name] = {k: r[k][: r["n_nodes"]] for k in
+                         ("tok", "parent", "depth", "node_row", "node_rank")}
+
+
+def test_expand_width_one_gives_pure_chains_and_invariants():
+    rng = W.rng_for(31)
+    case = W.make_expand_case(rng, n_starts=3, block_k=4, vocab=500, bmap=[1, 1, 1, 1],
+                              node_budget=64)
+    r = oracle.tree_expand(case.scores, 4, case.bucket, case.bmap, case.start_parent, 64)
+    assert r["n_nodes"] == 12
+    for i in range(3):
+        np.testing.assert_array_equal(r["parent"][4 * i: 4 * i + 4],
+                                      [-1, 4 * i, 4 * i + 1, 4 * i + 2])
+        np.testing.assert_array_equal(r["depth"][4 * i: 4 * i + 4], [0, 1, 2, 3])
+    np.testing.assert_array_equal(r["tok"][:12], np.argmax(case.scores, axis=1))
+    # random maps: budget respected, parents precede children, depth bounded by M*K
+    for trial in range(20):
+        bmap = rng.integers(0, 11, 4)
+        existing = W.random_tree(rng, 6, 3)
+        c = W.make_expand_case(rng, n_starts=5, block_k=4, vocab=300, bmap=bmap, node_budget=60,
+                               existing_parent=existing)
+        r = oracle.tree_expand(c.scores, 4, c.bucket, c.bmap, c.start_parent, 60, tree=c.tree)
+        n = r["n_nodes"]
+        assert 6 <= n <= 60
+        assert (r["parent"][6:n] < np.arange(6, n)).all()
+        assert r["depth"][:n].max() <= 3 + 4
+        assert (r["depth"][6:n] == r["depth"][r["parent"][6:n]] + 1).all()
+
+
+def test_expand_rejects_bad_arguments():
+    rng = W.rng_for(32)
+    c = W.make_expand_case(rng, n_starts=1, block_k=4, vocab=50, bmap=[2, 4, 10, 0],
+                           node_budget=20)
+    assert oracle.tree_expand(c.scores, 4, [0, 1, 4, 0], c.bmap, [-1], 20)["status"] == 1
+    assert oracle.tree_expand(c.scores, 4, c.bucket, [2, 4, 17, 0], [-1], 20)["status"] == 1
+    assert oracle.tree_expand(c.scores, 4, c.bucket, c.bmap, [0], 20)["status"] == 1
