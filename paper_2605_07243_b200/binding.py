@@ -1,0 +1,277 @@
+"""ctypes binding of libspecblock.so -- argument marshalling only.
+
+Every function here has the name of the C entry point it calls (include/specblock.h) and does
+nothing but turn torch CUDA tensors into device pointers, size the workspace and raise on a
+non-zero return code.  All computation happens in the CUDA library; there is no CPU fallback:
+if the library is missing or no CUDA device is present these calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+SB_MAX_NODES = 128
+SB_MAX_DEPTH = 32
+SB_KMAX = 16
+SB_BF16, SB_F32 = 0, 1
+
+STATUS_NAMES = {0: "SB_OK", 1: "SB_ERR_INVALID_ARG", 2: "SB_ERR_UNSUPPORTED", 3: "SB_ERR_WORKSPACE",
+                4: "SB_ERR_INVALID_TREE", 5: "SB_ERR_BOUNDS", 6: "SB_ERR_CUDA"}
+
+
+class SbError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)}")
+
+
+class _TreeBatch(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("page_size", C.c_int32), ("max_pages", C.c_int32), ("kv_capacity", C.c_int64),
+        ("num_pages", C.c_int32), ("total_nodes", C.c_int32), ("page_table", C.c_void_p),
+        ("prefix_len", C.c_void_p), ("node_offsets", C.c_void_p), ("parent", C.c_void_p),
+        ("max_nodes", C.c_int32), ("max_kv_len", C.c_int32),
+    ]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True):
+    """Load libspecblock.so (building it in-tree with nvcc when it is absent or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build() if build_if_missing else _build.LIB
+    if not os.path.exists(path):
+        raise RuntimeError("libspecblock.so is not built: run python -m paper_2605_07243_b200.build")
+    lib = C.CDLL(path)
+    lib.sb_status_string.restype = C.c_char_p
+    lib.sb_version.restype = C.c_int32
+    lib.sb_kernel_launch_count.restype = C.c_int64
+    for name in ("sb_tree_attention_workspace_bytes", "sb_tree_expand_workspace_bytes",
+                 "sb_verify_accept_workspace_bytes"):
+        getattr(lib, name).restype = C.c_size_t
+    for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
+                 "sb_kv_compact"):
+        getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspace_bytes",
+            "sb_tree_expand", "sb_tree_expand_workspace_bytes", "sb_verify_accept",
+            "sb_verify_accept_workspace_bytes", "sb_kv_compact", "sb_status_string", "sb_version",
+            "sb_kernel_launch_count")
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code, where):
+    if code != 0:
+        raise SbError(code, where)
+
+
+def sb_kernel_launch_count() -> int:
+    return int(load().sb_kernel_launch_count())
+
+
+def sb_version() -> int:
+    return int(load().sb_version())
+
+
+def sb_status_string(code: int) -> str:
+    return load().sb_status_string(C.c_int(code)).decode()
+
+
+@dataclass
+class TreeBatch:
+    """Device-side description of a ragged batch of trees over one layer's KV cache; mirrors the
+    C struct sb_tree_batch field for field.  k_cache / v_cache: bf16 tensors."""
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    k_cache: torch.Tensor
+    v_cache: torch.Tensor
+    prefix_len: torch.Tensor          # int32 [B]
+    node_offsets: torch.Tensor        # int32 [B+1]
+    parent: torch.Tensor              # int32 [total_nodes]
+    total_nodes: int
+    max_nodes: int
+    max_kv_len: int
+    page_size: int = 0
+    kv_capacity: int = 0
+    page_table: Optional[torch.Tensor] = None   # int32 [B, max_pages]
+    num_pages: int = 0
+    max_pages: int = 0
+
+    def c_struct(self, k_cache=None, v_cache=None) -> _TreeBatch:
+        k = self.k_cache if k_cache is None else k_cache
+        v = self.v_cache if v_cache is None else v_cache
+        s = _TreeBatch()
+        s.batch = self.prefix_len.numel()
+        s.n_q_heads, s.n_kv_heads, s.head_dim = self.n_q_heads, self.n_kv_heads, self.head_dim
+        s.k_cache = _ptr(k, torch.bfloat16).value
+        s.v_cache = _ptr(v, torch.bfloat16).value
+        s.page_size, s.max_pages, s.kv_capacity = self.page_size, self.max_pages, self.kv_capacity
+        s.num_pages, s.total_nodes = self.num_pages, self.total_nodes
+        s.page_table = None if self.page_table is None else _ptr(self.page_table, torch.int32).value
+        s.prefix_len = _ptr(self.prefix_len, torch.int32).value
+        s.node_offsets = _ptr(self.node_offsets, torch.int32).value
+        s.parent = _ptr(self.parent, torch.int32).value
+        s.max_nodes, s.max_kv_len = self.max_nodes, self.max_kv_len
+        return s
+
+
+def sb_tree_ancestors(node_offsets, parent, max_nodes, anc_mask=None, depth=None, status=None):
+    """-> (anc_mask int32 [total,4] holding the uint32 words, depth int32 [total], status [B])."""
+    batch = node_offsets.numel() - 1
+    total = parent.numel()
+    dev = parent.device
+    anc_mask = torch.empty((total, 4), dtype=torch.int32, device=dev) if anc_mask is None else anc_mask
+    depth = torch.empty(total, dtype=torch.int32, device=dev) if depth is None else depth
+    status = torch.empty(batch, dtype=torch.int32, device=dev) if status is None else status
+    rc = load().sb_tree_ancestors(C.c_int32(batch), _ptr(node_offsets, torch.int32),
+                                  _ptr(parent, torch.int32), C.c_int32(max_nodes), _ptr(anc_mask),
+                                  _ptr(depth, torch.int32), _ptr(status, torch.int32), _stream())
+    _check(rc, "sb_tree_ancestors")
+    return anc_mask, depth, status
+
+
+def sb_tree_attention_workspace_bytes(tb: TreeBatch, total_q: int, num_splits: int = 0) -> int:
+    s = tb.c_struct()
+    return int(load().sb_tree_attention_workspace_bytes(C.byref(s), C.c_int32(total_q),
+                                                        C.c_int32(num_splits)))
+
+
+def sb_tree_attention(tb: TreeBatch, q, out=None, lse=None, *, q_node_begin=None, q_offsets=None,
+                      scale=0.0, num_splits=0, workspace=None, status=None, want_lse=True,
+                      k_cache=None, v_cache=None):
+    """q bf16 [total_q, Hq, D] -> (out bf16 like q, lse fp32 [total_q, Hq] or None, status [B]).
+    k_cache / v_cache override the batch's layer (same layout) without rebuilding it."""
+    total_q = q.shape[0]
+    dev = q.device
+    out = torch.empty_like(q) if out is None else out
+    if lse is None and want_lse:
+        lse = torch.empty((total_q, tb.n_q_heads), dtype=torch.float32, device=dev)
+    status = torch.empty(tb.prefix_len.numel(), dtype=torch.int32, device=dev) if status is None else status
+    s = tb.c_struct(k_cache, v_cache)
+    lib = load()
+    if workspace is None:
+        need = int(lib.sb_tree_attention_workspace_bytes(C.byref(s), C.c_int32(total_q),
+                                                         C.c_int32(num_splits)))
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    rc = lib.sb_tree_attention(C.byref(s), _ptr(q_node_begin, torch.int32), _ptr(q_offsets, torch.int32),
+                               C.c_int32(total_q), _ptr(q, torch.bfloat16), _ptr(out, torch.bfloat16),
+                               _ptr(lse, torch.float32), C.c_float(scale), C.c_int32(num_splits),
+                               _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()),
+                               _ptr(status, torch.int32), _stream())
+    _check(rc, "sb_tree_attention")
+    return out, lse, status
+
+
+def sb_verify_accept_workspace_bytes(total_nodes: int, vocab: int) -> int:
+    return int(load().sb_verify_accept_workspace_bytes(C.c_int32(total_nodes), C.c_int32(vocab)))
+
+
+def sb_verify_accept(logits, node_offsets, parent, tok, max_depth, *, vocab=None, workspace=None,
+                     out=None):
+    """logits [total_nodes, stride] bf16 or fp32 -> dict(amax, accept_len, path_nodes, out_tokens,
+    bonus, status) of int32 device tensors (`out` may pass preallocated ones)."""
+    total, stride = logits.shape
+    vocab = stride if vocab is None else vocab
+    batch = node_offsets.numel() - 1
+    dev = logits.device
+    dt = {torch.bfloat16: SB_BF16, torch.float32: SB_F32}[logits.dtype]
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=dev)
+        out = dict(amax=torch.empty(total, **i32), accept_len=torch.empty(batch, **i32),
+                   path_nodes=torch.empty((batch, max_depth + 1), **i32),
+                   out_tokens=torch.empty((batch, max_depth + 1), **i32),
+                   bonus=torch.empty(batch, **i32), status=torch.empty(batch, **i32))
+    lib = load()
+    if workspace is None:
+        need = sb_verify_accept_workspace_bytes(total, vocab)
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    rc = lib.sb_verify_accept(_ptr(logits), C.c_int(dt), C.c_int64(stride), C.c_int32(vocab),
+                              C.c_int32(batch), C.c_int32(total), _ptr(node_offsets, torch.int32),
+                              _ptr(parent, torch.int32), _ptr(tok, torch.int32), C.c_int32(max_depth),
+                              _ptr(out["amax"]), _ptr(out["accept_len"]), _ptr(out["path_nodes"]),
+                              _ptr(out["out_tokens"]), _ptr(out["bonus"]), _ptr(workspace),
+                              C.c_size_t(workspace.numel()), _ptr(out["status"]), _stream())
+    _check(rc, "sb_verify_accept")
+    return out
+
+
+def sb_kv_compact(tb: TreeBatch, n_layers, layer_stride_elems, path_nodes, accept_len, max_depth,
+                  new_len=None, status=None):
+    """In-place compaction of tb.k_cache / tb.v_cache (layer 0 of n_layers).  -> (new_len, status)."""
+    batch = tb.prefix_len.numel()
+    dev = tb.prefix_len.device
+    new_len = torch.empty(batch, dtype=torch.int32, device=dev) if new_len is None else new_len
+    status = torch.empty(batch, dtype=torch.int32, device=dev) if status is None else status
+    s = tb.c_struct()
+    rc = load().sb_kv_compact(C.byref(s), C.c_int32(n_layers), C.c_int64(layer_stride_elems),
+                              _ptr(path_nodes, torch.int32), _ptr(accept_len, torch.int32),
+                              C.c_int32(max_depth), _ptr(new_len, torch.int32),
+                              _ptr(status, torch.int32), _stream())
+    _check(rc, "sb_kv_compact")
+    return new_len, status
+
+
+def sb_tree_expand_workspace_bytes(n_rows: int, vocab: int) -> int:
+    return int(load().sb_tree_expand_workspace_bytes(C.c_int32(n_rows), C.c_int32(vocab)))
+
+
+def sb_tree_expand(scores, block_k, bucket, bmap, start_parent, node_budget, tree, *, vocab=None,
+                   workspace=None, topk_tok=None, topk_val=None, status=None):
+    """scores fp32 [R, stride]; bucket uint8 [R]; bmap: 4 host ints; tree: dict of int32 device
+    tensors n_nodes [1], tok, parent, depth, node_row, node_rank (capacity node_budget), updated
+    in place.  -> (topk_tok [R,16], topk_val [R,16], status [1])."""
+    n_rows, stride = scores.shape
+    vocab = stride if vocab is None else vocab
+    dev = scores.device
+    topk_tok = torch.empty((n_rows, SB_KMAX), dtype=torch.int32, device=dev) if topk_tok is None else topk_tok
+    topk_val = torch.empty((n_rows, SB_KMAX), dtype=torch.float32, device=dev) if topk_val is None else topk_val
+    status = torch.empty(1, dtype=torch.int32, device=dev) if status is None else status
+    lib = load()
+    if workspace is None:
+        need = sb_tree_expand_workspace_bytes(n_rows, vocab)
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    bm = (C.c_int32 * 4)(*[int(x) for x in bmap])
+    rc = lib.sb_tree_expand(_ptr(scores, torch.float32), C.c_int64(stride), C.c_int32(n_rows),
+                            C.c_int32(vocab), C.c_int32(block_k), _ptr(bucket, torch.uint8), bm,
+                            _ptr(start_parent, torch.int32), C.c_int32(node_budget),
+                            _ptr(tree["n_nodes"], torch.int32), _ptr(tree["tok"], torch.int32),
+                            _ptr(tree["parent"], torch.int32), _ptr(tree["depth"], torch.int32),
+                            _ptr(tree["node_row"], torch.int32), _ptr(tree["node_rank"], torch.int32),
+                            _ptr(topk_tok, torch.int32), _ptr(topk_val, torch.float32), _ptr(workspace),
+                            C.c_size_t(workspace.numel()), _ptr(status, torch.int32), _stream())
+    _check(rc, "sb_tree_expand")
+    return topk_tok, topk_val, status

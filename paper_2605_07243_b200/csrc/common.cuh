@@ -1,0 +1,132 @@
+// Shared device/host helpers of the SpecBlock CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/specblock.h"
+
+namespace sb {
+
+// Host-side count of kernel launches made by this library (read by benchmarks).
+extern long long g_launch_count;
+
+inline sb_status launch_check() {
+  ++g_launch_count;
+  return cudaGetLastError() == cudaSuccess ? SB_OK : SB_ERR_CUDA;
+}
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Per-sequence facts every CTA of a sequence derives identically from device data.
+struct SeqInfo {
+  int n;       // tree nodes
+  int P;       // prefix length
+  int q0;      // first node with a query row
+  int q_off;   // first row of this sequence in q / out
+  int nq;      // query nodes
+  int err;     // 0 or an sb_status for this sequence (tree shape and lengths only)
+};
+
+// Length/shape checks that need no pass over arrays.
+__device__ inline SeqInfo load_seq_info(const sb_tree_batch& tb, const int* q_node_begin,
+                                        const int* q_offsets, int total_q, int b) {
+  SeqInfo s;
+  const int o = tb.node_offsets[b];
+  s.n = tb.node_offsets[b + 1] - o;
+  s.P = tb.prefix_len[b];
+  s.q0 = q_node_begin ? q_node_begin[b] : 0;
+  s.q_off = q_offsets ? q_offsets[b] : o;
+  s.nq = s.n - s.q0;
+  s.err = 0;
+  if (s.n < 0 || s.n > tb.max_nodes || s.n > SB_MAX_NODES || o < 0 ||
+      (long long)o + s.n > tb.total_nodes || s.q0 < 0 || s.q0 > s.n) {
+    s.err = SB_ERR_INVALID_TREE;
+  } else if (s.P < 0 || (long long)s.P + s.n > tb.max_kv_len ||
+             (tb.page_size == 0 ? (long long)s.P + s.n > tb.kv_capacity
+                                : (long long)s.P + s.n > (long long)tb.max_pages * tb.page_size) ||
+             s.q_off < 0 || (long long)s.q_off + s.nq > total_q) {
+    s.err = SB_ERR_BOUNDS;
+  }
+  if (s.err) { s.n = 0; s.nq = 0; s.P = 0; }
+  return s;
+}
+
+// Builds anc[i] = {i} U anc[parent[i]] for one tree into shared memory (4 words per node) and
+// returns false for an invalid tree.  `s_parent` is scratch of n ints.  Every thread of the
+// CTA must call it; it contains __syncthreads().
+__device__ inline bool build_ancestors_smem(const int* __restrict__ parent_g, int n,
+                                            int* s_parent, uint32_t* s_anc, int* s_depth) {
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int p = parent_g[i];
+    s_parent[i] = p;
+    if (p < -1 || p >= i) s_bad = 1;
+  }
+  __syncthreads();
+  const bool ok = s_bad == 0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;
+    int d = -1;
+    if (ok) {
+      // parent[a] < a for every a, so the walk ends after at most n steps
+      for (int a = i; a >= 0; a = s_parent[a]) {
+        const uint32_t bit = 1u << (a & 31);
+        const int w = a >> 5;
+        m0 |= w == 0 ? bit : 0u;
+        m1 |= w == 1 ? bit : 0u;
+        m2 |= w == 2 ? bit : 0u;
+        m3 |= w == 3 ? bit : 0u;
+        ++d;
+      }
+    }
+    s_anc[4 * i + 0] = m0;
+    s_anc[4 * i + 1] = m1;
+    s_anc[4 * i + 2] = m2;
+    s_anc[4 * i + 3] = m3;
+    if (s_depth) s_depth[i] = d < 0 ? 0 : d;
+  }
+  __syncthreads();
+  return ok;
+}
+
+// Element offset (in bf16 elements) of cache row (sequence b, logical position j), kv head 0.
+// Bad page ids are clamped to page 0 so that no access leaves the pool; the sequence's
+// designated CTA reports them.
+__device__ inline long long kv_row_elem_offset(const sb_tree_batch& tb, int b, int j) {
+  long long row;
+  if (tb.page_size == 0) {
+    row = (long long)b * tb.kv_capacity + j;
+  } else {
+    const int lp = j / tb.page_size;
+    int page = tb.page_table[(long long)b * tb.max_pages + lp];
+    if (page < 0 || page >= tb.num_pages) page = 0;
+    row = (long long)page * tb.page_size + (j - lp * tb.page_size);
+  }
+  return row * tb.n_kv_heads * (long long)tb.head_dim;
+}
+
+// True when every page the sequence's [0, len) positions need is inside the pool.
+__device__ inline bool pages_in_pool(const sb_tree_batch& tb, int b, int len) {
+  if (tb.page_size == 0) return true;
+  __shared__ int s_bad_page;
+  if (threadIdx.x == 0) s_bad_page = 0;
+  __syncthreads();
+  const int need = ceil_div(len, tb.page_size);
+  for (int p = threadIdx.x; p < need; p += blockDim.x) {
+    const int page = tb.page_table[(long long)b * tb.max_pages + p];
+    if (page < 0 || page >= tb.num_pages) s_bad_page = 1;
+  }
+  __syncthreads();
+  return s_bad_page == 0;
+}
+
+__device__ inline float bf16_bits_to_float(uint16_t h) { return __uint_as_float(((uint32_t)h) << 16); }
+
+// NaN takes part in max / top-k as -infinity.
+__device__ inline float score_of(float x) { return x != x ? -INFINITY : x; }
+
+}  // namespace sb

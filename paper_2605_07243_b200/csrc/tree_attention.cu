@@ -1,0 +1,648 @@
+// sb_tree_attention: tree-masked split-KV attention of one layer (Sec. 3.1; App. A.2; Alg. 1 "verify").
+//
+// Every node of a draft tree attends to the whole verified prefix plus its own ancestors
+// (itself included).  Query rows of one KV head are packed as (node, head-in-group) so a CTA's
+// 128-row tile shares every K/V tile it streams (GQA head packing).  The ancestor sets live in
+// shared memory as one 128-bit mask per node and are applied only to the KV tiles that overlap
+// the tree's cache slots; prefix tiles run unmasked.  The KV range of a (sequence, KV head, row
+// tile) is cut into `num_splits` chunks handled by different CTAs; a second kernel merges the
+// chunks' (out, log-sum-exp) pairs.
+//
+// Kernels in this file
+//   attn_simple_kernel : one warp per query row, fp32 FMA.  Slow, shape-agnostic check path
+//                        (environment SB_ATTN_IMPL=simple selects it).
+//   attn_mma_kernel    : flash-decode with bf16 tensor-core MMA (m16n8k16), fp32 accumulate,
+//                        3-stage cp.async K/V pipeline in XOR-swizzled shared memory.
+//   attn_merge_kernel  : log-sum-exp merge of the split partials.
+#include <cstdlib>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace sb {
+
+typedef __nv_bfloat16 bf16;
+
+struct AttnParams {
+  sb_tree_batch tb;
+  const int* q_node_begin;
+  const int* q_offsets;
+  int total_q;
+  const bf16* q;
+  bf16* out;
+  float* lse;
+  float scale_log2;  // softmax scale * log2(e): scores are kept in the base-2 domain
+  int num_splits;
+  float* part_o;    // [num_splits][total_q*Hq][D] normalised partial outputs
+  float* part_lse;  // [num_splits][total_q*Hq]    base-2 log-sum-exp of each partial
+  int* status;
+  int G;            // query heads per KV head
+};
+
+constexpr float kLn2 = 0.6931471805599453f;
+
+// What a CTA may do for its sequence after the shape checks.
+struct SeqPlan {
+  SeqInfo info;
+  bool can_write;  // the sequence's output rows are inside q/out
+  bool compute;    // tree and lengths are valid: run the attention
+};
+
+// Must be called by every thread of the CTA (contains barriers).  `designated` CTAs (one per
+// sequence) also scan the page table and publish the sequence's status word.
+__device__ inline SeqPlan plan_sequence(const AttnParams& p, int b, bool designated, int* s_parent,
+                                        uint32_t* s_anc) {
+  SeqPlan sp;
+  sp.info = load_seq_info(p.tb, p.q_node_begin, p.q_offsets, p.total_q, b);
+  int err = sp.info.err;
+  // Which rows may be zero-filled on error: recompute the raw row range.
+  const int o = p.tb.node_offsets[b];
+  const int n_raw = p.tb.node_offsets[b + 1] - o;
+  const int q0 = p.q_node_begin ? p.q_node_begin[b] : 0;
+  const int q_off = p.q_offsets ? p.q_offsets[b] : o;
+  const bool rows_ok = n_raw >= 0 && n_raw <= SB_MAX_NODES && n_raw <= p.tb.max_nodes && q0 >= 0 &&
+                       q0 <= n_raw && q_off >= 0 && (long long)q_off + (n_raw - q0) <= p.total_q &&
+                       o >= 0 && (long long)o + n_raw <= p.tb.total_nodes;
+  sp.can_write = rows_ok;
+  if (rows_ok && err) {  // lengths are bad but the rows exist: keep them for zero-filling
+    sp.info.nq = n_raw - q0;
+    sp.info.q0 = q0;
+    sp.info.q_off = q_off;
+  }
+  const bool tree_ok = build_ancestors_smem(p.tb.parent + (rows_ok ? o : 0), err ? 0 : sp.info.n,
+                                            s_parent, s_anc, nullptr);
+  if (!err && !tree_ok) err = SB_ERR_INVALID_TREE;
+  if (designated) {
+    const bool pages_ok = err ? true : pages_in_pool(p.tb, b, sp.info.P + sp.info.n);
+    if (!err && !pages_ok) err = SB_ERR_BOUNDS;  // reported; reads were clamped into the pool
+    if (threadIdx.x == 0) p.status[b] = err;
+    if (!pages_ok) err = 0;  // other CTAs cannot see this; stay consistent with them
+  }
+  sp.compute = err == 0;
+  return sp;
+}
+
+// ----------------------------------------------------------------------------------------------
+// Simple kernel: one warp per (node, head) row.
+// ----------------------------------------------------------------------------------------------
+
+template <int D>
+__global__ void __launch_bounds__(256) attn_simple_kernel(const AttnParams p) {
+  constexpr int E = D / 32;  // elements per lane
+  __shared__ int s_parent[SB_MAX_NODES];
+  __shared__ uint32_t s_anc[SB_MAX_NODES * 4];
+  const int b = blockIdx.y;
+  const SeqPlan sp = plan_sequence(p, b, blockIdx.x == 0, s_parent, s_anc);
+  const SeqInfo& si = sp.info;
+  const int Hq = p.tb.n_q_heads;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rr = blockIdx.x * 8 + warp;
+  if (!sp.can_write || rr >= si.nq * Hq) return;
+  const int node = si.q0 + rr / Hq, h = rr % Hq, g = h / p.G;
+  const long long grow = (long long)si.q_off * Hq + rr;
+  bf16* orow = p.out + grow * D + lane * E;
+  if (!sp.compute) {
+#pragma unroll
+    for (int e = 0; e < E; ++e) orow[e] = __float2bfloat16(0.f);
+    if (p.lse && lane == 0) p.lse[grow] = 0.f;
+    return;
+  }
+  float qv[E], acc[E];
+#pragma unroll
+  for (int e = 0; e < E; ++e) {
+    qv[e] = __bfloat162float(p.q[grow * D + lane * E + e]);
+    acc[e] = 0.f;
+  }
+  const bf16* kc = static_cast<const bf16*>(p.tb.k_cache);
+  const bf16* vc = static_cast<const bf16*>(p.tb.v_cache);
+  float m = -INFINITY, l = 0.f;
+  const int L = si.P + si.n;
+  for (int j = 0; j < L; ++j) {
+    const int rel = j - si.P;
+    if (rel >= 0 && !((s_anc[4 * node + (rel >> 5)] >> (rel & 31)) & 1u)) continue;
+    const long long off = kv_row_elem_offset(p.tb, b, j) + (long long)g * D + lane * E;
+    float dot = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) dot += qv[e] * __bfloat162float(kc[off + e]);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, s);
+    const float s2 = dot * p.scale_log2;
+    const float m_new = fmaxf(m, s2);
+    const float corr = exp2f(m - m_new);
+    const float pj = exp2f(s2 - m_new);
+    l = l * corr + pj;
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] = acc[e] * corr + pj * __bfloat162float(vc[off + e]);
+    m = m_new;
+  }
+#pragma unroll
+  for (int e = 0; e < E; ++e) orow[e] = __float2bfloat16(acc[e] / l);
+  if (p.lse && lane == 0) p.lse[grow] = (m + log2f(l)) * kLn2;
+}
+
+// ----------------------------------------------------------------------------------------------
+// Tensor-core (mma.sync) flash-decode kernel.
+// ----------------------------------------------------------------------------------------------
+
+constexpr int BM = 128;       // query rows per CTA (8 warps x 16 rows)
+constexpr int BN = 64;        // keys per pipeline stage
+constexpr int NTHREADS = 256;
+constexpr int STAGES = 3;
+
+__device__ inline void cp_async_16(void* smem_dst, const void* gmem_src, int src_bytes) {
+  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(gmem_src), "r"(src_bytes));
+}
+__device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ inline void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+__device__ inline void ldmatrix_x4(uint32_t (&r)[4], const void* smem_src) {
+  const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(smem_src));
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(a));
+}
+__device__ inline void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_src) {
+  const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(smem_src));
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(a));
+}
+__device__ inline void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ inline float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ inline uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// 64 visibility bits of one row for the keys [rel0, rel0 + 64) counted from the first tree slot:
+// keys before the tree (rel < 0) are prefix and visible, 0 <= rel < 128 follow the ancestor mask,
+// later keys do not exist.  rel0 is uniform over the CTA, so the branches do not diverge.
+__device__ inline uint64_t visibility_window(const uint32_t (&a)[4], int rel0) {
+  const uint64_t lo = (uint64_t)a[0] | ((uint64_t)a[1] << 32);
+  const uint64_t hi = (uint64_t)a[2] | ((uint64_t)a[3] << 32);
+  if (rel0 <= -64) return ~0ull;
+  if (rel0 < 0) return (lo << (-rel0)) | ((1ull << (-rel0)) - 1ull);
+  if (rel0 == 0) return lo;
+  if (rel0 < 64) return (lo >> rel0) | (hi << (64 - rel0));
+  if (rel0 == 64) return hi;
+  if (rel0 < 128) return hi >> (rel0 - 64);
+  return 0ull;
+}
+
+template <int D>
+constexpr size_t attn_mma_smem_bytes() {
+  return 2560 + (size_t)BM * D * 2 + 2 * (size_t)STAGES * BN * D * 2;
+}
+
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams p) {
+  constexpr int CH = D / 8;       // 16-byte chunks per row
+  constexpr int KSTEPS = D / 16;  // MMA k-steps of Q.K^T
+  constexpr int DT = D / 8;       // 8-wide column tiles of the output
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint32_t* s_anc = reinterpret_cast<uint32_t*>(smem);
+  int* s_parent = reinterpret_cast<int*>(smem + 2048);
+  bf16* s_q = reinterpret_cast<bf16*>(smem + 2560);
+  bf16* s_k = s_q + BM * D;
+  bf16* s_v = s_k + STAGES * BN * D;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int split = blockIdx.x;
+  const int Hkv = p.tb.n_kv_heads, Hq = p.tb.n_q_heads, G = p.G;
+  const int g = blockIdx.y % Hkv, tile = blockIdx.y / Hkv;
+  const int b = blockIdx.z;
+
+  const SeqPlan sp = plan_sequence(p, b, split == 0 && blockIdx.y == 0, s_parent, s_anc);
+  const SeqInfo& si = sp.info;
+  const int rows_total = si.nq * G;
+  const int row0 = tile * BM;
+  if (!sp.can_write || row0 >= rows_total) return;
+  const long long rows_all = (long long)p.total_q * Hq;
+
+  // This thread's two accumulator rows: r_lo = warp*16 + lane/4 and r_lo + 8.
+  int row_l[2];
+  bool row_ok[2];
+  long long grow[2];
+  uint32_t anc[2][4];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    row_l[i] = row0 + warp * 16 + (lane >> 2) + 8 * i;
+    row_ok[i] = row_l[i] < rows_total;
+    const int node_l = row_ok[i] ? row_l[i] / G : 0;
+    const int hh = row_ok[i] ? row_l[i] - node_l * G : 0;
+    grow[i] = ((long long)(si.q_off + node_l) * Hq + g * G + hh);
+    const int node = si.q0 + node_l;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) anc[i][w] = (row_ok[i] && sp.compute) ? s_anc[4 * node + w] : 0u;
+  }
+
+  const int L = si.P + si.n;
+  const int T = ceil_div(L, BN);
+  const int tps = ceil_div(T, p.num_splits);
+  const int t_begin = split * tps;
+  const int t_end = min(T, t_begin + tps);
+  const int n_tiles = sp.compute ? max(0, t_end - t_begin) : 0;
+
+  if (n_tiles == 0) {
+    // Nothing visible from this chunk: an empty partial, or zeros when there is no merge.
+    if (p.num_splits == 1) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (!row_ok[i]) continue;
+        for (int c = (lane & 3) * 2; c < D; c += 8)
+          *reinterpret_cast<uint32_t*>(p.out + grow[i] * D + c) = 0u;
+        if (p.lse && (lane & 3) == 0) p.lse[grow[i]] = 0.f;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+        if (row_ok[i] && (lane & 3) == 0) p.part_lse[split * rows_all + grow[i]] = -INFINITY;
+    }
+    return;
+  }
+
+  const bf16* kc = static_cast<const bf16*>(p.tb.k_cache) + (long long)g * D;
+  const bf16* vc = static_cast<const bf16*>(p.tb.v_cache) + (long long)g * D;
+
+  auto load_kv_tile = [&](int tile_idx, int stage) {
+    bf16* dk = s_k + stage * BN * D;
+    bf16* dv = s_v + stage * BN * D;
+#pragma unroll
+    for (int i = 0; i < BN * CH / NTHREADS; ++i) {
+      const int c = tid + i * NTHREADS;
+      const int r = c / CH, ch = c % CH;
+      const int j = tile_idx * BN + r;
+      const bool valid = j < L;
+      const long long off = valid ? kv_row_elem_offset(p.tb, b, j) + ch * 8 : 0;
+      const int so = r * D + ((ch ^ (r & 7)) * 8);
+      cp_async_16(dk + so, kc + off, valid ? 16 : 0);
+      cp_async_16(dv + so, vc + off, valid ? 16 : 0);
+    }
+  };
+
+  // Q tile -> shared memory (rows beyond the sequence's rows are zero-filled).
+#pragma unroll
+  for (int i = 0; i < BM * CH / NTHREADS; ++i) {
+    const int c = tid + i * NTHREADS;
+    const int r = c / CH, ch = c % CH;
+    const int R = row0 + r;
+    const bool valid = R < rows_total;
+    const int node_l = valid ? R / G : 0;
+    const int hh = valid ? R - node_l * G : 0;
+    const long long off = ((long long)(si.q_off + node_l) * Hq + g * G + hh) * D + ch * 8;
+    cp_async_16(s_q + r * D + ((ch ^ (r & 7)) * 8), p.q + (valid ? off : 0), valid ? 16 : 0);
+  }
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; ++s) {
+    if (s < n_tiles) load_kv_tile(t_begin + s, s);
+    cp_async_commit();
+  }
+
+  uint32_t qf[KSTEPS][4];
+  float o_acc[DT][4];
+#pragma unroll
+  for (int d = 0; d < DT; ++d)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o_acc[d][e] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+
+  for (int it = 0; it < n_tiles; ++it) {
+    cp_async_wait<STAGES - 2>();
+    __syncthreads();
+    if (it + STAGES - 1 < n_tiles) load_kv_tile(t_begin + it + STAGES - 1, (it + STAGES - 1) % STAGES);
+    cp_async_commit();
+
+    if (it == 0) {
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        const int r = warp * 16 + (lane & 15);
+        const int ch = 2 * ks + (lane >> 4);
+        ldmatrix_x4(qf[ks], s_q + r * D + ((ch ^ (r & 7)) * 8));
+      }
+    }
+    const bf16* sk = s_k + (it % STAGES) * BN * D;
+    const bf16* sv = s_v + (it % STAGES) * BN * D;
+
+    // S = Q K^T for 16 rows x 64 keys
+    float s_acc[BN / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < BN / 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s_acc[nt][e] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) {
+#pragma unroll
+      for (int np = 0; np < BN / 16; ++np) {
+        uint32_t kb[4];
+        const int r = np * 16 + (lane & 7) + ((lane >> 4) << 3);
+        const int ch = 2 * ks + ((lane >> 3) & 1);
+        ldmatrix_x4(kb, sk + r * D + ((ch ^ (r & 7)) * 8));
+        mma_bf16_16816(s_acc[2 * np], qf[ks], kb[0], kb[1]);
+        mma_bf16_16816(s_acc[2 * np + 1], qf[ks], kb[2], kb[3]);
+      }
+    }
+
+    // scale, tree mask (only tiles that reach past the prefix), online softmax
+    const int key0 = (t_begin + it) * BN;
+    const bool need_mask = key0 + BN > si.P;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      // bit c of `win`: is key key0 + (lane%4)*2 + c visible to this row
+      const uint64_t win = need_mask ? visibility_window(anc[i], key0 - si.P) >> ((lane & 3) * 2) : ~0ull;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          float s2 = s_acc[nt][2 * i + e] * p.scale_log2;
+          if (need_mask) s2 = ((win >> (nt * 8 + e)) & 1ull) ? s2 : -INFINITY;
+          s_acc[nt][2 * i + e] = s2;
+          mx = fmaxf(mx, s2);
+        }
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m_run[i], mx);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float corr = fast_exp2(m_run[i] - m_use);
+      m_run[i] = m_new;
+      l_run[i] *= corr;
+#pragma unroll
+      for (int d = 0; d < DT; ++d) {
+        o_acc[d][2 * i] *= corr;
+        o_acc[d][2 * i + 1] *= corr;
+      }
+      float ls = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float pe = fast_exp2(s_acc[nt][2 * i + e] - m_use);
+          s_acc[nt][2 * i + e] = pe;
+          ls += pe;
+        }
+      }
+      l_run[i] += ls;
+    }
+
+    // O += P V
+#pragma unroll
+    for (int kk = 0; kk < BN / 16; ++kk) {
+      uint32_t pa[4];
+      pa[0] = pack_bf16(s_acc[2 * kk][0], s_acc[2 * kk][1]);
+      pa[1] = pack_bf16(s_acc[2 * kk][2], s_acc[2 * kk][3]);
+      pa[2] = pack_bf16(s_acc[2 * kk + 1][0], s_acc[2 * kk + 1][1]);
+      pa[3] = pack_bf16(s_acc[2 * kk + 1][2], s_acc[2 * kk + 1][3]);
+#pragma unroll
+      for (int dp = 0; dp < D / 16; ++dp) {
+        uint32_t vb[4];
+        const int r = kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+        const int ch = 2 * dp + (lane >> 4);
+        ldmatrix_x4_trans(vb, sv + r * D + ((ch ^ (r & 7)) * 8));
+        mma_bf16_16816(o_acc[2 * dp], pa, vb[0], vb[1]);
+        mma_bf16_16816(o_acc[2 * dp + 1], pa, vb[2], vb[3]);
+      }
+    }
+  }
+  cp_async_wait<0>();
+
+  // epilogue
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    float l = l_run[i];
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    if (!row_ok[i]) continue;
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const float lse2 = l > 0.f ? m_run[i] + log2f(l) : -INFINITY;
+    const int c0 = (lane & 3) * 2;
+    if (p.num_splits == 1) {
+      bf16* orow = p.out + grow[i] * D;
+#pragma unroll
+      for (int d = 0; d < DT; ++d)
+        *reinterpret_cast<uint32_t*>(orow + d * 8 + c0) =
+            pack_bf16(o_acc[d][2 * i] * inv, o_acc[d][2 * i + 1] * inv);
+      if (p.lse && (lane & 3) == 0) p.lse[grow[i]] = l > 0.f ? lse2 * kLn2 : 0.f;
+    } else {
+      float* orow = p.part_o + (split * rows_all + grow[i]) * D;
+#pragma unroll
+      for (int d = 0; d < DT; ++d)
+        *reinterpret_cast<float2*>(orow + d * 8 + c0) =
+            make_float2(o_acc[d][2 * i] * inv, o_acc[d][2 * i + 1] * inv);
+      if ((lane & 3) == 0) p.part_lse[split * rows_all + grow[i]] = lse2;
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------------------------
+// Merge of split partials: out = sum_s w_s out_s, w_s = 2^(lse_s - M) / sum_s 2^(lse_s - M).
+// One warp per (node, head) row.
+// ----------------------------------------------------------------------------------------------
+
+template <int D>
+__global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
+  constexpr int E = D / 32;
+  const int b = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // Sequences whose lengths are bad still own their rows (zero-filled by the empty partials).
+  const int o = p.tb.node_offsets[b];
+  const int n_raw = p.tb.node_offsets[b + 1] - o;
+  const int q0 = p.q_node_begin ? p.q_node_begin[b] : 0;
+  const int q_off = p.q_offsets ? p.q_offsets[b] : o;
+  const bool rows_ok = n_raw >= 0 && n_raw <= SB_MAX_NODES && n_raw <= p.tb.max_nodes && q0 >= 0 &&
+                       q0 <= n_raw && q_off >= 0 && (long long)q_off + (n_raw - q0) <= p.total_q &&
+                       o >= 0 && (long long)o + n_raw <= p.tb.total_nodes;
+  if (!rows_ok) return;
+  const int Hq = p.tb.n_q_heads;
+  const int rr = blockIdx.x * 8 + warp;
+  if (rr >= (n_raw - q0) * Hq) return;
+  const long long rows_all = (long long)p.total_q * Hq;
+  const long long grow = (long long)q_off * Hq + rr;
+  float M = -INFINITY;
+  for (int s = 0; s < p.num_splits; ++s) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
+  float acc[E];
+#pragma unroll
+  for (int e = 0; e < E; ++e) acc[e] = 0.f;
+  float denom = 0.f;
+  if (M != -INFINITY) {
+    for (int s = 0; s < p.num_splits; ++s) {
+      const float ls = p.part_lse[s * rows_all + grow];
+      if (ls == -INFINITY) continue;  // that chunk saw no key for this row: its O is not written
+      const float w = exp2f(ls - M);
+      denom += w;
+      const float* po = p.part_o + (s * rows_all + grow) * D + lane * E;
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[e] += w * po[e];
+    }
+  }
+  const float inv = denom > 0.f ? 1.f / denom : 0.f;
+  bf16* orow = p.out + grow * D + lane * E;
+#pragma unroll
+  for (int e = 0; e < E; ++e) orow[e] = __float2bfloat16(acc[e] * inv);
+  if (p.lse && lane == 0) p.lse[grow] = denom > 0.f ? (M + log2f(denom)) * kLn2 : 0.f;
+}
+
+// ----------------------------------------------------------------------------------------------
+// Host side
+// ----------------------------------------------------------------------------------------------
+
+static int num_sms() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;
+  }
+  return sms;
+}
+
+static sb_status check_batch(const sb_tree_batch* tb) {
+  if (!tb || tb->batch < 1 || !tb->k_cache || !tb->v_cache || !tb->prefix_len || !tb->node_offsets ||
+      !tb->parent || tb->n_q_heads < 1 || tb->n_kv_heads < 1 || tb->n_q_heads % tb->n_kv_heads != 0 ||
+      tb->total_nodes < 0 || tb->max_kv_len < 1)
+    return SB_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(tb->k_cache) & 15) || (reinterpret_cast<uintptr_t>(tb->v_cache) & 15))
+    return SB_ERR_INVALID_ARG;
+  if (tb->head_dim != 64 && tb->head_dim != 128) return SB_ERR_UNSUPPORTED;
+  if (tb->n_q_heads / tb->n_kv_heads > 16) return SB_ERR_UNSUPPORTED;
+  if (tb->max_nodes < 1 || tb->max_nodes > SB_MAX_NODES) return SB_ERR_UNSUPPORTED;
+  if (tb->page_size < 0) return SB_ERR_INVALID_ARG;
+  if (tb->page_size > 0) {
+    if (tb->page_size < 16 || (tb->page_size & (tb->page_size - 1))) return SB_ERR_UNSUPPORTED;
+    if (!tb->page_table || tb->max_pages < 1 || tb->num_pages < 1) return SB_ERR_INVALID_ARG;
+  } else if (tb->kv_capacity < 1) {
+    return SB_ERR_INVALID_ARG;
+  }
+  return SB_OK;
+}
+
+// KV chunks per (sequence, KV head, row tile) when the caller leaves the choice to us: one wave
+// of CTAs when the batch is small, otherwise chunks of about 16 KV tiles to even out ragged
+// prefix lengths.
+static int choose_splits(const sb_tree_batch* tb, int num_splits) {
+  const int G = tb->n_q_heads / tb->n_kv_heads;
+  const int row_tiles = ceil_div(tb->max_nodes * G, BM);
+  const int max_tiles = ceil_div(tb->max_kv_len, BN);
+  if (num_splits > 0) return num_splits < max_tiles ? num_splits : max_tiles;
+  const long long base = (long long)tb->batch * tb->n_kv_heads * row_tiles;
+  const int sms = num_sms();
+  int s;
+  if (base <= sms) {
+    s = (int)(sms / base);
+  } else {
+    s = max_tiles / 16;
+    if (s > 16) s = 16;
+  }
+  if (s > max_tiles) s = max_tiles;
+  if (s < 1) s = 1;
+  return s;
+}
+
+static size_t workspace_bytes_for(const sb_tree_batch* tb, int total_q, int splits) {
+  if (splits <= 1) return 0;
+  const size_t rows = (size_t)total_q * tb->n_q_heads;
+  const size_t o = (size_t)splits * rows * tb->head_dim * sizeof(float);
+  const size_t l = (size_t)splits * rows * sizeof(float);
+  return ((o + 255) & ~(size_t)255) + ((l + 255) & ~(size_t)255);
+}
+
+}  // namespace sb
+
+extern "C" size_t sb_tree_attention_workspace_bytes(const sb_tree_batch* tb, int32_t total_q,
+                                                    int32_t num_splits) {
+  if (sb::check_batch(tb) != SB_OK || total_q < 0 || num_splits < 0) return 0;
+  return sb::workspace_bytes_for(tb, total_q, sb::choose_splits(tb, num_splits));
+}
+
+extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q_node_begin,
+                                       const int32_t* q_offsets, int32_t total_q, const void* q, void* out,
+                                       float* lse, float scale, int32_t num_splits, void* workspace,
+                                       size_t workspace_bytes, int32_t* status, void* stream) {
+  using namespace sb;
+  sb_status st = check_batch(tb);
+  if (st != SB_OK) return st;
+  if (!q || !out || !status || total_q < 1 || num_splits < 0 || !(scale >= 0.f)) return SB_ERR_INVALID_ARG;
+  if (q_node_begin && !q_offsets) return SB_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+    return SB_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int D = tb->head_dim;
+
+  AttnParams p;
+  p.tb = *tb;
+  p.q_node_begin = q_node_begin;
+  p.q_offsets = q_offsets;
+  p.total_q = total_q;
+  p.q = static_cast<const bf16*>(q);
+  p.out = static_cast<bf16*>(out);
+  p.lse = lse;
+  p.scale_log2 = (scale > 0.f ? scale : 1.0f / sqrtf((float)D)) * 1.4426950408889634f;
+  p.status = status;
+  p.G = tb->n_q_heads / tb->n_kv_heads;
+  p.part_o = nullptr;
+  p.part_lse = nullptr;
+
+  const char* impl = getenv("SB_ATTN_IMPL");
+  if (impl && strcmp(impl, "simple") == 0) {
+    p.num_splits = 1;
+    dim3 grid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);
+    if (D == 64) attn_simple_kernel<64><<<grid, 256, 0, cs>>>(p);
+    else attn_simple_kernel<128><<<grid, 256, 0, cs>>>(p);
+    return launch_check();
+  }
+
+  const int splits = choose_splits(tb, num_splits);
+  p.num_splits = splits;
+  if (splits > 1) {
+    const size_t need = workspace_bytes_for(tb, total_q, splits);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255))
+      return SB_ERR_WORKSPACE;
+    const size_t rows = (size_t)total_q * tb->n_q_heads;
+    const size_t o = ((size_t)splits * rows * D * sizeof(float) + 255) & ~(size_t)255;
+    p.part_o = static_cast<float*>(workspace);
+    p.part_lse = reinterpret_cast<float*>(static_cast<char*>(workspace) + o);
+  }
+  const int row_tiles = ceil_div(tb->max_nodes * p.G, BM);
+  dim3 grid(splits, row_tiles * tb->n_kv_heads, tb->batch);
+  if (grid.y > 65535 || grid.z > 65535) return SB_ERR_UNSUPPORTED;
+  if (D == 64) {
+    static bool attr64 = false;
+    if (!attr64) {
+      if (cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)attn_mma_smem_bytes<64>()) != cudaSuccess)
+        return SB_ERR_CUDA;
+      attr64 = true;
+    }
+    attn_mma_kernel<64><<<grid, NTHREADS, attn_mma_smem_bytes<64>(), cs>>>(p);
+  } else {
+    static bool attr128 = false;
+    if (!attr128) {
+      if (cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)attn_mma_smem_bytes<128>()) != cudaSuccess)
+        return SB_ERR_CUDA;
+      attr128 = true;
+    }
+    attn_mma_kernel<128><<<grid, NTHREADS, attn_mma_smem_bytes<128>(), cs>>>(p);
+  }
+  st = launch_check();
+  if (st != SB_OK || splits == 1) return st;
+  dim3 mgrid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);
+  if (D == 64) attn_merge_kernel<64><<<mgrid, 256, 0, cs>>>(p);
+  else attn_merge_kernel<128><<<mgrid, 256, 0, cs>>>(p);
+  return launch_check();
+}

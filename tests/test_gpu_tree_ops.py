@@ -1,0 +1,275 @@
+"""GPU parity of sb_verify_accept, sb_tree_expand and sb_kv_compact against the CPU oracle, through
+the C ABI.  Everything here is integer / byte work: the comparison is bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_07243_b200 import binding as sb
+from paper_2605_07243_b200 import device_inputs as dev
+from paper_2605_07243_b200 import workloads as W
+
+from gpu_helpers import require_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+# ---- verify / accept ----------------------------------------------------------------------------------
+
+def _logits_tensor(logits):
+    if logits.dtype == np.uint16:
+        return dev.bf16_tensor(logits)
+    return torch.from_numpy(logits).cuda()
+
+
+def _gpu_accept(case, vocab=None):
+    r = sb.sb_verify_accept(_logits_tensor(case.logits), dev.i32_tensor(case.node_offsets),
+                            dev.i32_tensor(case.parent), dev.i32_tensor(case.tok), case.max_depth,
+                            vocab=vocab)
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in r.items()}
+
+
+def _check_accept(case, vocab=None):
+    got = _gpu_accept(case, vocab)
+    ref = oracle.verify_accept(case.logits, case.node_offsets, case.parent, case.tok, case.max_depth,
+                               vocab=vocab)
+    for key in ("status", "amax", "accept_len", "path_nodes", "out_tokens", "bonus"):
+        np.testing.assert_array_equal(got[key], ref[key], err_msg=key)
+    return got
+
+
+def test_accept_config1_tiny():
+    _, ver = W.config1_tiny()
+    got = _check_accept(ver)
+    np.testing.assert_array_equal(got["accept_len"], ver.planted_len)
+    np.testing.assert_array_equal(got["bonus"], ver.planted_bonus)
+
+
+@pytest.mark.parametrize("accept_len", range(0, 9))
+def test_accept_config2_bf16_full_vocab(accept_len):
+    ver = W.config2_logits(accept_len=accept_len)
+    got = _check_accept(ver)
+    assert got["accept_len"][0] == ver.planted_len[0]
+    assert got["bonus"][0] == ver.planted_bonus[0]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("vocab", [1, 7, 1000, 4099, 32000])
+def test_accept_ragged_batches_vocab_sizes(dtype, vocab):
+    rng = W.rng_for(60 + vocab)
+    parents = [W.random_tree(rng, int(n), 10) for n in (1, 96, 33, 128, 2)]
+    if vocab < 200:
+        # a tiny vocabulary cannot hold distinct sibling tokens: draw tokens directly, many ties
+        total = sum(len(p) for p in parents)
+        x = np.round(rng.standard_normal((total, vocab), dtype=np.float32))
+        case = W.VerifyCase(W.f32_to_bf16_bits(x) if dtype == "bf16" else x,
+                            rng.integers(0, vocab, total).astype(np.int32),
+                            np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32),
+                            np.concatenate(parents), 10, None, None, None)
+    else:
+        case = W.make_verify_case(rng, parents=parents, vocab=vocab, dtype=dtype, max_depth=10)
+    _check_accept(case)
+
+
+def test_accept_row_stride_padding_nan_inf_and_ties():
+    rng = W.rng_for(61)
+    parents = [W.random_tree(rng, 20, 5)]
+    x = np.round(rng.standard_normal((20, 1003 + 5), dtype=np.float32) * 2)   # coarse: many ties
+    x[:, 1003:] = 1e9                       # padding beyond vocab must be ignored
+    x[3, :1003] = np.nan                     # all-NaN row -> id 0
+    x[4, 10] = np.nan
+    x[5, 77] = np.inf
+    x[6, :1003] = -np.inf
+    x[7, :1003] = 0.0
+    x[7, 5] = -0.0
+    case = W.VerifyCase(x, rng.integers(0, 1003, 20).astype(np.int32), np.asarray([0, 20], np.int32),
+                        parents[0], 5, None, None, None)
+    got = _check_accept(case, vocab=1003)
+    assert got["amax"][3] == 0 and got["amax"][5] == 77 and got["amax"][6] == 0 and got["amax"][7] == 0
+
+
+def test_accept_depth_cut_duplicates_and_invalid_trees():
+    rng = W.rng_for(62)
+    # duplicate sibling tokens and a tiny alphabet -> many equally long accepted paths
+    parents = [W.random_tree(rng, 40, 12), np.asarray([-1, -1, 0], np.int32), W.chain_tree(30),
+               np.asarray([-1, 0, 3, 1], np.int32)]
+    total = sum(len(p) for p in parents)
+    x = np.zeros((total, 3), np.float32)
+    choice = rng.integers(0, 3, total)
+    x[np.arange(total), choice] = 1.0
+    case = W.VerifyCase(x, rng.integers(0, 3, total).astype(np.int32),
+                        np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32),
+                        np.concatenate(parents), 4, None, None, None)
+    case.tok[43:73] = 1                      # the chain accepts everything: cut at max_depth
+    x[43:73] = [0, 1, 0]
+    got = _check_accept(case)
+    assert list(got["status"]) == [0, 4, 0, 4]
+    assert got["accept_len"][2] == 4
+
+
+def test_accept_config4_and_5_full_size():
+    _, ver4 = W.config4_batched()
+    got = _check_accept(ver4)
+    np.testing.assert_array_equal(got["accept_len"], ver4.planted_len)
+    _, ver5 = W.config5_long()
+    got = _check_accept(ver5)
+    np.testing.assert_array_equal(got["accept_len"], ver5.planted_len)
+    np.testing.assert_array_equal(got["bonus"], ver5.planted_bonus)
+
+
+# ---- expansion -------------------------------------------------------------------------------------------
+
+def _gpu_expand(case, vocab=None):
+    budget = case.node_budget
+    n0 = 0 if case.tree is None else len(case.tree["tok"])
+    tree = {k: torch.full((budget,), -1, dtype=torch.int32, device="cuda")
+            for k in ("tok", "parent", "depth", "node_row", "node_rank")}
+    if case.tree is not None:
+        for k in tree:
+            tree[k][:n0] = dev.i32_tensor(case.tree[k])
+    tree["n_nodes"] = torch.tensor([n0], dtype=torch.int32, device="cuda")
+    topk_tok, topk_val, status = sb.sb_tree_expand(
+        torch.from_numpy(case.scores).cuda(), case.block_k, torch.from_numpy(case.bucket).cuda(),
+        case.bmap, dev.i32_tensor(case.start_parent), budget, tree, vocab=vocab)
+    torch.cuda.synchronize()
+    out = {k: v.cpu().numpy() for k, v in tree.items()}
+    out.update(topk_tok=topk_tok.cpu().numpy(), topk_val=topk_val.cpu().numpy(),
+               status=int(status.cpu().numpy()[0]))
+    out["n_nodes"] = int(out["n_nodes"][0])
+    return out
+
+
+def _check_expand(case, vocab=None):
+    got = _gpu_expand(case, vocab)
+    ref = oracle.tree_expand(case.scores, case.block_k, case.bucket, case.bmap, case.start_parent,
+                             case.node_budget, tree=case.tree, vocab=vocab)
+    assert got["status"] == ref["status"]
+    np.testing.assert_array_equal(got["topk_tok"], ref["topk_tok"])
+    np.testing.assert_array_equal(got["topk_val"], ref["topk_val"])
+    if ref["status"] == 0:
+        assert got["n_nodes"] == ref["n_nodes"]
+        for k in ("tok", "parent", "depth", "node_row", "node_rank"):
+            np.testing.assert_array_equal(got[k], ref[k], err_msg=k)
+    return got
+
+
+def test_expand_config3_full_vocab():
+    _, exp = W.config3_drafter()
+    got = _check_expand(exp)
+    assert got["n_nodes"] > 12
+
+
+@pytest.mark.parametrize("bmap", [[2, 4, 10, 0], [2, 4, 6, 4], [16, 16, 16, 16], [0, 0, 0, 0]])
+@pytest.mark.parametrize("vocab", [5, 1000, 32000])
+def test_expand_printed_maps_and_vocab_sizes(bmap, vocab):
+    rng = W.rng_for(70 + vocab)
+    case = W.make_expand_case(rng, n_starts=3, block_k=4, vocab=vocab, bmap=bmap, node_budget=60,
+                              existing_parent=W.random_tree(rng, 5, 3), tie_rows=6)
+    _check_expand(case)
+
+
+def test_expand_ties_nan_inf_padding_and_budget():
+    rng = W.rng_for(71)
+    case = W.make_expand_case(rng, n_starts=2, block_k=4, vocab=2000 + 3, bmap=[3, 5, 10, 2],
+                              node_budget=17)
+    s = case.scores
+    s[:, 2000:] = 1e9                        # padding columns beyond vocab
+    s[0, :2000] = 1.0                        # all equal: ids 0..15 in order
+    s[1, :2000] = np.nan                     # all NaN: treated as -inf, ids 0..15
+    s[2, ::2] = np.inf
+    s[3, :2000] = np.round(s[3, :2000])      # heavy ties
+    s[4, :1990] = -np.inf                    # only 10 finite values
+    got = _check_expand(case, vocab=2000)
+    assert list(got["topk_tok"][0]) == list(range(16))
+    assert got["n_nodes"] == 17
+
+
+def test_expand_device_argument_errors():
+    rng = W.rng_for(72)
+    case = W.make_expand_case(rng, n_starts=1, block_k=4, vocab=100, bmap=[2, 4, 10, 0], node_budget=20)
+    case.bucket[2] = 9
+    assert _check_expand(case)["status"] == 1
+    case.bucket[2] = 1
+    case.start_parent[0] = 3                 # no such node
+    assert _check_expand(case)["status"] == 1
+
+
+# ---- compaction ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("page_size", [0, 64, 16])
+def test_kv_compact_matches_oracle(page_size):
+    rng = W.rng_for(80 + page_size)
+    parents = [W.random_tree(rng, 60, 8), W.chain_tree(40), W.random_tree(rng, 9, 4), W.chain_tree(3)]
+    L = 3
+    case = W.make_attn_case(rng, parents=parents, prefix_lens=[250, 64, 1, 0], n_q_heads=32, n_kv_heads=8,
+                            head_dim=128, page_size=page_size)
+    layer_elems = case.k.size
+    k_all = rng.integers(0, 65536, (L,) + case.k.shape).astype(np.uint16)
+    v_all = rng.integers(0, 65536, (L,) + case.v.shape).astype(np.uint16)
+    max_depth = 32
+    paths = np.full((4, max_depth + 1), -1, np.int32)
+    alen = np.zeros(4, np.int32)
+    # sequence 0: a real root-to-node path; 1: the full chain (identity moves only, 32 deep);
+    # 2: root only; 3: an invalid path (not increasing)
+    end = int(np.argmax(W.tree_depths(parents[0])))
+    p0 = [end]
+    while parents[0][p0[-1]] >= 0:
+        p0.append(int(parents[0][p0[-1]]))
+    p0 = p0[::-1]
+    paths[0, :len(p0)] = p0
+    alen[0] = len(p0) - 1
+    paths[1, :33] = np.arange(33)
+    alen[1] = 32
+    paths[2, 0] = 0
+    paths[3, :3] = [0, 2, 1]
+    alen[3] = 2
+    tb = dev.tree_batch(case, k=dev.bf16_tensor(k_all), v=dev.bf16_tensor(v_all))
+    new_len, status = sb.sb_kv_compact(tb, L, layer_elems, dev.i32_tensor(paths), dev.i32_tensor(alen),
+                                       max_depth)
+    torch.cuda.synchronize()
+    kw = dict(n_kv_heads=8, head_dim=128, n_layers=L, layer_stride_elems=layer_elems, page_size=page_size,
+              max_pages=case.max_pages, num_pages=case.num_pages, kv_capacity=case.kv_capacity,
+              page_table=case.page_table, prefix_len=case.prefix_len, node_offsets=case.node_offsets,
+              path_nodes=paths, accept_len=alen, max_depth=max_depth)
+    ref_k, ref_len, ref_st = oracle.kv_compact(cache=k_all.reshape(-1), **kw)
+    ref_v, _, _ = oracle.kv_compact(cache=v_all.reshape(-1), **kw)
+    np.testing.assert_array_equal(status.cpu().numpy(), ref_st)
+    np.testing.assert_array_equal(new_len.cpu().numpy(), ref_len)
+    assert list(ref_st) == [0, 0, 0, 4]
+    got_k = tb.k_cache.view(torch.int16).cpu().numpy().view(np.uint16).reshape(k_all.shape)
+    got_v = tb.v_cache.view(torch.int16).cpu().numpy().view(np.uint16).reshape(v_all.shape)
+    ref_k, ref_v = ref_k.reshape(k_all.shape), ref_v.reshape(v_all.shape)
+    # compare the live range [0, new_len) of every sequence, plus everything outside the trees
+    for b in range(4):
+        for pos in range(int(ref_len[b])):
+            sl = W.kv_slot(case, b, pos)
+            np.testing.assert_array_equal(got_k[(slice(None),) + sl], ref_k[(slice(None),) + sl])
+            np.testing.assert_array_equal(got_v[(slice(None),) + sl], ref_v[(slice(None),) + sl])
+    # the in-place result equals the out-of-place gather everywhere in this construction:
+    # a slot beyond new_len is never written by either
+    np.testing.assert_array_equal(got_k, ref_k)
+    np.testing.assert_array_equal(got_v, ref_v)
+
+
+def test_accept_then_compact_chain_on_device():
+    """sb_verify_accept's device outputs feed sb_kv_compact without a host round trip."""
+    par = W.config2_tree()
+    ver = W.config2_logits(accept_len=5, vocab=4096, par=par)
+    case = W.config2_verify_layer(prefix=200, par=par)
+    r = sb.sb_verify_accept(dev.bf16_tensor(ver.logits), dev.i32_tensor(ver.node_offsets),
+                            dev.i32_tensor(ver.parent), dev.i32_tensor(ver.tok), 8)
+    tb = dev.tree_batch(case)
+    new_len, status = sb.sb_kv_compact(tb, 1, 0, r["path_nodes"], r["accept_len"], 8)
+    torch.cuda.synchronize()
+    assert int(new_len[0]) == 200 + 5 + 1 and int(status[0]) == 0
+    path = r["path_nodes"].cpu().numpy()[0, :6]
+    assert list(path) == ver.planted_path[0]
+    got_k = tb.k_cache.view(torch.int16).cpu().numpy().view(np.uint16)
+    for j, node in enumerate(path):
+        np.testing.assert_array_equal(got_k[0, 200 + j], case.k[0, 200 + node])

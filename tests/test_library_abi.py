@@ -1,0 +1,48 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU, and exports every symbol that
+include/specblock.h declares.  No compute call is made here."""
+import ctypes
+import os
+import re
+
+from paper_2605_07243_b200 import binding, build
+
+
+def _declared_symbols():
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    text = open(os.path.join(root, "include", "specblock.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sb_[a-z_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported():
+    path = build.build()
+    lib = ctypes.CDLL(path)
+    declared = _declared_symbols()
+    assert "sb_tree_attention" in declared and "sb_kv_compact" in declared
+    for name in declared:
+        assert hasattr(lib, name), f"{name} is declared in specblock.h but not exported"
+    assert set(binding.EXPORTED) == set(declared)
+
+
+def test_host_only_entry_points():
+    lib = binding.load()
+    assert binding.sb_version() >= 100
+    assert binding.sb_status_string(0) == "ok"
+    assert binding.sb_status_string(4) == "invalid tree"
+    assert binding.sb_kernel_launch_count() >= 0
+    # workspace queries are host arithmetic
+    assert binding.sb_verify_accept_workspace_bytes(60, 128256) > 0
+    assert binding.sb_tree_expand_workspace_bytes(32, 128256) > 0
+    assert lib.sb_tree_attention_workspace_bytes(None, 1, 0) == 0
+
+
+def test_binding_struct_matches_header_layout():
+    """Field order and natural alignment of the ctypes mirror of sb_tree_batch."""
+    s = binding._TreeBatch
+    names = [f[0] for f in s._fields_]
+    assert names == ["batch", "n_q_heads", "n_kv_heads", "head_dim", "k_cache", "v_cache",
+                     "page_size", "max_pages", "kv_capacity", "num_pages", "total_nodes",
+                     "page_table", "prefix_len", "node_offsets", "parent", "max_nodes",
+                     "max_kv_len"]
+    assert s.k_cache.offset == 16 and s.kv_capacity.offset == 40 and s.page_table.offset == 56
+    assert ctypes.sizeof(s) == 96
