@@ -1,0 +1,219 @@
+"""One SpecBlock draft-and-verify iteration's device steps, chained on a stream (Alg. 1).
+
+`VerifyStep` owns the device buffers of one iteration of an L-layer target model and issues, in
+order: ancestor masks / position ids, the drafter's top-k expansion, tree attention for every
+layer, greedy acceptance, and KV compaction of every layer.  It only sequences calls of the
+C-ABI library (paper_2605_07243_b200.binding); every step runs in the library's kernels.
+
+Two ways to run it:
+  run_device()     all inputs already resident in device memory;
+  run_from_host()  inputs in pinned host memory: copies them in, runs, copies the results out.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as sb
+from . import device_inputs as dev
+
+
+class VerifyStep:
+    def __init__(self, layers: List, verify_case, expand_case=None, device="cuda", num_splits=0,
+                 keep_host=False):
+        """layers: one workloads.AttnCase per target layer (same tree and layout, different Q/K/V);
+        verify_case: workloads.VerifyCase over the same tree; expand_case: optional
+        workloads.ExpandCase (the drafter's batched block forward of this iteration)."""
+        self.device = device
+        self.n_layers = len(layers)
+        c0 = layers[0]
+        self.case0 = c0
+        self.num_splits = num_splits
+        self.max_depth = verify_case.max_depth
+        self.planted_len = verify_case.planted_len
+        L = self.n_layers
+        # K/V of all layers in one allocation each: layer l starts layer_stride elements after l-1
+        self.layer_stride = int(c0.k.size)
+        self.host = {}
+        k_all = np.stack([c.k for c in layers])
+        v_all = np.stack([c.v for c in layers])
+        q_all = np.stack([c.q for c in layers])
+        self.k_all = dev.bf16_tensor(k_all, device)
+        self.v_all = dev.bf16_tensor(v_all, device)
+        self.q_all = dev.bf16_tensor(q_all, device)
+        self.out_all = torch.empty_like(self.q_all)
+        self.lse_all = torch.empty((L, c0.total_q, c0.n_q_heads), dtype=torch.float32, device=device)
+        self.tb = dev.tree_batch(c0, device, k=self.k_all[0], v=self.v_all[0])
+        self.kw = {}
+        if c0.q_node_begin is not None:
+            self.kw = dict(q_node_begin=dev.i32_tensor(c0.q_node_begin, device),
+                           q_offsets=dev.i32_tensor(c0.q_offsets, device))
+        self.scale = float(c0.scale)
+        ws = sb.sb_tree_attention_workspace_bytes(self.tb, c0.total_q, num_splits)
+        self.attn_ws = torch.empty(max(ws, 256), dtype=torch.uint8, device=device)
+        B = c0.batch
+        i32 = dict(dtype=torch.int32, device=device)
+        self.attn_status = torch.empty(B, **i32)
+        self.anc = torch.empty((self.tb.total_nodes, 4), **i32)
+        self.depth = torch.empty(self.tb.total_nodes, **i32)
+        self.anc_status = torch.empty(B, **i32)
+        # verification inputs
+        if verify_case.logits.dtype == np.uint16:
+            self.logits = dev.bf16_tensor(verify_case.logits, device)
+        else:
+            self.logits = torch.from_numpy(verify_case.logits).to(device)
+        self.tok = dev.i32_tensor(verify_case.tok, device)
+        total = self.tb.total_nodes
+        md = self.max_depth
+        self.accept = dict(amax=torch.empty(total, **i32), accept_len=torch.empty(B, **i32),
+                           path_nodes=torch.empty((B, md + 1), **i32),
+                           out_tokens=torch.empty((B, md + 1), **i32), bonus=torch.empty(B, **i32),
+                           status=torch.empty(B, **i32))
+        vws = sb.sb_verify_accept_workspace_bytes(total, self.logits.shape[1])
+        self.accept_ws = torch.empty(max(vws, 256), dtype=torch.uint8, device=device)
+        self.new_len = torch.empty(B, **i32)
+        self.compact_status = torch.empty(B, **i32)
+        # expansion inputs
+        self.expand = None
+        if expand_case is not None:
+            e = expand_case
+            budget = e.node_budget
+            n0 = 0 if e.tree is None else len(e.tree["tok"])
+            tree0 = {k: torch.full((budget,), -1, **i32) for k in ("tok", "parent", "depth", "node_row", "node_rank")}
+            if e.tree is not None:
+                for k in tree0:
+                    tree0[k][:n0] = dev.i32_tensor(e.tree[k], device)
+            R, V = e.scores.shape
+            ews = sb.sb_tree_expand_workspace_bytes(R, V)
+            self.expand = dict(
+                scores=torch.from_numpy(e.scores).to(device), bucket=torch.from_numpy(e.bucket).to(device),
+                bmap=[int(x) for x in e.bmap], start_parent=dev.i32_tensor(e.start_parent, device),
+                budget=budget, block_k=e.block_k, n0=n0, tree0=tree0,
+                tree={k: t.clone() for k, t in tree0.items()},
+                n_nodes=torch.tensor([n0], **i32), n_nodes0=torch.tensor([n0], **i32),
+                topk_tok=torch.empty((R, sb.SB_KMAX), **i32),
+                topk_val=torch.empty((R, sb.SB_KMAX), dtype=torch.float32, device=device),
+                status=torch.empty(1, **i32), ws=torch.empty(max(ews, 256), dtype=torch.uint8, device=device))
+        if keep_host:
+            self._make_host_copies(k_all, v_all, q_all, verify_case, expand_case)
+
+    # ---- pieces ----------------------------------------------------------------------------
+
+    def run_ancestors(self):
+        sb.sb_tree_ancestors(self.tb.node_offsets, self.tb.parent, self.tb.max_nodes, self.anc, self.depth,
+                             self.anc_status)
+
+    def run_expand(self):
+        e = self.expand
+        if e is None:
+            return
+        e["n_nodes"].copy_(e["n_nodes0"])      # the tree arrays restart from the existing nodes
+        tree = dict(e["tree"], n_nodes=e["n_nodes"])
+        sb.sb_tree_expand(e["scores"], e["block_k"], e["bucket"], e["bmap"], e["start_parent"], e["budget"],
+                          tree, workspace=e["ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"],
+                          status=e["status"])
+
+    def run_attention(self, layers=None):
+        for l in range(self.n_layers) if layers is None else layers:
+            sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,
+                                 num_splits=self.num_splits, workspace=self.attn_ws, status=self.attn_status,
+                                 k_cache=self.k_all[l], v_cache=self.v_all[l], **self.kw)
+
+    def run_accept(self):
+        sb.sb_verify_accept(self.logits, self.tb.node_offsets, self.tb.parent, self.tok, self.max_depth,
+                            workspace=self.accept_ws, out=self.accept)
+
+    def run_compact(self):
+        sb.sb_kv_compact(self.tb, self.n_layers, self.layer_stride, self.accept["path_nodes"],
+                         self.accept["accept_len"], self.max_depth, self.new_len, self.compact_status)
+
+    # ---- whole step --------------------------------------------------------------------------
+
+    def run_device(self):
+        """The whole iteration with inputs resident in device memory (enqueue only)."""
+        self.run_ancestors()
+        self.run_expand()
+        self.run_attention()
+        self.run_accept()
+        self.run_compact()
+
+    def launches_per_step(self) -> int:
+        before = sb.sb_kernel_launch_count()
+        self.run_device()
+        return sb.sb_kernel_launch_count() - before
+
+    def _make_host_copies(self, k_all, v_all, q_all, verify_case, expand_case):
+        def pin(t):
+            return t.cpu().pin_memory()
+        h = self.host
+        h["k"], h["v"], h["q"] = pin(self.k_all), pin(self.v_all), pin(self.q_all)
+        h["parent"], h["node_offsets"] = pin(self.tb.parent), pin(self.tb.node_offsets)
+        h["prefix_len"], h["logits"], h["tok"] = pin(self.tb.prefix_len), pin(self.logits), pin(self.tok)
+        if self.tb.page_table is not None:
+            h["page_table"] = pin(self.tb.page_table)
+        if self.expand is not None:
+            h["scores"], h["bucket"] = pin(self.expand["scores"]), pin(self.expand["bucket"])
+            h["start_parent"] = pin(self.expand["start_parent"])
+        h["out"] = torch.empty(self.out_all.shape, dtype=self.out_all.dtype).pin_memory()
+        h["lse"] = torch.empty(self.lse_all.shape, dtype=torch.float32).pin_memory()
+        h["res"] = {k: torch.empty(t.shape, dtype=t.dtype).pin_memory() for k, t in self.accept.items()}
+        h["new_len"] = torch.empty(self.new_len.shape, dtype=torch.int32).pin_memory()
+
+    def host_bytes(self):
+        """(host->device, device->host) bytes of one run_from_host()."""
+        h = self.host
+        h2d = sum(h[k].numel() * h[k].element_size() for k in
+                  ("k", "v", "q", "parent", "node_offsets", "prefix_len", "logits", "tok", "page_table",
+                   "scores", "bucket", "start_parent") if k in h)
+        d2h = sum(t.numel() * t.element_size() for t in [h["out"], h["lse"], h["new_len"]] +
+                  list(h["res"].values()))
+        return h2d, d2h
+
+    def run_from_host(self):
+        """Inputs in pinned host memory -> device, the whole iteration, results -> pinned host
+        memory.  Enqueue only; synchronise the stream before reading the host results."""
+        h = self.host
+        self.k_all.copy_(h["k"], non_blocking=True)
+        self.v_all.copy_(h["v"], non_blocking=True)
+        self.q_all.copy_(h["q"], non_blocking=True)
+        self.tb.parent.copy_(h["parent"], non_blocking=True)
+        self.tb.node_offsets.copy_(h["node_offsets"], non_blocking=True)
+        self.tb.prefix_len.copy_(h["prefix_len"], non_blocking=True)
+        self.logits.copy_(h["logits"], non_blocking=True)
+        self.tok.copy_(h["tok"], non_blocking=True)
+        if "page_table" in h:
+            self.tb.page_table.copy_(h["page_table"], non_blocking=True)
+        if self.expand is not None:
+            self.expand["scores"].copy_(h["scores"], non_blocking=True)
+            self.expand["bucket"].copy_(h["bucket"], non_blocking=True)
+            self.expand["start_parent"].copy_(h["start_parent"], non_blocking=True)
+        self.run_device()
+        h["out"].copy_(self.out_all, non_blocking=True)
+        h["lse"].copy_(self.lse_all, non_blocking=True)
+        for k, t in self.accept.items():
+            h["res"][k].copy_(t, non_blocking=True)
+        h["new_len"].copy_(self.new_len, non_blocking=True)
+
+    # ---- accounting -------------------------------------------------------------------------
+
+    def algorithmic_bytes(self):
+        """Bytes each part of the step must move at minimum (every input read once, every output
+        written once)."""
+        c0 = self.case0
+        attn_layer = c0.algorithmic_bytes()
+        logits = self.logits.numel() * self.logits.element_size()
+        total = self.tb.total_nodes
+        accept = logits + total * 4 * 3
+        row = c0.n_kv_heads * c0.head_dim * 2
+        parts = dict(attention_per_layer=attn_layer, attention=attn_layer * self.n_layers, accept=accept,
+                     ancestors=total * 4 * 6)
+        if self.expand is not None:
+            s = self.expand["scores"]
+            parts["expand"] = s.numel() * 4 + s.shape[0] * sb.SB_KMAX * 8
+        # accepted path rows (the root stays in place) read + written, K and V, every layer
+        moved = int(np.sum(self.planted_len)) if self.planted_len is not None else 0
+        parts["compact"] = moved * row * 2 * 2 * self.n_layers
+        parts["total"] = sum(v for k, v in parts.items() if k != "attention_per_layer")
+        return parts
