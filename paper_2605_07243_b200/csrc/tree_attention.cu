@@ -5,82 +5,29 @@
 // 128-row tile shares every K/V tile it streams (GQA head packing).  The ancestor sets live in
 // shared memory as one 128-bit mask per node and are applied only to the KV tiles that overlap
 // the tree's cache slots; prefix tiles run unmasked.  The KV range of a (sequence, KV head, row
-// tile) is cut into `num_splits` chunks handled by different CTAs; a second kernel merges the
-// chunks' (out, log-sum-exp) pairs.
+// tile) is cut into `num_splits` chunks handled by different CTAs.  Up to 8 chunk-CTAs form a
+// thread-block cluster and merge their (out, max, sum) triples through distributed shared
+// memory, so for up to 8 chunks nothing but the final result is written; beyond 8 chunks each
+// cluster writes one partial and a second kernel merges the clusters' (out, log-sum-exp) pairs.
 //
 // Kernels in this file
 //   attn_simple_kernel : one warp per query row, fp32 FMA.  Slow, shape-agnostic check path
 //                        (environment SB_ATTN_IMPL=simple selects it).
-//   attn_mma_kernel    : flash-decode with bf16 tensor-core MMA (m16n8k16), fp32 accumulate,
-//                        3-stage cp.async K/V pipeline in XOR-swizzled shared memory.
-//   attn_merge_kernel  : log-sum-exp merge of the split partials.
+//   attn_mma_kernel    : flash-decode with bf16 mma.sync (m16n8k16), fp32 accumulate, 3-stage cp.async
+//                        K/V pipeline in XOR-swizzled shared memory (SB_ATTN_IMPL=mma selects it).
+//   (default)          : the tcgen05/TMEM kernel in tree_attention_tc.cu.
+//   attn_merge_kernel  : log-sum-exp merge of the clusters' partials (only beyond 8 chunks).
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
-#include "common.cuh"
+#include "attention_common.cuh"
 
 namespace sb {
 
-typedef __nv_bfloat16 bf16;
-
-struct AttnParams {
-  sb_tree_batch tb;
-  const int* q_node_begin;
-  const int* q_offsets;
-  int total_q;
-  const bf16* q;
-  bf16* out;
-  float* lse;
-  float scale_log2;  // softmax scale * log2(e): scores are kept in the base-2 domain
-  int num_splits;
-  float* part_o;    // [num_splits][total_q*Hq][D] normalised partial outputs
-  float* part_lse;  // [num_splits][total_q*Hq]    base-2 log-sum-exp of each partial
-  int* status;
-  int G;            // query heads per KV head
-};
-
-constexpr float kLn2 = 0.6931471805599453f;
-
-// What a CTA may do for its sequence after the shape checks.
-struct SeqPlan {
-  SeqInfo info;
-  bool can_write;  // the sequence's output rows are inside q/out
-  bool compute;    // tree and lengths are valid: run the attention
-};
-
-// Must be called by every thread of the CTA (contains barriers).  `designated` CTAs (one per
-// sequence) also scan the page table and publish the sequence's status word.
-__device__ inline SeqPlan plan_sequence(const AttnParams& p, int b, bool designated, int* s_parent,
-                                        uint32_t* s_anc) {
-  SeqPlan sp;
-  sp.info = load_seq_info(p.tb, p.q_node_begin, p.q_offsets, p.total_q, b);
-  int err = sp.info.err;
-  // Which rows may be zero-filled on error: recompute the raw row range.
-  const int o = p.tb.node_offsets[b];
-  const int n_raw = p.tb.node_offsets[b + 1] - o;
-  const int q0 = p.q_node_begin ? p.q_node_begin[b] : 0;
-  const int q_off = p.q_offsets ? p.q_offsets[b] : o;
-  const bool rows_ok = n_raw >= 0 && n_raw <= SB_MAX_NODES && n_raw <= p.tb.max_nodes && q0 >= 0 &&
-                       q0 <= n_raw && q_off >= 0 && (long long)q_off + (n_raw - q0) <= p.total_q &&
-                       o >= 0 && (long long)o + n_raw <= p.tb.total_nodes;
-  sp.can_write = rows_ok;
-  if (rows_ok && err) {  // lengths are bad but the rows exist: keep them for zero-filling
-    sp.info.nq = n_raw - q0;
-    sp.info.q0 = q0;
-    sp.info.q_off = q_off;
-  }
-  const bool tree_ok = build_ancestors_smem(p.tb.parent + (rows_ok ? o : 0), err ? 0 : sp.info.n,
-                                            s_parent, s_anc, nullptr);
-  if (!err && !tree_ok) err = SB_ERR_INVALID_TREE;
-  if (designated) {
-    const bool pages_ok = err ? true : pages_in_pool(p.tb, b, sp.info.P + sp.info.n);
-    if (!err && !pages_ok) err = SB_ERR_BOUNDS;  // reported; reads were clamped into the pool
-    if (threadIdx.x == 0) p.status[b] = err;
-    if (!pages_ok) err = 0;  // other CTAs cannot see this; stay consistent with them
-  }
-  sp.compute = err == 0;
-  return sp;
-}
+// tcgen05 kernel (tree_attention_tc.cu)
+sb_status launch_attn_tc(const AttnParams& p, dim3 grid, int cluster, cudaStream_t cs);
+int attn_tc_max_active_clusters(int D, int cluster);
 
 // ----------------------------------------------------------------------------------------------
 // Simple kernel: one warp per (node, head) row.
@@ -177,31 +124,6 @@ __device__ inline void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uin
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ inline float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ inline uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// 64 visibility bits of one row for the keys [rel0, rel0 + 64) counted from the first tree slot:
-// keys before the tree (rel < 0) are prefix and visible, 0 <= rel < 128 follow the ancestor mask,
-// later keys do not exist.  rel0 is uniform over the CTA, so the branches do not diverge.
-__device__ inline uint64_t visibility_window(const uint32_t (&a)[4], int rel0) {
-  const uint64_t lo = (uint64_t)a[0] | ((uint64_t)a[1] << 32);
-  const uint64_t hi = (uint64_t)a[2] | ((uint64_t)a[3] << 32);
-  if (rel0 <= -64) return ~0ull;
-  if (rel0 < 0) return (lo << (-rel0)) | ((1ull << (-rel0)) - 1ull);
-  if (rel0 == 0) return lo;
-  if (rel0 < 64) return (lo >> rel0) | (hi << (64 - rel0));
-  if (rel0 == 64) return hi;
-  if (rel0 < 128) return hi >> (rel0 - 64);
-  return 0ull;
-}
-
 template <int D>
 constexpr size_t attn_mma_smem_bytes() {
   return 2560 + (size_t)BM * D * 2 + 2 * (size_t)STAGES * BN * D * 2;
@@ -220,7 +142,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
   bf16* s_v = s_k + STAGES * BN * D;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int split = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int S = (int)cluster.num_blocks();   // chunk-CTAs that merge through shared memory
+  const int crank = (int)cluster.block_rank();
+  const int split = blockIdx.x;              // chunk index among num_splits = S * outer
   const int Hkv = p.tb.n_kv_heads, Hq = p.tb.n_q_heads, G = p.G;
   const int g = blockIdx.y % Hkv, tile = blockIdx.y / Hkv;
   const int b = blockIdx.z;
@@ -229,50 +154,27 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
   const SeqInfo& si = sp.info;
   const int rows_total = si.nq * G;
   const int row0 = tile * BM;
+  // Uniform over the cluster (depends on the sequence and the row tile only).
   if (!sp.can_write || row0 >= rows_total) return;
   const long long rows_all = (long long)p.total_q * Hq;
 
-  // This thread's two accumulator rows: r_lo = warp*16 + lane/4 and r_lo + 8.
-  int row_l[2];
-  bool row_ok[2];
-  long long grow[2];
+  // This thread's two accumulator rows: warp*16 + lane/4 and that + 8.
   uint32_t anc[2][4];
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
-    row_l[i] = row0 + warp * 16 + (lane >> 2) + 8 * i;
-    row_ok[i] = row_l[i] < rows_total;
-    const int node_l = row_ok[i] ? row_l[i] / G : 0;
-    const int hh = row_ok[i] ? row_l[i] - node_l * G : 0;
-    grow[i] = ((long long)(si.q_off + node_l) * Hq + g * G + hh);
-    const int node = si.q0 + node_l;
+    const int R = row0 + warp * 16 + (lane >> 2) + 8 * i;
+    const bool ok = R < rows_total && sp.compute;
+    const int node = ok ? si.q0 + R / G : 0;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) anc[i][w] = (row_ok[i] && sp.compute) ? s_anc[4 * node + w] : 0u;
+    for (int w = 0; w < 4; ++w) anc[i][w] = ok ? s_anc[4 * node + w] : 0u;
   }
 
+  // Balanced cut of the sequence's T key tiles into num_splits chunks.
   const int L = si.P + si.n;
   const int T = ceil_div(L, BN);
-  const int tps = ceil_div(T, p.num_splits);
-  const int t_begin = split * tps;
-  const int t_end = min(T, t_begin + tps);
-  const int n_tiles = sp.compute ? max(0, t_end - t_begin) : 0;
-
-  if (n_tiles == 0) {
-    // Nothing visible from this chunk: an empty partial, or zeros when there is no merge.
-    if (p.num_splits == 1) {
-#pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        if (!row_ok[i]) continue;
-        for (int c = (lane & 3) * 2; c < D; c += 8)
-          *reinterpret_cast<uint32_t*>(p.out + grow[i] * D + c) = 0u;
-        if (p.lse && (lane & 3) == 0) p.lse[grow[i]] = 0.f;
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 2; ++i)
-        if (row_ok[i] && (lane & 3) == 0) p.part_lse[split * rows_all + grow[i]] = -INFINITY;
-    }
-    return;
-  }
+  const int t_base = T / p.num_splits, t_rem = T % p.num_splits;
+  const int t_begin = split * t_base + min(split, t_rem);
+  const int n_tiles = sp.compute ? t_base + (split < t_rem ? 1 : 0) : 0;
 
   const bf16* kc = static_cast<const bf16*>(p.tb.k_cache) + (long long)g * D;
   const bf16* vc = static_cast<const bf16*>(p.tb.v_cache) + (long long)g * D;
@@ -295,7 +197,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
 
   // Q tile -> shared memory (rows beyond the sequence's rows are zero-filled).
 #pragma unroll
-  for (int i = 0; i < BM * CH / NTHREADS; ++i) {
+  for (int i = 0; n_tiles > 0 && i < BM * CH / NTHREADS; ++i) {
     const int c = tid + i * NTHREADS;
     const int r = c / CH, ch = c % CH;
     const int R = row0 + r;
@@ -419,33 +321,37 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
     }
   }
   cp_async_wait<0>();
+  __syncthreads();  // every warp is done with the K/V stages: reuse them as the merge buffer
 
-  // epilogue
+  // ---- epilogue: merge the cluster's chunks through (distributed) shared memory -------------
+  // Each CTA parks its unnormalised O tile, row maxima and row sums in its own shared memory;
+  // CTA `crank` of the cluster then reduces rows [crank*rows_per, (crank+1)*rows_per) over all S
+  // CTAs and writes them out.  With S = 1 this is just a coalescing stage.
+  constexpr int RS = D + 8;  // padded row stride (floats) of the parked tile
+  float* s_red = reinterpret_cast<float*>(s_k);
+  float* s_m = s_red + BM * RS;
+  float* s_l = s_m + BM;
+  float* s_w = s_l + BM;          // [rows_per][S] merge weights of this CTA's rows
+  float* s_lse = s_w + BM + 8;    // [rows_per]
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     float l = l_run[i];
     l += __shfl_xor_sync(0xffffffffu, l, 1);
     l += __shfl_xor_sync(0xffffffffu, l, 2);
-    if (!row_ok[i]) continue;
-    const float inv = l > 0.f ? 1.f / l : 0.f;
-    const float lse2 = l > 0.f ? m_run[i] + log2f(l) : -INFINITY;
+    const int r = warp * 16 + (lane >> 2) + 8 * i;
     const int c0 = (lane & 3) * 2;
-    if (p.num_splits == 1) {
-      bf16* orow = p.out + grow[i] * D;
+    if (n_tiles > 0) {
 #pragma unroll
       for (int d = 0; d < DT; ++d)
-        *reinterpret_cast<uint32_t*>(orow + d * 8 + c0) =
-            pack_bf16(o_acc[d][2 * i] * inv, o_acc[d][2 * i + 1] * inv);
-      if (p.lse && (lane & 3) == 0) p.lse[grow[i]] = l > 0.f ? lse2 * kLn2 : 0.f;
-    } else {
-      float* orow = p.part_o + (split * rows_all + grow[i]) * D;
-#pragma unroll
-      for (int d = 0; d < DT; ++d)
-        *reinterpret_cast<float2*>(orow + d * 8 + c0) =
-            make_float2(o_acc[d][2 * i] * inv, o_acc[d][2 * i + 1] * inv);
-      if ((lane & 3) == 0) p.part_lse[split * rows_all + grow[i]] = lse2;
+        *reinterpret_cast<float2*>(s_red + r * RS + d * 8 + c0) = make_float2(o_acc[d][2 * i], o_acc[d][2 * i + 1]);
     }
+    if ((lane & 3) == 0) { s_m[r] = m_run[i]; s_l[r] = l; }
   }
+  if (S > 1) cluster.sync(); else __syncthreads();
+
+  cluster_merge_and_store<D, BM>(p, cluster, S, crank, s_red, s_m, s_l, s_w, s_lse, split / S, row0, rows_total, g, si.q_off,
+                                 rows_all, tid, NTHREADS);
+  if (S > 1) cluster.sync();  // nobody leaves while a peer may still read its shared memory
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -473,13 +379,13 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
   const long long rows_all = (long long)p.total_q * Hq;
   const long long grow = (long long)q_off * Hq + rr;
   float M = -INFINITY;
-  for (int s = 0; s < p.num_splits; ++s) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
+  for (int s = 0; s < p.outer; ++s) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
   float acc[E];
 #pragma unroll
   for (int e = 0; e < E; ++e) acc[e] = 0.f;
   float denom = 0.f;
   if (M != -INFINITY) {
-    for (int s = 0; s < p.num_splits; ++s) {
+    for (int s = 0; s < p.outer; ++s) {
       const float ls = p.part_lse[s * rows_all + grow];
       if (ls == -INFINITY) continue;  // that chunk saw no key for this row: its O is not written
       const float w = exp2f(ls - M);
@@ -531,34 +437,137 @@ static sb_status check_batch(const sb_tree_batch* tb) {
   return SB_OK;
 }
 
-// KV chunks per (sequence, KV head, row tile) when the caller leaves the choice to us: one wave
-// of CTAs when the batch is small, otherwise chunks of about 16 KV tiles to even out ragged
-// prefix lengths.
-static int choose_splits(const sb_tree_batch* tb, int num_splits) {
-  const int G = tb->n_q_heads / tb->n_kv_heads;
-  const int row_tiles = ceil_div(tb->max_nodes * G, BM);
-  const int max_tiles = ceil_div(tb->max_kv_len, BN);
-  if (num_splits > 0) return num_splits < max_tiles ? num_splits : max_tiles;
-  const long long base = (long long)tb->batch * tb->n_kv_heads * row_tiles;
-  const int sms = num_sms();
-  int s;
-  if (base <= sms) {
-    s = (int)(sms / base);
-  } else {
-    s = max_tiles / 16;
-    if (s > 16) s = 16;
+constexpr int kMaxCluster = 8;  // portable thread-block cluster size
+
+struct SplitPlan {
+  int cluster;  // chunk-CTAs merged through distributed shared memory
+  int outer;    // clusters per (sequence, KV head, row tile)
+};
+
+// How many clusters of `cluster` CTAs of the attention kernel can be resident at once (0 when the
+// query fails).  Cached per (head_dim, cluster size); 8-CTA clusters of full-SM CTAs do not tile
+// the 148 SMs evenly, so this is what decides whether a grid runs as one wave.
+static int max_active_clusters(int D, int cluster) {
+  static int cache[2][kMaxCluster + 1];
+  static bool have[2][kMaxCluster + 1];
+  const int di = D == 64 ? 0 : 1;
+  if (!have[di][cluster]) {
+    const size_t smem = 2560 + (size_t)BM * D * 2 + 2 * (size_t)STAGES * BN * D * 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cluster * 64, 1, 1);
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    cudaError_t e;
+    if (D == 64) {
+      cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      e = cudaOccupancyMaxActiveClusters(&n, attn_mma_kernel<64>, &cfg);
+    } else {
+      cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      e = cudaOccupancyMaxActiveClusters(&n, attn_mma_kernel<128>, &cfg);
+    }
+    if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
+    cache[di][cluster] = n;
+    have[di][cluster] = true;
   }
-  if (s > max_tiles) s = max_tiles;
-  if (s < 1) s = 1;
-  return s;
+  return cache[di][cluster];
 }
 
-static size_t workspace_bytes_for(const sb_tree_batch* tb, int total_q, int splits) {
-  if (splits <= 1) return 0;
+static SplitPlan plan_for(int s) {
+  SplitPlan sp;
+  sp.cluster = 1;
+  for (int c = kMaxCluster; c >= 1; --c)
+    if (s % c == 0) { sp.cluster = c; break; }
+  sp.outer = s / sp.cluster;
+  return sp;
+}
+
+enum AttnImpl { IMPL_TC = 0, IMPL_MMA = 1, IMPL_SIMPLE = 2 };
+
+static AttnImpl attn_impl() {
+  const char* impl = getenv("SB_ATTN_IMPL");
+  if (impl && strcmp(impl, "simple") == 0) return IMPL_SIMPLE;
+  if (impl && strcmp(impl, "mma") == 0) return IMPL_MMA;
+  return IMPL_TC;
+}
+
+// KV chunks per (sequence, KV head, row tile).  When the caller leaves the choice to us: the
+// largest count whose clusters are all resident at once when the batch is small, otherwise
+// chunks of a few KV blocks to even out ragged prefix lengths.  The chunks are grouped into
+// clusters of the largest divisor <= 8.  `granule` is the kernel's key-block size.
+static SplitPlan choose_splits(const sb_tree_batch* tb, int num_splits, AttnImpl impl) {
+  const int G = tb->n_q_heads / tb->n_kv_heads;
+  const int row_tiles = ceil_div(tb->max_nodes * G, BM);
+  const int granule = impl == IMPL_TC ? 128 : BN;
+  const int max_blocks = ceil_div(tb->max_kv_len, granule);
+  if (num_splits > 0) return plan_for(num_splits < max_blocks ? num_splits : max_blocks);
+  const long long base = (long long)tb->batch * tb->n_kv_heads * row_tiles;
+  const int sms = num_sms();
+  if (base > sms) {
+    int s = impl == IMPL_TC ? max_blocks / 8 : max_blocks / 16;
+    if (s > 16) s = 16;
+    if (s < 1) s = 1;
+    return plan_for(s);
+  }
+  int s = (int)(sms / base);
+  if (s > max_blocks) s = max_blocks;
+  for (; s > 1; --s) {
+    const SplitPlan sp = plan_for(s);
+    if (sp.outer > 1 && sp.cluster < 4) continue;  // partial traffic for little gain
+    const int fit = impl == IMPL_TC ? attn_tc_max_active_clusters(tb->head_dim, sp.cluster)
+                                    : max_active_clusters(tb->head_dim, sp.cluster);
+    if (fit <= 0 || base * sp.outer <= fit) return sp;
+  }
+  return plan_for(1);
+}
+
+static size_t workspace_bytes_for(const sb_tree_batch* tb, int total_q, int outer) {
+  if (outer <= 1) return 0;
   const size_t rows = (size_t)total_q * tb->n_q_heads;
-  const size_t o = (size_t)splits * rows * tb->head_dim * sizeof(float);
-  const size_t l = (size_t)splits * rows * sizeof(float);
+  const size_t o = (size_t)outer * rows * tb->head_dim * sizeof(float);
+  const size_t l = (size_t)outer * rows * sizeof(float);
   return ((o + 255) & ~(size_t)255) + ((l + 255) & ~(size_t)255);
+}
+
+template <int D>
+static sb_status launch_attn_mma(const AttnParams& p, dim3 grid, int cluster, cudaStream_t cs) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_mma_smem_bytes<D>()) != cudaSuccess)
+      return SB_ERR_CUDA;
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(NTHREADS);
+  cfg.dynamicSmemBytes = attn_mma_smem_bytes<D>();
+  cfg.stream = cs;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (getenv("SB_DEBUG")) {
+    int max_clusters = -1;
+    cudaOccupancyMaxActiveClusters(&max_clusters, attn_mma_kernel<D>, &cfg);
+    fprintf(stderr, "[sb] attn_mma<%d> grid (%u,%u,%u) cluster %d outer %d: max active clusters %d\n", D, grid.x,
+            grid.y, grid.z, cluster, p.outer, max_clusters);
+  }
+  if (cudaLaunchKernelEx(&cfg, attn_mma_kernel<D>, p) != cudaSuccess) {
+    cudaGetLastError();
+    return SB_ERR_CUDA;
+  }
+  return launch_check();
 }
 
 }  // namespace sb
@@ -566,7 +575,7 @@ static size_t workspace_bytes_for(const sb_tree_batch* tb, int total_q, int spli
 extern "C" size_t sb_tree_attention_workspace_bytes(const sb_tree_batch* tb, int32_t total_q,
                                                     int32_t num_splits) {
   if (sb::check_batch(tb) != SB_OK || total_q < 0 || num_splits < 0) return 0;
-  return sb::workspace_bytes_for(tb, total_q, sb::choose_splits(tb, num_splits));
+  return sb::workspace_bytes_for(tb, total_q, sb::choose_splits(tb, num_splits, sb::attn_impl()).outer);
 }
 
 extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q_node_begin,
@@ -597,50 +606,34 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   p.part_o = nullptr;
   p.part_lse = nullptr;
 
-  const char* impl = getenv("SB_ATTN_IMPL");
-  if (impl && strcmp(impl, "simple") == 0) {
+  const AttnImpl impl = attn_impl();
+  if (impl == IMPL_SIMPLE) {
     p.num_splits = 1;
+    p.outer = 1;
     dim3 grid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);
     if (D == 64) attn_simple_kernel<64><<<grid, 256, 0, cs>>>(p);
     else attn_simple_kernel<128><<<grid, 256, 0, cs>>>(p);
     return launch_check();
   }
 
-  const int splits = choose_splits(tb, num_splits);
-  p.num_splits = splits;
-  if (splits > 1) {
-    const size_t need = workspace_bytes_for(tb, total_q, splits);
+  const SplitPlan plan = choose_splits(tb, num_splits, impl);
+  p.num_splits = plan.cluster * plan.outer;
+  p.outer = plan.outer;
+  if (plan.outer > 1) {
+    const size_t need = workspace_bytes_for(tb, total_q, plan.outer);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255))
       return SB_ERR_WORKSPACE;
     const size_t rows = (size_t)total_q * tb->n_q_heads;
-    const size_t o = ((size_t)splits * rows * D * sizeof(float) + 255) & ~(size_t)255;
+    const size_t o = ((size_t)plan.outer * rows * D * sizeof(float) + 255) & ~(size_t)255;
     p.part_o = static_cast<float*>(workspace);
     p.part_lse = reinterpret_cast<float*>(static_cast<char*>(workspace) + o);
   }
   const int row_tiles = ceil_div(tb->max_nodes * p.G, BM);
-  dim3 grid(splits, row_tiles * tb->n_kv_heads, tb->batch);
+  dim3 grid(p.num_splits, row_tiles * tb->n_kv_heads, tb->batch);
   if (grid.y > 65535 || grid.z > 65535) return SB_ERR_UNSUPPORTED;
-  if (D == 64) {
-    static bool attr64 = false;
-    if (!attr64) {
-      if (cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)attn_mma_smem_bytes<64>()) != cudaSuccess)
-        return SB_ERR_CUDA;
-      attr64 = true;
-    }
-    attn_mma_kernel<64><<<grid, NTHREADS, attn_mma_smem_bytes<64>(), cs>>>(p);
-  } else {
-    static bool attr128 = false;
-    if (!attr128) {
-      if (cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)attn_mma_smem_bytes<128>()) != cudaSuccess)
-        return SB_ERR_CUDA;
-      attr128 = true;
-    }
-    attn_mma_kernel<128><<<grid, NTHREADS, attn_mma_smem_bytes<128>(), cs>>>(p);
-  }
-  st = launch_check();
-  if (st != SB_OK || splits == 1) return st;
+  if (impl == IMPL_TC) st = launch_attn_tc(p, grid, plan.cluster, cs);
+  else st = D == 64 ? launch_attn_mma<64>(p, grid, plan.cluster, cs) : launch_attn_mma<128>(p, grid, plan.cluster, cs);
+  if (st != SB_OK || plan.outer == 1) return st;
   dim3 mgrid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);
   if (D == 64) attn_merge_kernel<64><<<mgrid, 256, 0, cs>>>(p);
   else attn_merge_kernel<128><<<mgrid, 256, 0, cs>>>(p);

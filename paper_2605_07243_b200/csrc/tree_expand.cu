@@ -1,14 +1,18 @@
 // sb_tree_expand: per-row top-k over the drafter's scores and bucket-driven branching
 // (Sec. 3.2; App. A.5 maps b(.); Alg. 1 "attach the top-b(bkt) tokens").
 //
-//   topk_partial_kernel : streams the [rows][vocab] fp32 scores once.  A CTA owns one (row, vocab
-//                         chunk); each thread keeps its 16 best in registers (ids ascend inside a
-//                         thread, so insertion only needs a strict compare against the current
-//                         worst), the CTA then pops the 16 best of all threads in order.
-//   expand_finish_kernel: one CTA: a warp per row merges the chunk lists (value descending, id
-//                         ascending); then one thread walks the rows in order and appends the
-//                         new nodes -- the append order is sequential by definition and touches at
-//                         most `node_budget` (<= a few hundred) entries.
+//   topk_partial_kernel : streams the [rows][vocab] fp32 scores once from HBM (a second pass hits
+//                         L1/L2).  A CTA owns one (row, vocab chunk).  Pass 1: every thread takes the
+//                         maximum of its strided elements; the 16th largest of the 256 thread maxima is
+//                         a threshold tau that at least 16 elements of the chunk reach.  Pass 2: only
+//                         elements >= tau (a handful per CTA unless values tie) enter the per-thread
+//                         sorted lists; ids ascend inside a thread, so the order (value descending, id
+//                         ascending) is kept by strict compares.  The CTA then pops its 16 best in order.
+//   expand_finish_kernel: one CTA.  A warp per row merges the chunk lists held in registers; then the
+//                         append is done in parallel: a row is alive iff every earlier position of its
+//                         block has width >= 1, its first node id is an exclusive prefix sum of the
+//                         alive rows' widths, and the node budget clips the tail (a clipped rank-0 node
+//                         can only silence rows that the full budget silences anyway).
 #include "common.cuh"
 
 namespace sb {
@@ -33,6 +37,33 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
   const int begin = c * chunk;
   const int end = min(vocab, begin + chunk);
 
+  // pass 1: thread maxima -> threshold tau = 16th largest of them
+  const int n_vec = vec_ok ? max(0, (end - begin) / 4) : 0;
+  const float4* vb = reinterpret_cast<const float4*>(base + begin);
+  float tmax = -INFINITY;
+  for (int t = tid; t < n_vec; t += TOPK_THREADS) {
+    const float4 x = __ldg(vb + t);
+    tmax = fmaxf(tmax, fmaxf(fmaxf(score_of(x.x), score_of(x.y)), fmaxf(score_of(x.z), score_of(x.w))));
+  }
+  for (int i = begin + n_vec * 4 + tid; i < end; i += TOPK_THREADS) tmax = fmaxf(tmax, score_of(base[i]));
+  float* s_max = &s_val[0][0];  // the lists are written only after pass 2
+  __shared__ float s_tau;
+  s_max[tid] = tmax;
+  if (tid == 0) s_tau = -INFINITY;
+  __syncthreads();
+  {
+    int gt = 0, ge = 0;
+    for (int t = 0; t < TOPK_THREADS; ++t) {
+      const float o = s_max[t];
+      gt += o > tmax;
+      ge += o >= tmax;
+    }
+    if (gt < SB_KMAX && ge >= SB_KMAX) s_tau = tmax;  // every writer holds the same value
+  }
+  __syncthreads();
+  const float tau = s_tau;
+  __syncthreads();  // s_max (aliasing the lists) is dead from here on
+
   float v[SB_KMAX];
   int id[SB_KMAX];
 #pragma unroll
@@ -40,6 +71,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
 
   auto offer = [&](float x, int xi) {
     x = score_of(x);
+    if (x < tau) return;  // at least 16 elements of the chunk reach tau
     if (!ranks_before(x, xi, v[SB_KMAX - 1], id[SB_KMAX - 1])) return;
     v[SB_KMAX - 1] = x;
     id[SB_KMAX - 1] = xi;
@@ -53,8 +85,6 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
   };
 
   if (vec_ok) {
-    const int n_vec = max(0, (end - begin) / 4);
-    const float4* vb = reinterpret_cast<const float4*>(base + begin);
     for (int t = tid; t < n_vec; t += TOPK_THREADS) {
       const float4 x = __ldg(vb + t);
       const int i0 = begin + 4 * t;
@@ -110,18 +140,37 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
     int* __restrict__ node_row, int* __restrict__ node_rank, int* __restrict__ topk_tok,
     float* __restrict__ topk_val, int* __restrict__ status) {
   __shared__ int s_bad;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) s_bad = 0;
+  __shared__ int s_warp_sum[FINISH_THREADS / 32];
+  __shared__ int s_first[FINISH_THREADS + 1];  // first node id of each row of the current slab
+  __shared__ int s_carry;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) s_bad = 0;
   __syncthreads();
-  // (1) merge the chunk lists of every row: lane c walks chunk c's sorted list
+  // (1) merge the chunk lists of every row: lane c holds chunk c's sorted list in registers and
+  //     pops it by shifting
   for (int r = warp; r < n_rows; r += FINISH_THREADS / 32) {
-    int pos = 0;
-    const long long lb = ((long long)r * n_chunks + lane) * SB_KMAX;
+    float lv[SB_KMAX];
+    int li[SB_KMAX];
+    if (lane < n_chunks) {
+      const float4* pv = reinterpret_cast<const float4*>(part_val + ((long long)r * n_chunks + lane) * SB_KMAX);
+      const int4* pi = reinterpret_cast<const int4*>(part_idx + ((long long)r * n_chunks + lane) * SB_KMAX);
+#pragma unroll
+      for (int q = 0; q < SB_KMAX / 4; ++q) {
+        const float4 a = pv[q];
+        const int4 c = pi[q];
+        lv[4 * q] = a.x; lv[4 * q + 1] = a.y; lv[4 * q + 2] = a.z; lv[4 * q + 3] = a.w;
+        li[4 * q] = c.x; li[4 * q + 1] = c.y; li[4 * q + 2] = c.z; li[4 * q + 3] = c.w;
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < SB_KMAX; ++k) { lv[k] = -INFINITY; li[k] = kNoId; }
+    }
+    float keep_v = -INFINITY;
+    int keep_i = -1;
+#pragma unroll
     for (int round = 0; round < SB_KMAX; ++round) {
-      const bool have = lane < n_chunks && pos < SB_KMAX;
-      float hv = have ? part_val[lb + pos] : -INFINITY;
-      int hi = have ? part_idx[lb + pos] : kNoId;
-      int hl = lane;
+      float hv = lv[0];
+      int hi = li[0], hl = lane;
 #pragma unroll
       for (int s = 16; s > 0; s >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, hv, s);
@@ -129,49 +178,94 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
         const int ol = __shfl_xor_sync(0xffffffffu, hl, s);
         if (ranks_before(ov, oi, hv, hi)) { hv = ov; hi = oi; hl = ol; }
       }
-      if (lane == 0) {
-        topk_tok[r * SB_KMAX + round] = hi == kNoId ? -1 : hi;
-        topk_val[r * SB_KMAX + round] = hv;
+      if (lane == round) { keep_v = hv; keep_i = hi == kNoId ? -1 : hi; }
+      if (hi != kNoId && lane == hl) {
+#pragma unroll
+        for (int k = 0; k + 1 < SB_KMAX; ++k) { lv[k] = lv[k + 1]; li[k] = li[k + 1]; }
+        lv[SB_KMAX - 1] = -INFINITY;
+        li[SB_KMAX - 1] = kNoId;
       }
-      if (hi != kNoId && lane == hl) ++pos;
+    }
+    if (lane < SB_KMAX) {
+      topk_tok[r * SB_KMAX + lane] = keep_i;
+      topk_val[r * SB_KMAX + lane] = keep_v;
     }
   }
   // (2) argument checks that need device data
   const int n0 = *n_nodes;
-  if (threadIdx.x == 0 && (n0 < 0 || n0 > node_budget)) s_bad = 1;
-  for (int r = threadIdx.x; r < n_rows; r += FINISH_THREADS)
+  if (tid == 0 && (n0 < 0 || n0 > node_budget)) s_bad = 1;
+  for (int r = tid; r < n_rows; r += FINISH_THREADS)
     if (bucket[r] > 3) s_bad = 1;
-  for (int i = threadIdx.x; i < n_rows / block_k; i += FINISH_THREADS)
+  for (int i = tid; i < n_rows / block_k; i += FINISH_THREADS)
     if (start_parent[i] < -1 || start_parent[i] >= n0) s_bad = 1;
-  __syncthreads();
+  if (tid == 0) s_carry = n0;
+  __syncthreads();  // also publishes the merged lists to the whole CTA
   if (s_bad) {
-    if (threadIdx.x == 0) *status = SB_ERR_INVALID_ARG;
+    if (tid == 0) *status = SB_ERR_INVALID_ARG;
     return;
   }
-  // (3) append in row order
-  if (threadIdx.x == 0) {
-    const int widths[4] = {bmap.x, bmap.y, bmap.z, bmap.w};
-    int n = n0, chain = -1;
-    bool chain_alive = false;
-    for (int r = 0; r < n_rows; ++r) {
-      const int kpos = r % block_k;
-      int b = widths[bucket[r]];
-      if (b > vocab) b = vocab;
-      const int attach = kpos == 0 ? start_parent[r / block_k] : chain;
-      const bool alive = kpos == 0 ? true : chain_alive;
-      chain_alive = false;
-      if (!alive) continue;
-      for (int j = 0; j < b && n < node_budget; ++j) {
+  // (3) append, a slab of FINISH_THREADS rows at a time (slabs are cut at block boundaries)
+  const int rows_per_slab = (FINISH_THREADS / block_k) * block_k > 0 ? (FINISH_THREADS / block_k) * block_k : 0;
+  if (rows_per_slab == 0) {  // a block longer than a slab is not supported
+    if (tid == 0) *status = SB_ERR_UNSUPPORTED;
+    return;
+  }
+  for (int slab = 0; slab < n_rows; slab += rows_per_slab) {
+    const int r = slab + tid;
+    int width = 0, kpos = 0, start = -1;
+    if (tid < rows_per_slab && r < n_rows) {
+      kpos = r % block_k;
+      start = start_parent[r / block_k];
+      auto width_of = [&](int row) {
+        const int bk = bucket[row];
+        const int w = bk == 0 ? bmap.x : bk == 1 ? bmap.y : bk == 2 ? bmap.z : bmap.w;
+        return w < vocab ? w : vocab;
+      };
+      bool alive = true;
+      for (int k = 1; k <= kpos; ++k) alive = alive && width_of(r - k) >= 1;
+      width = alive ? width_of(r) : 0;
+    }
+    // exclusive scan of the widths over the slab
+    int incl = width;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, s);
+      if (lane >= s) incl += o;
+    }
+    if (lane == 31) s_warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = s_warp_sum[lane];
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, w, s);
+        if (lane >= s) w += o;
+      }
+      s_warp_sum[lane] = w;  // inclusive over warps
+    }
+    __syncthreads();
+    const int carry = s_carry;
+    const int first = carry + (warp > 0 ? s_warp_sum[warp - 1] : 0) + incl - width;
+    s_first[tid] = first;
+    __syncthreads();
+    if (width > 0) {
+      const int par = kpos == 0 ? start : s_first[tid - 1];  // rank-0 node of the previous position
+      const int base_depth = start == -1 ? 0 : depth[start] + 1;
+      for (int j = 0; j < width && first + j < node_budget; ++j) {
+        const int n = first + j;
         tok[n] = topk_tok[r * SB_KMAX + j];
-        parent[n] = attach;
-        depth[n] = attach == -1 ? 0 : depth[attach] + 1;
+        parent[n] = par;
+        depth[n] = base_depth + kpos;
         node_row[n] = r;
         node_rank[n] = j;
-        if (j == 0) { chain = n; chain_alive = true; }
-        ++n;
       }
     }
-    *n_nodes = n;
+    __syncthreads();
+    if (tid == 0) s_carry = carry + s_warp_sum[FINISH_THREADS / 32 - 1];
+    __syncthreads();
+  }
+  if (tid == 0) {
+    *n_nodes = s_carry < node_budget ? s_carry : node_budget;
     *status = SB_OK;
   }
 }
@@ -206,7 +300,7 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
     return SB_ERR_INVALID_ARG;
   for (int m = 0; m < 4; ++m)
     if (bmap[m] < 0 || bmap[m] > SB_KMAX) return SB_ERR_INVALID_ARG;
-  if (n_rows > 65535) return SB_ERR_UNSUPPORTED;
+  if (n_rows > 65535 || block_k > FINISH_THREADS) return SB_ERR_UNSUPPORTED;
   const size_t need = sb_tree_expand_workspace_bytes(n_rows, vocab);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255))
     return SB_ERR_WORKSPACE;

@@ -52,9 +52,26 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) row_argmax_kernel(const T* __r
   Best best = {-INFINITY, 0x7fffffff};
   if (vec_ok) {
     // chunk is a multiple of VEC and rows are 16-byte aligned
-    const int n_vec = (end - begin) / VEC;
+    const int n_vec = max(0, (end - begin) / VEC);
     const uint4* vb = reinterpret_cast<const uint4*>(base + begin);
-    for (int t = threadIdx.x; t < n_vec; t += ARGMAX_THREADS) {
+    constexpr int UNROLL = 4;  // independent 16-byte loads in flight per thread
+    int t = threadIdx.x;
+    for (; t + (UNROLL - 1) * ARGMAX_THREADS < n_vec; t += UNROLL * ARGMAX_THREADS) {
+      uint4 raw[UNROLL];
+#pragma unroll
+      for (int q = 0; q < UNROLL; ++q) raw[q] = __ldg(vb + t + q * ARGMAX_THREADS);
+#pragma unroll
+      for (int q = 0; q < UNROLL; ++q) {
+        const T* e = reinterpret_cast<const T*>(&raw[q]);
+#pragma unroll
+        for (int u = 0; u < VEC; ++u) {
+          const float x = logit_to_float<T>(e[u]);
+          const int id = begin + (t + q * ARGMAX_THREADS) * VEC + u;
+          if (x > best.v) { best.v = x; best.i = id; }  // ids ascend inside a thread: strict keeps the first
+        }
+      }
+    }
+    for (; t < n_vec; t += ARGMAX_THREADS) {
       const uint4 raw = __ldg(vb + t);
       const T* e = reinterpret_cast<const T*>(&raw);
 #pragma unroll

@@ -181,6 +181,20 @@ def test_chunk_without_visible_key():
     check_attention(case, "P=0, 2 chunks", num_splits=2)
 
 
+@pytest.mark.parametrize("impl", ["mma", "tc"])
+def test_both_tensor_core_paths(monkeypatch, impl):
+    """The tcgen05 kernel is the default; the mma.sync kernel stays selectable and correct."""
+    monkeypatch.setenv("SB_ATTN_IMPL", impl)
+    attn, _ = W.config1_tiny()
+    check_attention(attn, f"{impl}: config 1", num_splits=2)
+    check_attention(W.config2_verify_layer(prefix=777), f"{impl}: 8B-shaped, P=777")
+    check_attention(W.config2_verify_layer(prefix=777), f"{impl}: 8B-shaped, P=777, 16 chunks", num_splits=16)
+    rng = W.rng_for(50)
+    case = W.make_attn_case(rng, parents=[W.random_tree(rng, 128, 12), W.chain_tree(5), W.random_tree(rng, 40, 6)],
+                            prefix_lens=[333, 0, 2000], n_q_heads=64, n_kv_heads=8, head_dim=128, page_size=64)
+    check_attention(case, f"{impl}: ragged paged G=8", num_splits=5)
+
+
 def test_simple_kernel_path(monkeypatch):
     monkeypatch.setenv("SB_ATTN_IMPL", "simple")
     attn, _ = W.config1_tiny()
@@ -221,11 +235,15 @@ def test_bad_page_id_is_reported_without_fault():
 
 
 def test_host_argument_errors():
+    big = W.config2_verify_layer(prefix=1500)
+    tb, q, kw = dev.attention_args(big)
+    assert sb.sb_tree_attention_workspace_bytes(tb, q.shape[0], 8) == 0      # one cluster: no scratch
+    assert sb.sb_tree_attention_workspace_bytes(tb, q.shape[0], 16) > 0      # two clusters: partials
+    with pytest.raises(sb.SbError) as e:
+        sb.sb_tree_attention(tb, q, num_splits=16, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == 3
     attn, _ = W.config1_tiny()
     tb, q, kw = dev.attention_args(attn)
-    with pytest.raises(sb.SbError) as e:
-        sb.sb_tree_attention(tb, q, num_splits=2, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
-    assert e.value.code == 3
     tb.head_dim = 48
     with pytest.raises(sb.SbError) as e:
         sb.sb_tree_attention(tb, q)
