@@ -37,13 +37,17 @@ struct SeqPlan {
   bool compute;    // tree and lengths are valid: run the attention
 };
 
-// Must be called by every thread of the CTA (contains barriers).  `designated` CTAs (one per
-// sequence) also scan the page table and publish the sequence's status word.
-__device__ inline SeqPlan plan_sequence(const AttnParams& p, int b, bool designated, int* s_parent,
-                                        uint32_t* s_anc) {
-  SeqPlan sp;
-  sp.info = load_seq_info(p.tb, p.q_node_begin, p.q_offsets, p.total_q, b);
-  int err = sp.info.err;
+// First half of the planning: lengths and row ranges from the per-sequence scalars (no barrier,
+// every thread computes the same values).
+struct SeqPre {
+  SeqInfo info;
+  bool can_write;
+  int node_base;  // offset of the sequence's parent[] slice (0 when it cannot be trusted)
+};
+
+__device__ inline SeqPre plan_lengths(const AttnParams& p, int b) {
+  SeqPre pre;
+  pre.info = load_seq_info(p.tb, p.q_node_begin, p.q_offsets, p.total_q, b);
   // Which rows may be zero-filled on error: recompute the raw row range.
   const int o = p.tb.node_offsets[b];
   const int n_raw = p.tb.node_offsets[b + 1] - o;
@@ -52,14 +56,26 @@ __device__ inline SeqPlan plan_sequence(const AttnParams& p, int b, bool designa
   const bool rows_ok = n_raw >= 0 && n_raw <= SB_MAX_NODES && n_raw <= p.tb.max_nodes && q0 >= 0 &&
                        q0 <= n_raw && q_off >= 0 && (long long)q_off + (n_raw - q0) <= p.total_q &&
                        o >= 0 && (long long)o + n_raw <= p.tb.total_nodes;
-  sp.can_write = rows_ok;
-  if (rows_ok && err) {  // lengths are bad but the rows exist: keep them for zero-filling
-    sp.info.nq = n_raw - q0;
-    sp.info.q0 = q0;
-    sp.info.q_off = q_off;
+  pre.can_write = rows_ok;
+  pre.node_base = rows_ok ? o : 0;
+  if (rows_ok && pre.info.err) {  // lengths are bad but the rows exist: keep them for zero-filling
+    pre.info.nq = n_raw - q0;
+    pre.info.q0 = q0;
+    pre.info.q_off = q_off;
   }
-  const bool tree_ok = build_ancestors_smem(p.tb.parent + (rows_ok ? o : 0), err ? 0 : sp.info.n,
-                                            s_parent, s_anc, nullptr);
+  return pre;
+}
+
+// Second half: ancestor sets into shared memory, tree validity, status word.  Must be called by
+// every thread of the CTA (contains barriers).  `designated` CTAs (one per sequence) also scan
+// the page table and publish the sequence's status word.
+__device__ inline SeqPlan plan_tree(const AttnParams& p, int b, bool designated, const SeqPre& pre, int* s_parent,
+                                    uint32_t* s_anc) {
+  SeqPlan sp;
+  sp.info = pre.info;
+  sp.can_write = pre.can_write;
+  int err = sp.info.err;
+  const bool tree_ok = build_ancestors_smem(p.tb.parent + pre.node_base, err ? 0 : sp.info.n, s_parent, s_anc, nullptr);
   if (!err && !tree_ok) err = SB_ERR_INVALID_TREE;
   if (designated) {
     const bool pages_ok = err ? true : pages_in_pool(p.tb, b, sp.info.P + sp.info.n);
@@ -69,6 +85,12 @@ __device__ inline SeqPlan plan_sequence(const AttnParams& p, int b, bool designa
   }
   sp.compute = err == 0;
   return sp;
+}
+
+__device__ inline SeqPlan plan_sequence(const AttnParams& p, int b, bool designated, int* s_parent,
+                                        uint32_t* s_anc) {
+  const SeqPre pre = plan_lengths(p, b);
+  return plan_tree(p, b, designated, pre, s_parent, s_anc);
 }
 
 __device__ inline float fast_exp2(float x) {
@@ -97,55 +119,105 @@ __device__ inline uint64_t visibility_window(const uint32_t (&a)[4], int rel0) {
 }
 
 
-// Merge of the cluster's KV chunks and final store (called by every thread of every CTA of the
-// cluster after a cluster-wide barrier).  Each CTA has parked, in its own shared memory, its
-// unnormalised O tile `s_red` [BM_][D+PAD], row maxima `s_m` and row sums `s_l` (base-2 domain).
-// CTA `crank` reduces rows [crank*rows_per, (crank+1)*rows_per) over all S CTAs through
-// distributed shared memory and writes them: final bf16 rows + natural-log LSE when the grid has
-// one cluster per row tile, else one fp32 partial per cluster for the merge kernel.
-template <int D, int BM_, int PAD = 8>
-__device__ inline void cluster_merge_and_store(const AttnParams& p, cg::cluster_group& cluster, int S, int crank,
-                                               float* s_red, float* s_m, float* s_l, float* s_w, float* s_lse,
-                                               int outer_idx, int row0, int rows_total, int g, int q_off,
-                                               long long rows_all, int tid, int nthreads) {
-  constexpr int RS = D + PAD;
+// ---- in-cluster merge of KV chunks (push model) ---------------------------------------------------
+// The S chunk-CTAs of a cluster each hold an unnormalised O tile [BM][D] with row maxima m and row
+// sums l (base-2 domain).  Row r of the tile is owned by CTA r / rows_per (rows_per = ceil(BM/S)).
+// Every CTA stores each of its rows straight into the OWNER's shared memory (distributed shared
+// memory stores need no round trip), slot [source rank][row - owner's first row]; after one
+// cluster barrier each owner reduces its rows from local shared memory and writes them out.
+// Buffer layout in every CTA, starting at `buf`:
+//   red [S*rows_per][D+8] | m [S*rows_per] | l [S*rows_per] | w [rows_per*S] | lse [rows_per]
+template <int D>
+struct MergeBuf {
+  static constexpr int RS = D + 8;
+  float* red;
+  float* m;
+  float* l;
+  float* w;
+  float* lse;
+  int rows_per;
+  __device__ MergeBuf(float* buf, int BM, int S) {
+    rows_per = ceil_div(BM, S);
+    const int slots = S * rows_per;
+    red = buf;
+    m = red + slots * RS;
+    l = m + slots;
+    w = l + slots;
+    lse = w + slots;
+  }
+  // floats needed for a tile of BM rows and any cluster size up to 8
+  static constexpr int floats(int BM) { return (BM + 8) * RS + 4 * (BM + 8); }
+};
+
+// Destination (in the owner's shared memory) of row r of the CTA with cluster rank `crank`.
+template <int D>
+__device__ inline float* merge_row_dst(cg::cluster_group& cluster, const MergeBuf<D>& mb, int crank, int r, int* slot) {
+  const int owner = r / mb.rows_per;
+  *slot = crank * mb.rows_per + (r - owner * mb.rows_per);
+  return cluster.map_shared_rank(mb.red, owner) + *slot * MergeBuf<D>::RS;
+}
+template <int D>
+__device__ inline void merge_push_ml(cg::cluster_group& cluster, const MergeBuf<D>& mb, int crank, int r, float m, float l) {
+  const int owner = r / mb.rows_per;
+  const int slot = crank * mb.rows_per + (r - owner * mb.rows_per);
+  cluster.map_shared_rank(mb.m, owner)[slot] = m;
+  cluster.map_shared_rank(mb.l, owner)[slot] = l;
+}
+
+// After the cluster barrier: reduce this CTA's rows over the S sources and store them -- final bf16
+// rows + natural-log LSE when the grid has one cluster per row tile, else one fp32 partial per
+// cluster for the merge kernel.
+template <int D, int BM>
+__device__ inline void merge_reduce_and_store(const AttnParams& p, const MergeBuf<D>& mb, int S, int crank, int outer_idx,
+                                              int row0, int rows_total, int g, int q_off, long long rows_all, int tid,
+                                              int nthreads) {
+  constexpr int RS = MergeBuf<D>::RS;
+  constexpr int MAXS = 8;
   const int Hq = p.tb.n_q_heads, G = p.G;
-  constexpr int BM = BM_;
-  const int NTHREADS = nthreads;
-  const int rows_per = ceil_div(BM, S);
+  const int rows_per = mb.rows_per;
   const int r_begin = crank * rows_per;
-  const int r_end = min(BM, r_begin + rows_per);
-  for (int t = tid; t < r_end - r_begin; t += NTHREADS) {
-    const int r = r_begin + t;
+  const int n_rows = max(0, min(BM, r_begin + rows_per) - r_begin);
+  for (int t = tid; t < n_rows; t += nthreads) {
+    float mc[MAXS], lc[MAXS];
+#pragma unroll
+    for (int c = 0; c < MAXS; ++c) {
+      mc[c] = c < S ? mb.m[c * rows_per + t] : -INFINITY;
+      lc[c] = c < S ? mb.l[c * rows_per + t] : 0.f;
+    }
     float M = -INFINITY;
-    for (int c = 0; c < S; ++c) M = fmaxf(M, cluster.map_shared_rank(s_m, c)[r]);
+#pragma unroll
+    for (int c = 0; c < MAXS; ++c) M = fmaxf(M, mc[c]);
     float Lsum = 0.f;
-    for (int c = 0; c < S; ++c) {
-      const float mc = cluster.map_shared_rank(s_m, c)[r];
-      const float wc = mc == -INFINITY ? 0.f : fast_exp2(mc - M);
-      s_w[t * S + c] = wc;
-      Lsum += wc * cluster.map_shared_rank(s_l, c)[r];
+    float wc[MAXS];
+#pragma unroll
+    for (int c = 0; c < MAXS; ++c) {
+      wc[c] = mc[c] == -INFINITY ? 0.f : fast_exp2(mc[c] - M);
+      Lsum += wc[c] * lc[c];
     }
     const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
-    for (int c = 0; c < S; ++c) s_w[t * S + c] *= inv;
-    s_lse[t] = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
+#pragma unroll
+    for (int c = 0; c < MAXS; ++c)
+      if (c < S) mb.w[t * S + c] = wc[c] * inv;
+    mb.lse[t] = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
   }
   __syncthreads();
-  for (int idx = tid; idx < (r_end - r_begin) * (D / 4); idx += NTHREADS) {
+  for (int idx = tid; idx < n_rows * (D / 4); idx += nthreads) {
     const int t = idx / (D / 4), c4 = idx % (D / 4);
-    const int r = r_begin + t;
-    const int R = row0 + r;
+    const int R = row0 + r_begin + t;
     if (R >= rows_total) continue;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = 0; c < S; ++c) {
-      const float w = s_w[t * S + c];
-      if (w == 0.f) continue;  // that chunk saw no key for this row (its tile may be unwritten)
-      const float4 v = *reinterpret_cast<const float4*>(cluster.map_shared_rank(s_red, c) + r * RS + c4 * 4);
-      acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+#pragma unroll
+    for (int c = 0; c < MAXS; ++c) {
+      const float w = c < S ? mb.w[t * S + c] : 0.f;
+      // a chunk that saw no key for this row has weight 0 and left its slot unwritten
+      if (w != 0.f) {
+        const float4 v = *reinterpret_cast<const float4*>(mb.red + (c * rows_per + t) * RS + c4 * 4);
+        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+      }
     }
     const int node_l = R / G, hh = R - node_l * G;
     const long long grow = (long long)(q_off + node_l) * Hq + g * G + hh;
-    const float lse2 = s_lse[t];
+    const float lse2 = mb.lse[t];
     if (p.outer == 1) {
       uint2 packed;
       packed.x = pack_bf16(acc.x, acc.y);

@@ -322,17 +322,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
   }
   cp_async_wait<0>();
   __syncthreads();  // every warp is done with the K/V stages: reuse them as the merge buffer
+  if (S > 1) cluster.sync();  // ... in every CTA of the cluster: peers are about to write into them
 
-  // ---- epilogue: merge the cluster's chunks through (distributed) shared memory -------------
-  // Each CTA parks its unnormalised O tile, row maxima and row sums in its own shared memory;
-  // CTA `crank` of the cluster then reduces rows [crank*rows_per, (crank+1)*rows_per) over all S
-  // CTAs and writes them out.  With S = 1 this is just a coalescing stage.
-  constexpr int RS = D + 8;  // padded row stride (floats) of the parked tile
-  float* s_red = reinterpret_cast<float*>(s_k);
-  float* s_m = s_red + BM * RS;
-  float* s_l = s_m + BM;
-  float* s_w = s_l + BM;          // [rows_per][S] merge weights of this CTA's rows
-  float* s_lse = s_w + BM + 8;    // [rows_per]
+  // ---- epilogue: every row goes to the shared memory of the cluster CTA that owns it; one cluster
+  // barrier; each CTA reduces and stores its rows (with S = 1 this is just a coalescing stage).
+  MergeBuf<D> mb(reinterpret_cast<float*>(s_k), BM, S);
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     float l = l_run[i];
@@ -340,18 +334,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
     l += __shfl_xor_sync(0xffffffffu, l, 2);
     const int r = warp * 16 + (lane >> 2) + 8 * i;
     const int c0 = (lane & 3) * 2;
+    int slot;
+    float* dst = merge_row_dst<D>(cluster, mb, crank, r, &slot);
     if (n_tiles > 0) {
 #pragma unroll
       for (int d = 0; d < DT; ++d)
-        *reinterpret_cast<float2*>(s_red + r * RS + d * 8 + c0) = make_float2(o_acc[d][2 * i], o_acc[d][2 * i + 1]);
+        *reinterpret_cast<float2*>(dst + d * 8 + c0) = make_float2(o_acc[d][2 * i], o_acc[d][2 * i + 1]);
     }
-    if ((lane & 3) == 0) { s_m[r] = m_run[i]; s_l[r] = l; }
+    if ((lane & 3) == 0) merge_push_ml<D>(cluster, mb, crank, r, n_tiles > 0 ? m_run[i] : -INFINITY, n_tiles > 0 ? l : 0.f);
   }
   if (S > 1) cluster.sync(); else __syncthreads();
-
-  cluster_merge_and_store<D, BM>(p, cluster, S, crank, s_red, s_m, s_l, s_w, s_lse, split / S, row0, rows_total, g, si.q_off,
-                                 rows_all, tid, NTHREADS);
-  if (S > 1) cluster.sync();  // nobody leaves while a peer may still read its shared memory
+  merge_reduce_and_store<D, BM>(p, mb, S, crank, split / S, row0, rows_total, g, si.q_off, rows_all, tid, NTHREADS);
 }
 
 // ----------------------------------------------------------------------------------------------

@@ -4,19 +4,28 @@
 // is the M = 128 dimension of the MMA and one row per TMEM lane) and a chunk of the sequence's
 // keys, walked in blocks of up to 128 keys:
 //
-//   loader warps   (2 for K and the Q tile, 1 for V) K and V blocks -> shared memory in the 128-byte-swizzled layouts the
-//                  tensor core reads (K, Q, P: K-major; V: MN-major), 16-byte cp.async, 2 stages each;
+//   loader warps   one thread per operand issues TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle,
+//                  no multicast) of the K and V blocks straight into the shared-memory layouts the
+//                  tensor core reads (K, Q, P: K-major; V: MN-major), 2 stages each, completion by
+//                  mbarrier transaction count; paged caches load one box per page piece.  V rows past
+//                  the end of the sequence are zeroed (P is 0 there, but 0 * garbage must stay 0).
+//                  The Q tile is one TMA box {64 columns, G heads, 128/G nodes} per column half when
+//                  G divides 128, else a 16-byte cp.async gather by the softmax warps;
 //   MMA warp       one thread issues  S_j = Q K_j^T  (tcgen05.mma, fp32 accumulator in TMEM, two S
 //                  buffers so S_{j+1} runs under the softmax of block j) and  PV_j = P_j V_j;
-//   softmax warps  4 warps, thread t owns row t: reads its S row from TMEM (tcgen05.ld), applies the
-//                  softmax scale and the tree mask (one 128-bit ancestor set per row, turned into
-//                  two 64-bit visibility windows per block; prefix-only blocks skip it), keeps the
-//                  running max / sum, writes P_j as bf16 into shared memory for the PV product and
-//                  folds PV_{j-1} from TMEM into its fp32 output row held in registers.
+//   softmax warps  8 warps, two threads per row (TMEM lane), each owning 64 of a block's 128 columns
+//                  and half of the output row: read S from TMEM (tcgen05.ld), apply the softmax scale
+//                  and the tree mask (one 128-bit ancestor set per row, turned into a 64-bit
+//                  visibility window per block half; prefix-only blocks skip it), exchange the row
+//                  maximum through shared memory, keep the running max / sum, write P_j as bf16
+//                  into shared memory for the PV product and fold PV_{j-1} from TMEM into the fp32
+//                  output half-row held in registers.
 //
 // All hand-offs are mbarriers (tcgen05.commit on the MMA side); every wait is bounded and reports
 // SB_ERR_CUDA instead of spinning forever.  The chunk results of the CTAs of a cluster are merged
 // through distributed shared memory exactly as in the mma.sync kernel.
+#include <cuda.h>
+
 #include <cstdio>
 #include <cstdlib>
 
@@ -26,18 +35,16 @@ namespace sb {
 
 constexpr int TC_BM = 128;           // rows per CTA
 constexpr int TC_BN = 128;           // keys per block
-constexpr int TC_SOFTMAX_THREADS = 128;
-constexpr int TC_MMA_WARP = 4;
-constexpr int TC_KLOAD_THREAD0 = 160;  // warps 5,6: K blocks and the Q tile
-constexpr int TC_VLOAD_THREAD0 = 224;  // warp 7: V blocks
-constexpr int TC_KLOADERS = 64;
-constexpr int TC_VLOADERS = 32;
-constexpr int TC_THREADS = 256;        // 8 warps = 2 per scheduler: up to 255 registers per thread
+constexpr int TC_SOFTMAX_THREADS = 256;  // warps 0-3: columns [0,64) of a block, warps 4-7: [64,128)
+constexpr int TC_MMA_WARP = 8;
+constexpr int TC_KLOAD_WARP = 9;     // lane 0 issues the Q and K loads
+constexpr int TC_VLOAD_WARP = 10;    // lane 0 issues the V loads; the warp zeroes rows past the sequence
+constexpr int TC_THREADS = 384;      // 12 warps (warp 11 only takes part in the barriers)
 constexpr int TC_TMEM_COLS = 512;
-constexpr int TC_SMALL_BYTES = 4096;   // ancestor masks, parents, barriers
+constexpr int TC_SMALL_BYTES = 8192; // ancestor masks, parents, barriers, softmax exchange
 
 enum TcBar { K_FULL0, K_FULL1, K_EMPTY0, K_EMPTY1, V_FULL0, V_FULL1, V_EMPTY0, V_EMPTY1, S_FULL0, S_FULL1,
-             S_EMPTY0, S_EMPTY1, P_FULL, PV_FULL, PV_EMPTY, TC_NUM_BARS };
+             S_EMPTY0, S_EMPTY1, P_FULL, PV_FULL, PV_EMPTY, V_TMA0, V_TMA1, Q_FULL, TC_NUM_BARS };
 
 template <int D>
 constexpr size_t attn_tc_smem_bytes() {
@@ -115,6 +122,24 @@ __device__ inline void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ inline void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// TMA tile load of one box of a rank-4 tensor (d, kv head, row in page, page) into shared memory.
+__device__ inline void tma_load_4d(uint32_t smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                   uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(smem_dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ inline void tma_load_3d(uint32_t smem_dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ inline void softmax_group_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ inline void cp_async_16_tc(uint32_t smem_dst, const void* gmem_src, int src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_dst), "l"(gmem_src), "r"(src_bytes));
 }
@@ -126,22 +151,29 @@ __device__ inline uint32_t sw128_chunk_off(int r, int ch, int rows) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams p,
+                                                                const __grid_constant__ CUtensorMap kmap,
+                                                                const __grid_constant__ CUtensorMap vmap,
+                                                                const __grid_constant__ CUtensorMap qmap,
+                                                                const int box_rows, const int q_tma) {
   constexpr int CH = D / 8;                   // 16-byte chunks per row
   constexpr int TILE_BYTES = TC_BN * D * 2;   // one K or V stage
+  constexpr int DH = D / 2;                   // output columns per softmax thread
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint32_t* s_anc = reinterpret_cast<uint32_t*>(base);               // 2048 B
   int* s_parent = reinterpret_cast<int*>(base + 2048);               // 512 B
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(base + 2560);        // TC_NUM_BARS * 8
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(base + 2560 + 256);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(base + 2560 + 260);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(base + 2816);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(base + 2820);
+  float* s_xmax = reinterpret_cast<float*>(base + 3072);             // [2 parities][2 halves][128 rows]
+  float* s_xl = reinterpret_cast<float*>(base + 5120);               // [2 halves][128 rows]
   uint8_t* sQ = base + TC_SMALL_BYTES;
   uint8_t* sK = sQ + TC_BM * D * 2;
   uint8_t* sV = sK + 2 * TILE_BYTES;
   uint8_t* sP = sV + 2 * TILE_BYTES;
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   cg::cluster_group cluster = cg::this_cluster();
   const int S = (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
@@ -149,26 +181,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const int Hkv = p.tb.n_kv_heads, Hq = p.tb.n_q_heads, G = p.G;
   const int g = blockIdx.y % Hkv, tile = blockIdx.y / Hkv;
   const int b = blockIdx.z;
-
-  if (tid == 0) *s_abort = 0;
-  const SeqPlan sp = plan_sequence(p, b, split == 0 && blockIdx.y == 0, s_parent, s_anc);
-  const SeqInfo& si = sp.info;
-  const int rows_total = si.nq * G;
+  const SeqPre pre = plan_lengths(p, b);
+  const int rows_total = pre.info.nq * G;
   const int row0 = tile * TC_BM;
-  if (!sp.can_write || row0 >= rows_total) return;  // uniform over the cluster
+  if (!pre.can_write || row0 >= rows_total) {  // uniform over the cluster
+    // the designated CTA always owns rows unless the sequence has none; its status is still due
+    if (split == 0 && blockIdx.y == 0 && tid == 0) p.status[b] = pre.info.err;
+    return;
+  }
   const long long rows_all = (long long)p.total_q * Hq;
 
-  // Balanced cut of the sequence's keys, in units of 16, into num_splits chunks.
-  const int L = si.P + si.n;
-  const int units = ceil_div(L, 16);
-  const int u_base = units / p.num_splits, u_rem = units % p.num_splits;
-  const int key_begin = 16 * (split * u_base + min(split, u_rem));
-  const int chunk_keys = sp.compute ? 16 * (u_base + (split < u_rem ? 1 : 0)) : 0;
-  const int nb = ceil_div(chunk_keys, TC_BN);
+  // Balanced cut of the sequence's 128-key blocks into num_splits chunks (block-aligned, so a
+  // TMA box never straddles a page); the sequence's last block is trimmed to a multiple of 16 keys.
+  const int L = pre.info.P + pre.info.n;
+  const int blocks_total = ceil_div(L, TC_BN);
+  const int b_base = blocks_total / p.num_splits, b_rem = blocks_total % p.num_splits;
+  const int key_begin = TC_BN * (split * b_base + min(split, b_rem));
+  const int nb = pre.info.err == 0 ? b_base + (split < b_rem ? 1 : 0) : 0;
+  const int chunk_keys = nb == 0 ? 0 : min(nb * TC_BN, ceil_div(L - key_begin, 16) * 16);
 
   if (tid == 0) {
-    const int counts[TC_NUM_BARS] = {TC_KLOADERS, TC_KLOADERS, 1, 1, TC_VLOADERS, TC_VLOADERS, 1, 1, 1, 1,
-                                     TC_SOFTMAX_THREADS, TC_SOFTMAX_THREADS, TC_SOFTMAX_THREADS, 1, TC_SOFTMAX_THREADS};
+    *s_abort = 0;
+    const int n = TC_SOFTMAX_THREADS;
+    const int counts[TC_NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, n, n, n, 1, n, 1, 1, q_tma ? 1 : n};
     for (int i = 0; i < TC_NUM_BARS; ++i) mbar_init(&s_bar[i], counts[i]);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -182,15 +217,78 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const uint32_t tmem = *s_tmem;
   const uint32_t tmem_pv = tmem + 2 * TC_BN;  // S buffers at columns [0,128) and [128,256), PV after them
 
-  // Row state of the softmax threads (thread t <-> row t <-> TMEM lane t).
-  float o_row[D];
+  // One TMA box per page piece of a block: box_rows keys x 64 columns, per 64-column half.
+  auto issue_block = [&](int j, const CUtensorMap* map, uint32_t stage_addr, uint64_t* bar) {
+    const int nj = min(TC_BN, chunk_keys - j * TC_BN);
+    const int k0 = key_begin + j * TC_BN;
+    const int pieces = ceil_div(nj, box_rows);
+    mbar_expect_tx(bar, (uint32_t)(pieces * box_rows * D * 2));
+    for (int i = 0; i < pieces; ++i) {
+      const int key = k0 + i * box_rows;
+      int c2, c3;
+      if (p.tb.page_size == 0) {
+        c2 = key;
+        c3 = b;
+      } else {
+        const int lp = key / p.tb.page_size;
+        int page = p.tb.page_table[(long long)b * p.tb.max_pages + lp];
+        if (page < 0 || page >= p.tb.num_pages) page = 0;  // reported by the designated CTA
+        c2 = key - lp * p.tb.page_size;
+        c3 = page;
+      }
+#pragma unroll
+      for (int h = 0; h < D / 64; ++h)
+        tma_load_4d(stage_addr + h * (TC_BN * 128) + i * box_rows * 128, map, h * 64, g, c2, c3, bar);
+    }
+  };
+  // The first loads go out before anything else: they only need the sequence's lengths.
+  if (nb > 0 && lane == 0) {
+    if (warp == TC_KLOAD_WARP) {
+      if (q_tma) {
+        mbar_expect_tx(&s_bar[Q_FULL], (uint32_t)(TC_BM * D * 2));
+#pragma unroll
+        for (int h = 0; h < D / 64; ++h)
+          tma_load_3d(smem_u32(sQ) + h * (TC_BM * 128), &qmap, h * 64, g * G, pre.info.q_off + tile * (TC_BM / G),
+                      &s_bar[Q_FULL]);
+      }
+      issue_block(0, &kmap, smem_u32(sK), &s_bar[K_FULL0]);
+      if (nb > 1) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
+    } else if (warp == TC_VLOAD_WARP) {
+      issue_block(0, &vmap, smem_u32(sV), &s_bar[V_TMA0]);
+      if (nb > 1) issue_block(1, &vmap, smem_u32(sV) + TILE_BYTES, &s_bar[V_TMA1]);
+    }
+  }
+  const SeqPlan sp = plan_tree(p, b, split == 0 && blockIdx.y == 0, pre, s_parent, s_anc);
+  const SeqInfo& si = sp.info;
+
+  // Row state of the softmax threads: row = TMEM lane, `half` selects the 64 columns of every block
+  // and the half of the output row this thread owns.
+  float o_row[DH];
   float m_run = -INFINITY, l_run = 0.f;
 #pragma unroll
-  for (int d = 0; d < D; ++d) o_row[d] = 0.f;
+  for (int d = 0; d < DH; ++d) o_row[d] = 0.f;
+  const int half = (warp >> 2) & 1;
+  const int row = (warp & 3) * 32 + lane;
 
   if (tid < TC_SOFTMAX_THREADS) {
     // ------------------------------------------------------------------ softmax warps
-    const int R = row0 + tid;
+    if (!q_tma && nb > 0) {  // Q tile as a gather of (node, head) rows
+      const uint32_t qd = smem_u32(sQ);
+      for (int c = tid; c < TC_BM * CH; c += TC_SOFTMAX_THREADS) {
+        const int r = c / CH, ch = c % CH;
+        const int R = row0 + r;
+        const bool valid = R < rows_total;
+        const int node_l = valid ? R / G : 0;
+        const int hh = valid ? R - node_l * G : 0;
+        const long long off = ((long long)(si.q_off + node_l) * Hq + g * G + hh) * D + ch * 8;
+        cp_async_16_tc(qd + sw128_chunk_off(r, ch, TC_BM), p.q + (valid ? off : 0), valid ? 16 : 0);
+      }
+      asm volatile("cp.async.commit_group;\n" ::);
+      asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+      fence_async_smem();
+      mbar_arrive(&s_bar[Q_FULL]);
+    }
+    const int R = row0 + row;
     const bool row_live = R < rows_total && sp.compute;
     uint32_t anc[4];
     {
@@ -198,52 +296,49 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
 #pragma unroll
       for (int w = 0; w < 4; ++w) anc[w] = row_live ? s_anc[4 * node + w] : 0u;
     }
-    const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
+    const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
     float corr_prev = 1.f;  // rescale of o_row that belongs to the PV block still in flight
     bool ok = true;
-    for (int j = 0; j < nb && ok; ++j) {
+    // The trip count and the named barrier inside are uniform over the 256 threads: after a failed
+    // wait the remaining waits return at once (abort flag) and the loop just runs out.
+    for (int j = 0; j < nb; ++j) {
       const int k0 = key_begin + j * TC_BN;
       const int nj = min(TC_BN, chunk_keys - j * TC_BN);  // keys of this block (multiple of 16)
-      ok = mbar_wait(&s_bar[S_FULL0 + (j & 1)], (j >> 1) & 1, s_abort);
-      if (!ok) break;
+      const int my_cols = nj - 64 * half;                 // valid columns among this thread's 64
+      if (ok) ok = mbar_wait(&s_bar[S_FULL0 + (j & 1)], (j >> 1) & 1, s_abort);
       tc_fence_after();
-      const uint32_t t_s = tmem + lane_base + (j & 1) * TC_BN;
-      // visibility of columns [0,64) and [64,128): tree mask where the block reaches past the
-      // prefix, and only the block's own nj columns
-      uint64_t win[2];
-      const bool need_mask = k0 + TC_BN > si.P;
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint64_t w = need_mask ? visibility_window(anc, k0 + 64 * h - si.P) : ~0ull;
-        const int cols = nj - 64 * h;
-        w &= cols >= 64 ? ~0ull : (cols <= 0 ? 0ull : ((1ull << cols) - 1ull));
-        win[h] = w;
-      }
-      // pass 1: row maximum
+      const uint32_t t_s = tmem + lane_base + (j & 1) * TC_BN + 64 * half;
+      // visibility of this thread's 64 columns: tree mask where the block reaches past the prefix,
+      // and only the block's own nj columns
+      uint64_t win = k0 + TC_BN > si.P ? visibility_window(anc, k0 + 64 * half - si.P) : ~0ull;
+      win &= my_cols >= 64 ? ~0ull : (my_cols <= 0 ? 0ull : ((1ull << my_cols) - 1ull));
+      // pass 1: row maximum over both halves
       float mx = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < TC_BN / 32; ++c) {
-        if (c * 32 < nj) {
+      for (int c = 0; c < 2; ++c) {
+        if (c * 32 < my_cols) {
           uint32_t r[32];
           tmem_ld32(t_s + c * 32, r);
-          const uint32_t m32 = (uint32_t)(win[c >> 1] >> ((c & 1) * 32));
+          const uint32_t m32 = (uint32_t)(win >> (c * 32));
 #pragma unroll
           for (int i = 0; i < 32; ++i) mx = fmaxf(mx, ((m32 >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
         }
       }
+      s_xmax[((j & 1) * 2 + half) * TC_BM + row] = mx;
+      softmax_group_sync();
+      mx = fmaxf(mx, s_xmax[((j & 1) * 2 + (half ^ 1)) * TC_BM + row]);
       mx *= p.scale_log2;  // scale > 0: max commutes with it (-inf stays -inf)
       const float m_new = fmaxf(m_run, mx);
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       const float corr = fast_exp2(m_run - m_use);
-      // fold the previous block's PV into the output row (also frees P and the PV accumulator)
+      // fold the previous block's PV into the output half-row (also frees P and the PV accumulator)
       if (j > 0) {
-        ok = mbar_wait(&s_bar[PV_FULL], (j - 1) & 1, s_abort);
-        if (!ok) break;
+        if (ok) ok = mbar_wait(&s_bar[PV_FULL], (j - 1) & 1, s_abort);
         tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < DH / 32; ++c) {
           uint32_t r[32];
-          tmem_ld32(tmem_pv + lane_base + c * 32, r);
+          tmem_ld32(tmem_pv + lane_base + half * DH + c * 32, r);
 #pragma unroll
           for (int i = 0; i < 32; ++i) o_row[c * 32 + i] = o_row[c * 32 + i] * corr_prev + __uint_as_float(r[i]);
         }
@@ -253,11 +348,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       // pass 2: probabilities -> P (bf16, K-major swizzled), running sum
       float lsum = 0.f;
 #pragma unroll
-      for (int c = 0; c < TC_BN / 32; ++c) {
-        if (c * 32 < nj) {
+      for (int c = 0; c < 2; ++c) {
+        if (c * 32 < my_cols) {
           uint32_t r[32];
           tmem_ld32(t_s + c * 32, r);
-          const uint32_t m32 = (uint32_t)(win[c >> 1] >> ((c & 1) * 32));
+          const uint32_t m32 = (uint32_t)(win >> (c * 32));
           uint32_t packed[16];
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
@@ -269,8 +364,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
           }
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            const int ch = c * 4 + q;  // 16-byte chunk (8 keys) of this row
-            *reinterpret_cast<uint4*>(sP + sw128_chunk_off(tid, ch, TC_BM)) =
+            const int ch = half * 8 + c * 4 + q;  // 16-byte chunk (8 keys) of this row
+            *reinterpret_cast<uint4*>(sP + sw128_chunk_off(row, ch, TC_BM)) =
                 make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
           }
         }
@@ -283,23 +378,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       fence_async_smem();
       mbar_arrive(&s_bar[P_FULL]);
     }
-    if (ok && nb > 0) {
-      ok = mbar_wait(&s_bar[PV_FULL], (nb - 1) & 1, s_abort);
-      if (ok) {
-        tc_fence_after();
+    if (nb > 0) {
+      if (ok) ok = mbar_wait(&s_bar[PV_FULL], (nb - 1) & 1, s_abort);
+      tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tmem_pv + lane_base + c * 32, r);
+      for (int c = 0; c < DH / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_pv + lane_base + half * DH + c * 32, r);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o_row[c * 32 + i] = o_row[c * 32 + i] * corr_prev + __uint_as_float(r[i]);
-        }
+        for (int i = 0; i < 32; ++i) o_row[c * 32 + i] = o_row[c * 32 + i] * corr_prev + __uint_as_float(r[i]);
       }
     }
+    s_xl[half * TC_BM + row] = l_run;
     if (!ok) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
   } else if (warp == TC_MMA_WARP) {
     // ------------------------------------------------------------------ MMA issuer
-    if ((tid & 31) == 0 && nb > 0) {
+    if (lane == 0 && nb > 0) {
       const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV), p_addr = smem_u32(sP);
       bool ok = true;
       auto issue_s = [&](int j) {
@@ -315,7 +409,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
         tc_commit(&s_bar[S_FULL0 + (j & 1)]);
         tc_commit(&s_bar[K_EMPTY0 + (j & 1)]);
       };
-      ok = mbar_wait(&s_bar[K_FULL0], 0, s_abort);
+      ok = mbar_wait(&s_bar[Q_FULL], 0, s_abort);
+      if (ok) ok = mbar_wait(&s_bar[K_FULL0], 0, s_abort);
       if (ok) {
         tc_fence_after();
         issue_s(0);
@@ -347,96 +442,126 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       }
       if (!ok) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
     }
-  } else {
-    // ------------------------------------------------------------------ loader warps
-    const bool is_k = tid < TC_VLOAD_THREAD0;
-    const int lt = tid - (is_k ? TC_KLOAD_THREAD0 : TC_VLOAD_THREAD0);
-    const int n_loaders = is_k ? TC_KLOADERS : TC_VLOADERS;
-    const bf16* src = static_cast<const bf16*>(is_k ? p.tb.k_cache : p.tb.v_cache) + (long long)g * D;
-    const uint32_t dst0 = smem_u32(is_k ? sK : sV);
-    auto issue_block = [&](int j) {
-      const int nj = min(TC_BN, chunk_keys - j * TC_BN);
-      const int k0 = key_begin + j * TC_BN;
-      const uint32_t dst = dst0 + (j & 1) * TILE_BYTES;
-      for (int c = lt; c < nj * CH; c += n_loaders) {
-        const int r = c / CH, ch = c % CH;
-        const int key = k0 + r;
-        const bool valid = key < L;  // keys past the sequence inside the last unit of 16: zeros
-        const long long off = valid ? kv_row_elem_offset(p.tb, b, key) + ch * 8 : 0;
-        cp_async_16_tc(dst + sw128_chunk_off(r, ch, TC_BN), src + off, valid ? 16 : 0);
-      }
-    };
-    if (nb > 0) {
-      if (is_k) {
-        // the query tile travels with the first K block
-        const uint32_t qd = smem_u32(sQ);
-        for (int c = lt; c < TC_BM * CH; c += n_loaders) {
-          const int r = c / CH, ch = c % CH;
-          const int R = row0 + r;
-          const bool valid = R < rows_total;
-          const int node_l = valid ? R / G : 0;
-          const int hh = valid ? R - node_l * G : 0;
-          const long long off = ((long long)(si.q_off + node_l) * Hq + g * G + hh) * D + ch * 8;
-          cp_async_16_tc(qd + sw128_chunk_off(r, ch, TC_BM), p.q + (valid ? off : 0), valid ? 16 : 0);
-        }
-      }
-      issue_block(0);
-      asm volatile("cp.async.commit_group;\n" ::);
-      if (nb > 1) {
-        issue_block(1);
-        asm volatile("cp.async.commit_group;\n" ::);
-      }
+  } else if (warp == TC_KLOAD_WARP) {
+    // ------------------------------------------------------------------ K loader (blocks 2..)
+    if (lane == 0) {
       bool ok = true;
-      uint64_t* full = &s_bar[is_k ? K_FULL0 : V_FULL0];
-      uint64_t* empty = &s_bar[is_k ? K_EMPTY0 : V_EMPTY0];
-      for (int j = 0; j < nb; ++j) {
-        if (j + 1 < nb) asm volatile("cp.async.wait_group 1;\n" ::: "memory");
-        else asm volatile("cp.async.wait_group 0;\n" ::: "memory");
-        fence_async_smem();
-        mbar_arrive(&full[j & 1]);
-        if (j + 2 < nb) {
-          ok = mbar_wait(&empty[j & 1], (j >> 1) & 1, s_abort);
-          if (!ok) break;
-          issue_block(j + 2);
-          asm volatile("cp.async.commit_group;\n" ::);
-        }
+      for (int j = 2; j < nb && ok; ++j) {
+        ok = mbar_wait(&s_bar[K_EMPTY0 + (j & 1)], ((j >> 1) - 1) & 1, s_abort);
+        if (ok) issue_block(j, &kmap, smem_u32(sK) + (j & 1) * TILE_BYTES, &s_bar[K_FULL0 + (j & 1)]);
       }
-      asm volatile("cp.async.wait_group 0;\n" ::: "memory");
       if (!ok) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
     }
+  } else if (warp == TC_VLOAD_WARP) {
+    // ------------------------------------------------------------------ V loader
+    bool ok = true;
+    for (int j = 0; j < nb && ok; ++j) {
+      ok = mbar_wait(&s_bar[V_TMA0 + (j & 1)], (j >> 1) & 1, s_abort);
+      if (!ok) break;
+      // rows of this block that lie past the end of the sequence: zero them (at most 15)
+      const int nj = min(TC_BN, chunk_keys - j * TC_BN);
+      const int first_bad = L - (key_begin + j * TC_BN);
+      if (first_bad < nj) {
+        uint8_t* stage = sV + (j & 1) * TILE_BYTES;
+        for (int c = lane; c < (nj - first_bad) * CH; c += 32) {
+          const int r = first_bad + c / CH, ch = c % CH;
+          *reinterpret_cast<uint4*>(stage + sw128_chunk_off(r, ch, TC_BN)) = make_uint4(0, 0, 0, 0);
+        }
+        fence_async_smem();
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&s_bar[V_FULL0 + (j & 1)]);
+        if (j + 2 < nb) {
+          ok = mbar_wait(&s_bar[V_EMPTY0 + (j & 1)], (j >> 1) & 1, s_abort);
+          if (ok) issue_block(j + 2, &vmap, smem_u32(sV) + (j & 1) * TILE_BYTES, &s_bar[V_TMA0 + (j & 1)]);
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    }
+    if (!ok && lane == 0) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
   }
 
-  // ---- park (O, m, l) of this chunk, merge over the cluster, store ----------------------------
-  constexpr int RS = D + 8;
-  float* s_red = reinterpret_cast<float*>(sK);  // the K/V stages are idle once the last PV is folded
-  float* s_m = s_red + TC_BM * RS;
-  float* s_l = s_m + TC_BM;
-  float* s_w = s_l + TC_BM;
-  float* s_lse = s_w + TC_BM + 8;
+  // ---- push (O, m, l) of this chunk to the owning CTAs of the cluster, reduce, store -------------
+  MergeBuf<D> mb(reinterpret_cast<float*>(sK), TC_BM, S);  // the K/V stages are idle once the last PV is folded
   tc_fence_before();
   __syncthreads();  // every role is done: no async read of the stages is in flight any more
+  if (S > 1) cluster.sync();  // ... in any CTA of the cluster: their stages are about to be written remotely
   if (tid < TC_SOFTMAX_THREADS) {
-    if (nb > 0) {
+    const bool have = nb > 0 && sp.compute;
+    if (have) {
+      int slot;
+      float* dst = merge_row_dst<D>(cluster, mb, crank, row, &slot) + half * DH;
 #pragma unroll
-      for (int d = 0; d < D; d += 4)
-        *reinterpret_cast<float4*>(s_red + tid * RS + d) = make_float4(o_row[d], o_row[d + 1], o_row[d + 2], o_row[d + 3]);
+      for (int d = 0; d < DH; d += 4)
+        *reinterpret_cast<float4*>(dst + d) = make_float4(o_row[d], o_row[d + 1], o_row[d + 2], o_row[d + 3]);
     }
-    s_m[tid] = m_run;
-    s_l[tid] = l_run;
+    if (half == 0)
+      merge_push_ml<D>(cluster, mb, crank, row, have ? m_run : -INFINITY, have ? s_xl[row] + s_xl[TC_BM + row] : 0.f);
   }
   if (S > 1) cluster.sync(); else __syncthreads();
   if (warp == TC_MMA_WARP) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS));
   }
-  cluster_merge_and_store<D, TC_BM>(p, cluster, S, crank, s_red, s_m, s_l, s_w, s_lse, split / S, row0, rows_total, g,
-                                    si.q_off, rows_all, tid, TC_THREADS);
-  if (S > 1) cluster.sync();
+  merge_reduce_and_store<D, TC_BM>(p, mb, S, crank, split / S, row0, rows_total, g, si.q_off, rows_all, tid, TC_THREADS);
 }
 
 // ---------------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------------
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+// Rank-4 view (d, kv head, row, page) of a K or V cache; a contiguous cache is one "page" of
+// kv_capacity rows per sequence.  Box = 64 columns x 1 head x box_rows rows, 128-byte swizzle,
+// out-of-range rows read as zero.
+static bool make_kv_map(CUtensorMap* map, const sb_tree_batch& tb, const void* cache, int box_rows) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return false;
+  const cuuint64_t D = (cuuint64_t)tb.head_dim, H = (cuuint64_t)tb.n_kv_heads;
+  const cuuint64_t rows = tb.page_size == 0 ? (cuuint64_t)tb.kv_capacity : (cuuint64_t)tb.page_size;
+  const cuuint64_t pages = tb.page_size == 0 ? (cuuint64_t)tb.batch : (cuuint64_t)tb.num_pages;
+  const cuuint64_t dims[4] = {D, H, rows, pages};
+  const cuuint64_t strides[3] = {D * 2, H * D * 2, rows * H * D * 2};
+  const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
+  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(cache), dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Rank-3 view (d, query head, query row) of Q; box = 64 columns x G heads x 128/G rows lands in
+// shared memory as the tile's 128 packed (node, head-in-group) rows.
+static bool make_q_map(CUtensorMap* map, const AttnParams& p) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return false;
+  const cuuint64_t D = (cuuint64_t)p.tb.head_dim, H = (cuuint64_t)p.tb.n_q_heads;
+  const cuuint64_t dims[3] = {D, H, (cuuint64_t)p.total_q};
+  const cuuint64_t strides[2] = {D * 2, H * D * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)p.G, (cuuint32_t)(TC_BM / p.G)};
+  const cuuint32_t elem[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(p.q), dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 template <int D>
 static cudaLaunchConfig_t tc_config(dim3 grid, int cluster, cudaStream_t cs, cudaLaunchAttribute* attr) {
@@ -499,7 +624,17 @@ static sb_status launch_tc(const AttnParams& p, dim3 grid, int cluster, cudaStre
   if (getenv("SB_DEBUG"))
     fprintf(stderr, "[sb] attn_tc<%d> grid (%u,%u,%u) cluster %d outer %d: max active clusters %d\n", D, grid.x, grid.y,
             grid.z, cluster, p.outer, attn_tc_max_active_clusters(D, cluster));
-  if (cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p) != cudaSuccess) {
+  const int box_rows = p.tb.page_size == 0 ? TC_BN : (p.tb.page_size < TC_BN ? p.tb.page_size : TC_BN);
+  CUtensorMap kmap, vmap, qmap;
+  if (!make_kv_map(&kmap, p.tb, p.tb.k_cache, box_rows) || !make_kv_map(&vmap, p.tb, p.tb.v_cache, box_rows))
+    return SB_ERR_CUDA;
+  const int q_tma = (TC_BM % p.G == 0) ? 1 : 0;
+  if (q_tma) {
+    if (!make_q_map(&qmap, p)) return SB_ERR_CUDA;
+  } else {
+    qmap = kmap;  // unused by the kernel in this mode
+  }
+  if (cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, kmap, vmap, qmap, box_rows, q_tma) != cudaSuccess) {
     cudaGetLastError();
     return SB_ERR_CUDA;
   }
