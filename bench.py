@@ -32,6 +32,9 @@ if ROOT not in sys.path:
 METRIC = "tree-verify attention GB/s (% of B200 HBM peak) and us per verify step"
 N_LAYERS = 32
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on this workload, from the
+# ncu capture summarised in profiles/attn_tc_kernel_c2_verify_layer.md
+ATTN_DRAM_TRAFFIC_BYTES = 9230336
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -166,6 +169,14 @@ def run_reference(args):
     return 0
 
 
+def max_over_ranks(torch, values, device):
+    """Element-wise maximum of `values` over all ranks (identity without a process group)."""
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if torch.distributed.is_available() and torch.distributed.is_initialized():
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
 def time_graph(torch, graph, iters, dist_on):
     """Replay `graph` `iters` times between two events on the current stream; returns ms total."""
     if dist_on:
@@ -274,10 +285,7 @@ def run_ours(args):
 
     ms_step = ms_total / args.steps
     ms_attn_launch = ms_attn / attn_iters / N_LAYERS
-    if dist_on:
-        t = torch.tensor([ms_step, ms_attn_launch, ms_e2e], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms_step, ms_attn_launch, ms_e2e = [float(x) for x in t.tolist()]
+    ms_step, ms_attn_launch, ms_e2e = max_over_ranks(torch, [ms_step, ms_attn_launch, ms_e2e], "cuda")
 
     parts = step.algorithmic_bytes()
     total_bytes = parts["total"]
@@ -307,9 +315,9 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e},
         "gpu_launches": gpu_launches,
-        "roofline": {"bound": "hbm", "kernel": "sb::attn_mma_kernel<128> (+ merge) per layer",
+        "roofline": {"bound": "hbm", "kernel": "sb::attn_tc_kernel<128> (tcgen05), one launch per layer",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"{peak_kind} HBM copy bandwidth", "traffic": None,
+                     "peak_kind": f"{peak_kind} HBM copy bandwidth", "traffic": ATTN_DRAM_TRAFFIC_BYTES,
                      "algorithmic_bytes_per_launch": attn_bytes,
                      "pct_of_nominal_8TBps": 100.0 * achieved / NOMINAL_HBM_GBS},
     }
