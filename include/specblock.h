@@ -190,6 +190,35 @@ sb_status sb_verify_accept(const void* logits, sb_dtype dtype, int64_t row_strid
 size_t sb_verify_accept_workspace_bytes(int32_t total_nodes, int32_t vocab);
 
 /*
+ * sb_verify_accept_static -- sb_verify_accept for callers that cannot provide scratch memory.
+ * (The paper has no counterpart for this call; it exists for integration reasons only.)
+ *
+ *   Some hosts of this library never get to call cudaMalloc themselves: a plugin that runs inside
+ *   another runtime's pre-sized memory arena, a process whose device memory was carved up once at
+ *   start-up, or code that runs where an allocation would synchronise the device at a bad moment.
+ *   For them this variant takes no workspace: the per-chunk argmax partials live in a fixed
+ *   SB_STATIC_SCRATCH_BYTES array that is part of the library image (every GPU that loads the
+ *   library holds these bytes until the process exits).  Arguments, results and status words are
+ *   exactly those of sb_verify_accept; inputs and outputs are still the caller's buffers.
+ *
+ *   - The call allocates and frees nothing, on the host or on the device.
+ *   - Problems whose scratch need (sb_verify_accept_workspace_bytes) exceeds SB_STATIC_SCRATCH_BYTES
+ *     are refused with SB_ERR_WORKSPACE; use sb_verify_accept with your own workspace for those.
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it
+ *     (nothing in it has to start at zero: every partial is rewritten before it is read).  Two
+ *     calls that can overlap on the GPU -- different streams, or graph branches -- race on it;
+ *     serialise them or use sb_verify_accept with separate workspaces.
+ */
+#define SB_STATIC_SCRATCH_BYTES (256 * 1024)
+sb_status sb_verify_accept_static(const void* logits, sb_dtype dtype, int64_t row_stride, int32_t vocab,
+                                  int32_t batch, int32_t total_nodes, const int32_t* node_offsets,
+                                  const int32_t* parent, const int32_t* tok, int32_t max_depth,
+                                  int32_t* amax, int32_t* accept_len, int32_t* path_nodes,
+                                  int32_t* out_tokens, int32_t* bonus, int32_t* status, void* stream);
+
+/*
  * sb_kv_compact -- keep the committed positions' K/V, drop the rest (Sec. 3.1 / App. A.2: later
  * forwards see every committed position's cached keys and values as the verified prefix).
  *

@@ -65,7 +65,7 @@ def load(build_if_missing: bool = True):
                  "sb_verify_accept_workspace_bytes"):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
-                 "sb_kv_compact"):
+                 "sb_verify_accept_static", "sb_kv_compact"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -73,7 +73,8 @@ def load(build_if_missing: bool = True):
 
 EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspace_bytes",
             "sb_tree_expand", "sb_tree_expand_workspace_bytes", "sb_verify_accept",
-            "sb_verify_accept_workspace_bytes", "sb_kv_compact", "sb_status_string", "sb_version",
+            "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
+            "sb_status_string", "sb_version",
             "sb_kernel_launch_count")
 
 
@@ -226,6 +227,28 @@ def sb_verify_accept(logits, node_offsets, parent, tok, max_depth, *, vocab=None
                               _ptr(out["out_tokens"]), _ptr(out["bonus"]), _ptr(workspace),
                               C.c_size_t(workspace.numel()), _ptr(out["status"]), _stream())
     _check(rc, "sb_verify_accept")
+    return out
+
+
+SB_STATIC_SCRATCH_BYTES = 256 * 1024
+
+
+def sb_verify_accept_static(logits, node_offsets, parent, tok, max_depth, out, *, vocab=None):
+    """sb_verify_accept without a workspace, for callers that cannot allocate device memory: the
+    library's own fixed scratch array is used (at most SB_STATIC_SCRATCH_BYTES of partials, else
+    SB_ERR_WORKSPACE).  `out` must hold the preallocated result tensors (amax, accept_len,
+    path_nodes, out_tokens, bonus, status): nothing is allocated here either.  Calls that may
+    overlap on the GPU share that array and must be serialised by the caller."""
+    total, stride = logits.shape
+    vocab = stride if vocab is None else vocab
+    batch = node_offsets.numel() - 1
+    dt = {torch.bfloat16: SB_BF16, torch.float32: SB_F32}[logits.dtype]
+    rc = load().sb_verify_accept_static(
+        _ptr(logits), C.c_int(dt), C.c_int64(stride), C.c_int32(vocab), C.c_int32(batch), C.c_int32(total),
+        _ptr(node_offsets, torch.int32), _ptr(parent, torch.int32), _ptr(tok, torch.int32),
+        C.c_int32(max_depth), _ptr(out["amax"]), _ptr(out["accept_len"]), _ptr(out["path_nodes"]),
+        _ptr(out["out_tokens"]), _ptr(out["bonus"]), _ptr(out["status"]), _stream())
+    _check(rc, "sb_verify_accept_static")
     return out
 
 

@@ -235,3 +235,67 @@ extern "C" sb_status sb_verify_accept(const void* logits, sb_dtype dtype, int64_
                                                 out_tokens, bonus, status);
   return launch_check();
 }
+
+// ---------------------------------------------------------------------------------------------------
+// sb_verify_accept_static: the same two kernels, with their scratch in a fixed array of the library
+// image instead of a caller workspace -- for callers that have no way to allocate device memory.
+// ---------------------------------------------------------------------------------------------------
+
+// In host code this name is only a handle for the runtime, not a device address: the address each
+// device uses comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_accept_scratch[SB_STATIC_SCRATCH_BYTES];
+
+extern "C" sb_status sb_verify_accept_static(const void* logits, sb_dtype dtype, int64_t row_stride, int32_t vocab,
+                                             int32_t batch, int32_t total_nodes, const int32_t* node_offsets,
+                                             const int32_t* parent, const int32_t* tok, int32_t max_depth,
+                                             int32_t* amax, int32_t* accept_len, int32_t* path_nodes,
+                                             int32_t* out_tokens, int32_t* bonus, int32_t* status, void* stream) {
+  using namespace sb;
+  if (!logits || !node_offsets || !parent || !tok || !amax || !accept_len || !path_nodes || !out_tokens ||
+      !bonus || !status || batch < 1 || total_nodes < 1 || vocab < 1 || row_stride < vocab)
+    return SB_ERR_INVALID_ARG;
+  if (dtype != SB_BF16 && dtype != SB_F32) return SB_ERR_INVALID_ARG;
+  if (max_depth < 0 || max_depth > SB_MAX_DEPTH || total_nodes > 65535) return SB_ERR_UNSUPPORTED;
+  const size_t need = sb_verify_accept_workspace_bytes(total_nodes, vocab);
+  if (need > (size_t)SB_STATIC_SCRATCH_BYTES) return SB_ERR_WORKSPACE;  // larger than the fixed array
+
+  // Device address of the array, looked up once per device with that device current.
+  constexpr int kMaxDevices = 64;
+  static void* scratch_of_device[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return SB_ERR_CUDA;
+  if (dev >= kMaxDevices) return SB_ERR_UNSUPPORTED;
+  if (!scratch_of_device[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_accept_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return SB_ERR_CUDA;
+    }
+    scratch_of_device[dev] = ptr;
+  }
+  char* scratch = static_cast<char*>(scratch_of_device[dev]);
+
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int esz = dtype == SB_BF16 ? 2 : 4;
+  const int vec = 16 / esz;
+  const int nc = argmax_chunks(total_nodes, vocab, vec);
+  int chunk = ceil_div(vocab, nc);
+  chunk = ceil_div(chunk, vec) * vec;
+  const bool vec_ok = (reinterpret_cast<uintptr_t>(logits) & 15) == 0 && (row_stride * esz) % 16 == 0;
+  float* part_val = reinterpret_cast<float*>(scratch);
+  int* part_idx = reinterpret_cast<int*>(scratch + need / 2);
+  dim3 grid(nc, total_nodes);
+  if (dtype == SB_BF16)
+    row_argmax_kernel<uint16_t><<<grid, ARGMAX_THREADS, 0, cs>>>(static_cast<const uint16_t*>(logits),
+                                                                 row_stride, vocab, chunk, nc, vec_ok,
+                                                                 part_val, part_idx);
+  else
+    row_argmax_kernel<float><<<grid, ARGMAX_THREADS, 0, cs>>>(static_cast<const float*>(logits), row_stride,
+                                                              vocab, chunk, nc, vec_ok, part_val, part_idx);
+  sb_status st = launch_check();
+  if (st != SB_OK) return st;
+  accept_kernel<<<batch, SB_MAX_NODES, 0, cs>>>(nc, part_val, part_idx, node_offsets, parent, tok,
+                                                total_nodes, max_depth, amax, accept_len, path_nodes,
+                                                out_tokens, bonus, status);
+  return launch_check();
+}
