@@ -12,14 +12,16 @@
 //                  The Q tile is one TMA box {64 columns, G heads, 128/G nodes} per column half when
 //                  G divides 128, else a 16-byte cp.async gather by the softmax warps;
 //   MMA warp       one thread issues  S_j = Q K_j^T  (tcgen05.mma, fp32 accumulator in TMEM, two S
-//                  buffers so S_{j+1} runs under the softmax of block j) and  PV_j = P_j V_j;
-//   softmax warps  8 warps, two threads per row (TMEM lane), each owning 64 of a block's 128 columns
-//                  and half of the output row: read S from TMEM (tcgen05.ld), apply the softmax scale
-//                  and the tree mask (one 128-bit ancestor set per row, turned into a 64-bit
-//                  visibility window per block half; prefix-only blocks skip it), exchange the row
-//                  maximum through shared memory, keep the running max / sum, write P_j as bf16
-//                  into shared memory for the PV product and fold PV_{j-1} from TMEM into the fp32
-//                  output half-row held in registers.
+//                  buffers) and  O += P_j V_j  with P_j read from TMEM and O accumulated in TMEM;
+//   softmax warps  8 warps, two threads per row (TMEM lane), each owning 64 of a block's 128 columns:
+//                  read S once from TMEM into registers (tcgen05.ld; the S buffer is released at
+//                  once), apply the softmax scale and the tree mask (one 128-bit ancestor set per
+//                  row, turned into a 64-bit visibility window per block half; prefix-only blocks
+//                  skip it), exchange the row maximum through shared memory, and write
+//                  P_j = 2^(s - m_ref) as packed bf16 back into TMEM (tcgen05.st, two P buffers).
+//                  m_ref is a lazily updated reference maximum: it moves (and O and the running
+//                  sum are rescaled, tcgen05.ld/st) only when a block's maximum exceeds it by more
+//                  than 8 in the base-2 domain, so P never exceeds 2^8 and the rescale is rare.
 //
 // All hand-offs are mbarriers (tcgen05.commit on the MMA side); every wait is bounded and reports
 // SB_ERR_CUDA instead of spinning forever.  The chunk results of the CTAs of a cluster are merged
@@ -42,14 +44,16 @@ constexpr int TC_VLOAD_WARP = 10;    // lane 0 issues the V loads; the warp zero
 constexpr int TC_THREADS = 384;      // 12 warps (warp 11 only takes part in the barriers)
 constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_SMALL_BYTES = 8192; // ancestor masks, parents, barriers, softmax exchange
+constexpr int TC_MERGE_TAIL = 8192;  // the merge receive buffer = the V stages + this tail
 
 enum TcBar { K_FULL0, K_FULL1, K_EMPTY0, K_EMPTY1, V_FULL0, V_FULL1, V_EMPTY0, V_EMPTY1, S_FULL0, S_FULL1,
-             S_EMPTY0, S_EMPTY1, P_FULL, PV_FULL, PV_EMPTY, V_TMA0, V_TMA1, Q_FULL, TC_NUM_BARS };
+             S_EMPTY0, S_EMPTY1, P_FULL, PV_FULL, V_TMA0, V_TMA1, Q_FULL, MERGE_BAR, TC_NUM_BARS };
 
 template <int D>
 constexpr size_t attn_tc_smem_bytes() {
-  // small region + Q + 2 K stages + 2 V stages + P, plus slack to align the tiles to 1024 bytes
-  return 1024 + TC_SMALL_BYTES + (size_t)TC_BM * D * 2 + 4 * (size_t)TC_BN * D * 2 + (size_t)TC_BM * TC_BN * 2;
+  // small region + Q + 2 K stages + 2 V stages + tail of the merge receive buffer, plus slack to
+  // align the tiles to 1024 bytes
+  return 1024 + TC_SMALL_BYTES + (size_t)TC_BM * D * 2 + 4 * (size_t)TC_BN * D * 2 + TC_MERGE_TAIL;
 }
 
 __device__ inline uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -139,7 +143,59 @@ __device__ inline void tma_load_3d(uint32_t smem_dst, const CUtensorMap* map, in
       ::"r"(smem_dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// Address of `smem_addr` (a shared::cta address of this CTA's window) in CTA `rank` of the cluster.
+__device__ inline uint32_t mapa_u32(uint32_t smem_addr, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+// Bulk asynchronous copy from this CTA's shared memory into a cluster peer's; the bytes are
+// credited to the peer's mbarrier.  Sizes and addresses are multiples of 16 bytes.
+__device__ inline void dsmem_bulk_copy(uint32_t dst_cluster_addr, uint32_t src_cta_addr, uint32_t bytes,
+                                       uint32_t mbar_cluster_addr) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   dst_cluster_addr),
+               "r"(src_cta_addr), "r"(bytes), "r"(mbar_cluster_addr)
+               : "memory");
+}
 __device__ inline void softmax_group_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// 32 consecutive 32-bit columns of this thread's TMEM lane <- registers.
+__device__ inline void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ inline void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Two 32-column loads in flight, one wait.
+__device__ inline void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        : "=r"(r[32 * h + 0]), "=r"(r[32 * h + 1]), "=r"(r[32 * h + 2]), "=r"(r[32 * h + 3]), "=r"(r[32 * h + 4]),
+          "=r"(r[32 * h + 5]), "=r"(r[32 * h + 6]), "=r"(r[32 * h + 7]), "=r"(r[32 * h + 8]), "=r"(r[32 * h + 9]),
+          "=r"(r[32 * h + 10]), "=r"(r[32 * h + 11]), "=r"(r[32 * h + 12]), "=r"(r[32 * h + 13]), "=r"(r[32 * h + 14]),
+          "=r"(r[32 * h + 15]), "=r"(r[32 * h + 16]), "=r"(r[32 * h + 17]), "=r"(r[32 * h + 18]), "=r"(r[32 * h + 19]),
+          "=r"(r[32 * h + 20]), "=r"(r[32 * h + 21]), "=r"(r[32 * h + 22]), "=r"(r[32 * h + 23]), "=r"(r[32 * h + 24]),
+          "=r"(r[32 * h + 25]), "=r"(r[32 * h + 26]), "=r"(r[32 * h + 27]), "=r"(r[32 * h + 28]), "=r"(r[32 * h + 29]),
+          "=r"(r[32 * h + 30]), "=r"(r[32 * h + 31])
+        : "r"(taddr + 32 * h));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]: A is read from tensor memory (row = lane, bf16 pairs along columns).
+__device__ inline void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ inline void cp_async_16_tc(uint32_t smem_dst, const void* gmem_src, int src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_dst), "l"(gmem_src), "r"(src_bytes));
 }
@@ -171,7 +227,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   uint8_t* sQ = base + TC_SMALL_BYTES;
   uint8_t* sK = sQ + TC_BM * D * 2;
   uint8_t* sV = sK + 2 * TILE_BYTES;
-  uint8_t* sP = sV + 2 * TILE_BYTES;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   cg::cluster_group cluster = cg::this_cluster();
@@ -203,7 +258,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   if (tid == 0) {
     *s_abort = 0;
     const int n = TC_SOFTMAX_THREADS;
-    const int counts[TC_NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, n, n, n, 1, n, 1, 1, q_tma ? 1 : n};
+    const int counts[TC_NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, n, n, n, 1, 1, 1, q_tma ? 1 : n, 1};
     for (int i = 0; i < TC_NUM_BARS; ++i) mbar_init(&s_bar[i], counts[i]);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -215,7 +270,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  const uint32_t tmem_pv = tmem + 2 * TC_BN;  // S buffers at columns [0,128) and [128,256), PV after them
+  // TMEM columns: S buffers [0,128) and [128,256), O [256,256+D), P buffers (packed bf16) [384,448), [448,512)
+  const uint32_t tmem_o = tmem + 2 * TC_BN;
+  const uint32_t tmem_p = tmem + 3 * TC_BN;
 
   // One TMA box per page piece of a block: box_rows keys x 64 columns, per 64-column half.
   auto issue_block = [&](int j, const CUtensorMap* map, uint32_t stage_addr, uint64_t* bar) {
@@ -263,10 +320,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
 
   // Row state of the softmax threads: row = TMEM lane, `half` selects the 64 columns of every block
   // and the half of the output row this thread owns.
+  constexpr float kRescaleStep = 8.f;  // m_ref follows the row maximum in steps of at least 2^8
   float o_row[DH];
-  float m_run = -INFINITY, l_run = 0.f;
-#pragma unroll
-  for (int d = 0; d < DH; ++d) o_row[d] = 0.f;
+  float m_ref = -INFINITY, l_run = 0.f;
   const int half = (warp >> 2) & 1;
   const int row = (warp & 3) * 32 + lane;
 
@@ -297,7 +353,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       for (int w = 0; w < 4; ++w) anc[w] = row_live ? s_anc[4 * node + w] : 0u;
     }
     const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
-    float corr_prev = 1.f;  // rescale of o_row that belongs to the PV block still in flight
     bool ok = true;
     // The trip count and the named barrier inside are uniform over the 256 threads: after a failed
     // wait the remaining waits return at once (abort flag) and the loop just runs out.
@@ -307,86 +362,79 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       const int my_cols = nj - 64 * half;                 // valid columns among this thread's 64
       if (ok) ok = mbar_wait(&s_bar[S_FULL0 + (j & 1)], (j >> 1) & 1, s_abort);
       tc_fence_after();
-      const uint32_t t_s = tmem + lane_base + (j & 1) * TC_BN + 64 * half;
+      uint32_t sr[64];
+      tmem_ld64(tmem + lane_base + (j & 1) * TC_BN + 64 * half, sr);
+      tc_fence_before();
+      mbar_arrive(&s_bar[S_EMPTY0 + (j & 1)]);  // S is in registers: the buffer may be refilled
       // visibility of this thread's 64 columns: tree mask where the block reaches past the prefix,
       // and only the block's own nj columns
       uint64_t win = k0 + TC_BN > si.P ? visibility_window(anc, k0 + 64 * half - si.P) : ~0ull;
       win &= my_cols >= 64 ? ~0ull : (my_cols <= 0 ? 0ull : ((1ull << my_cols) - 1ull));
-      // pass 1: row maximum over both halves
       float mx = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        if (c * 32 < my_cols) {
-          uint32_t r[32];
-          tmem_ld32(t_s + c * 32, r);
-          const uint32_t m32 = (uint32_t)(win >> (c * 32));
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, ((m32 >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
-        }
+      for (int i = 0; i < 64; ++i) {
+        const float sv = ((win >> i) & 1ull) ? __uint_as_float(sr[i]) * p.scale_log2 : -INFINITY;
+        sr[i] = __float_as_uint(sv);
+        mx = fmaxf(mx, sv);
       }
       s_xmax[((j & 1) * 2 + half) * TC_BM + row] = mx;
       softmax_group_sync();
       mx = fmaxf(mx, s_xmax[((j & 1) * 2 + (half ^ 1)) * TC_BM + row]);
-      mx *= p.scale_log2;  // scale > 0: max commutes with it (-inf stays -inf)
-      const float m_new = fmaxf(m_run, mx);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      const float corr = fast_exp2(m_run - m_use);
-      // fold the previous block's PV into the output half-row (also frees P and the PV accumulator)
-      if (j > 0) {
+      // lazy reference maximum: both threads of a row take the same decision
+      const bool step = mx > m_ref + kRescaleStep || (m_ref == -INFINITY && mx > -INFINITY);
+      bool pv_waited = false;
+      if (__any_sync(0xffffffffu, step)) {
+        const float factor = (step && m_ref != -INFINITY) ? fast_exp2(m_ref - mx) : 1.f;
+        if (j > 0) {  // O holds blocks 0..j-1: rescale this thread's half-row in tensor memory
+          if (ok) ok = mbar_wait(&s_bar[PV_FULL], (j - 1) & 1, s_abort);
+          pv_waited = true;
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < DH / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(tmem_o + lane_base + half * DH + c * 32, r);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
+            tmem_st32(tmem_o + lane_base + half * DH + c * 32, r);
+          }
+          tmem_wait_st();
+        }
+        l_run *= factor;
+        if (step) m_ref = mx;
+      }
+      const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+      // probabilities -> packed bf16 pairs, written to the block's P buffer in tensor memory
+      float lsum = 0.f;
+      uint32_t packed[32];
+#pragma unroll
+      for (int i = 0; i < 64; i += 2) {
+        const float p0 = fast_exp2(__uint_as_float(sr[i]) - m_use), p1 = fast_exp2(__uint_as_float(sr[i + 1]) - m_use);
+        lsum += p0 + p1;
+        packed[i >> 1] = pack_bf16(p0, p1);
+      }
+      l_run += lsum;
+      // Every PV phase is waited for, in order (a parity wait must never lag a whole phase), and
+      // late: PV_{j-1} done also means PV_{j-2} has consumed the P buffer about to be overwritten.
+      if (j > 0 && !pv_waited) {
         if (ok) ok = mbar_wait(&s_bar[PV_FULL], (j - 1) & 1, s_abort);
         tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < DH / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tmem_pv + lane_base + half * DH + c * 32, r);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o_row[c * 32 + i] = o_row[c * 32 + i] * corr_prev + __uint_as_float(r[i]);
-        }
-        tc_fence_before();
-        mbar_arrive(&s_bar[PV_EMPTY]);
       }
-      // pass 2: probabilities -> P (bf16, K-major swizzled), running sum
-      float lsum = 0.f;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        if (c * 32 < my_cols) {
-          uint32_t r[32];
-          tmem_ld32(t_s + c * 32, r);
-          const uint32_t m32 = (uint32_t)(win >> (c * 32));
-          uint32_t packed[16];
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const float s0 = ((m32 >> i) & 1u) ? __uint_as_float(r[i]) * p.scale_log2 - m_use : -INFINITY;
-            const float s1 = ((m32 >> (i + 1)) & 1u) ? __uint_as_float(r[i + 1]) * p.scale_log2 - m_use : -INFINITY;
-            const float p0 = fast_exp2(s0), p1 = fast_exp2(s1);
-            lsum += p0 + p1;
-            packed[i >> 1] = pack_bf16(p0, p1);
-          }
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int ch = half * 8 + c * 4 + q;  // 16-byte chunk (8 keys) of this row
-            *reinterpret_cast<uint4*>(sP + sw128_chunk_off(row, ch, TC_BM)) =
-                make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-          }
-        }
-      }
-      l_run = l_run * corr + lsum;
-      m_run = m_new;
-      corr_prev = corr;
+      tmem_st32(tmem_p + lane_base + (j & 1) * 64 + half * 32, packed);
+      tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&s_bar[S_EMPTY0 + (j & 1)]);
-      fence_async_smem();
       mbar_arrive(&s_bar[P_FULL]);
     }
+#pragma unroll
+    for (int d = 0; d < DH; ++d) o_row[d] = 0.f;
     if (nb > 0) {
       if (ok) ok = mbar_wait(&s_bar[PV_FULL], (nb - 1) & 1, s_abort);
       tc_fence_after();
 #pragma unroll
       for (int c = 0; c < DH / 32; ++c) {
         uint32_t r[32];
-        tmem_ld32(tmem_pv + lane_base + half * DH + c * 32, r);
+        tmem_ld32(tmem_o + lane_base + half * DH + c * 32, r);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) o_row[c * 32 + i] = o_row[c * 32 + i] * corr_prev + __uint_as_float(r[i]);
+        for (int i = 0; i < 32; ++i) o_row[c * 32 + i] = __uint_as_float(r[i]);
       }
     }
     s_xl[half * TC_BM + row] = l_run;
@@ -394,7 +442,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   } else if (warp == TC_MMA_WARP) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && nb > 0) {
-      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV), p_addr = smem_u32(sP);
+      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
       bool ok = true;
       auto issue_s = [&](int j) {
         const int nj = min(TC_BN, chunk_keys - j * TC_BN);
@@ -426,17 +474,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
         }
         ok = mbar_wait(&s_bar[P_FULL], j & 1, s_abort);
         if (ok) ok = mbar_wait(&s_bar[V_FULL0 + (j & 1)], (j >> 1) & 1, s_abort);
-        if (ok && j > 0) ok = mbar_wait(&s_bar[PV_EMPTY], (j - 1) & 1, s_abort);
         if (!ok) break;
         tc_fence_after();
         const int nj = min(TC_BN, chunk_keys - j * TC_BN);
         const uint32_t idesc = tc_idesc(TC_BM, D, 1);
         const uint32_t vb = v_addr + (j & 1) * TILE_BYTES;
-        for (int ks = 0; ks < nj / 16; ++ks) {
-          const uint32_t aoff = (ks >> 2) * (TC_BM * 128) + (ks & 3) * 32;
-          tc_mma(tmem_pv, tc_smem_desc(p_addr + aoff, 16, 1024), tc_smem_desc(vb + ks * 2048, TC_BN * 128, 1024), idesc,
-                 ks > 0);
-        }
+        for (int ks = 0; ks < nj / 16; ++ks)  // 16 keys = 8 packed columns of P per step
+          tc_mma_ts(tmem_o, tmem_p + (j & 1) * 64 + ks * 8, tc_smem_desc(vb + ks * 2048, TC_BN * 128, 1024), idesc,
+                    (j > 0 || ks > 0) ? 1u : 0u);
         tc_commit(&s_bar[PV_FULL]);
         tc_commit(&s_bar[V_EMPTY0 + (j & 1)]);
       }
@@ -482,29 +527,102 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     if (!ok && lane == 0) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
   }
 
-  // ---- push (O, m, l) of this chunk to the owning CTAs of the cluster, reduce, store -------------
-  MergeBuf<D> mb(reinterpret_cast<float*>(sK), TC_BM, S);  // the K/V stages are idle once the last PV is folded
+  // ---- merge the cluster's chunks and store -------------------------------------------------------
+  // Row r of the tile is owned by cluster CTA r / rows_per.  Every CTA stages its 128 rows
+  // [O (D floats) | m | l | pad] in its own shared memory, then sends each owner its slice with ONE
+  // bulk asynchronous shared-to-shared copy that is credited to the owner's mbarrier; the owner
+  // reduces its rows over the S sources from local shared memory and stores them.
+  constexpr int RS = D + 8;                         // floats per staged row (16-byte multiple)
+  float* stg = reinterpret_cast<float*>(sQ);        // [128][RS]: Q and the K stages are idle by now
+  float* rcv = reinterpret_cast<float*>(sV);        // [S][rows_per][RS]: the V stages + tail
+  const int rows_per = ceil_div(TC_BM, S);
+  const int my_first = crank * rows_per;
+  const int my_rows = max(0, min(TC_BM, my_first + rows_per) - my_first);
   tc_fence_before();
-  __syncthreads();  // every role is done: no async read of the stages is in flight any more
-  if (S > 1) cluster.sync();  // ... in any CTA of the cluster: their stages are about to be written remotely
-  if (tid < TC_SOFTMAX_THREADS) {
-    const bool have = nb > 0 && sp.compute;
-    if (have) {
-      int slot;
-      float* dst = merge_row_dst<D>(cluster, mb, crank, row, &slot) + half * DH;
-#pragma unroll
-      for (int d = 0; d < DH; d += 4)
-        *reinterpret_cast<float4*>(dst + d) = make_float4(o_row[d], o_row[d + 1], o_row[d + 2], o_row[d + 3]);
-    }
-    if (half == 0)
-      merge_push_ml<D>(cluster, mb, crank, row, have ? m_run : -INFINITY, have ? s_xl[row] + s_xl[TC_BM + row] : 0.f);
-  }
-  if (S > 1) cluster.sync(); else __syncthreads();
+  __syncthreads();  // every role is done: no async access to Q/K/V stages is in flight any more
   if (warp == TC_MMA_WARP) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS));
   }
-  merge_reduce_and_store<D, TC_BM>(p, mb, S, crank, split / S, row0, rows_total, g, si.q_off, rows_all, tid, TC_THREADS);
+  if (tid < TC_SOFTMAX_THREADS) {
+    const bool have = nb > 0 && sp.compute;
+    float* dst = stg + row * RS;
+    if (have) {
+#pragma unroll
+      for (int d = 0; d < DH; d += 4)
+        *reinterpret_cast<float4*>(dst + half * DH + d) = make_float4(o_row[d], o_row[d + 1], o_row[d + 2], o_row[d + 3]);
+    }
+    if (half == 0) {
+      dst[D] = have ? m_ref : -INFINITY;
+      dst[D + 1] = have ? s_xl[row] + s_xl[TC_BM + row] : 0.f;
+    }
+  }
+  if (S > 1) {
+    if (tid == 0) mbar_expect_tx(&s_bar[MERGE_BAR], (uint32_t)(S * my_rows * RS * 4));
+    fence_async_smem();  // the staged rows are read by the bulk-copy engine
+    cluster.sync();      // all peers are done with their V stages and have armed their barriers
+    if (tid < S) {       // thread c sends owner c its slice
+      const int c = tid;
+      const int first = c * rows_per;
+      const int n = max(0, min(TC_BM, first + rows_per) - first);
+      if (n > 0)
+        dsmem_bulk_copy(mapa_u32(smem_u32(rcv + (size_t)crank * rows_per * RS), c), smem_u32(stg + (size_t)first * RS),
+                        (uint32_t)(n * RS * 4), mapa_u32(smem_u32(&s_bar[MERGE_BAR]), c));
+    }
+    if (!mbar_wait(&s_bar[MERGE_BAR], 0, s_abort) && tid == 0) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
+  } else {
+    __syncthreads();
+  }
+  {
+    const float* src = S > 1 ? rcv : stg;  // [source][row in my slice][RS]
+    const int Hq_ = Hq;
+    for (int idx = tid; idx < my_rows * (D / 4); idx += TC_THREADS) {
+      const int t = idx / (D / 4), c4 = idx % (D / 4);
+      const int Rr = row0 + my_first + t;
+      if (Rr >= rows_total) continue;
+      // weights of the S sources for this row (recomputed per thread: broadcast loads, no barrier)
+      float mc[8], lc[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        mc[c] = c < S ? src[((size_t)c * rows_per + t) * RS + D] : -INFINITY;
+        lc[c] = c < S ? src[((size_t)c * rows_per + t) * RS + D + 1] : 0.f;
+      }
+      float M = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) M = fmaxf(M, mc[c]);
+      float w[8], Lsum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        w[c] = mc[c] == -INFINITY ? 0.f : fast_exp2(mc[c] - M);
+        Lsum += w[c] * lc[c];
+      }
+      const float inv = Lsum > 0.f ? __fdividef(1.f, Lsum) : 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (w[c] != 0.f) {  // a source that saw no key for this row left its O unwritten
+          const float4 v = *reinterpret_cast<const float4*>(src + ((size_t)c * rows_per + t) * RS + c4 * 4);
+          acc.x += w[c] * v.x; acc.y += w[c] * v.y; acc.z += w[c] * v.z; acc.w += w[c] * v.w;
+        }
+      }
+      acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+      const int node_l = Rr / G, hh = Rr - node_l * G;
+      const long long grow = (long long)(si.q_off + node_l) * Hq_ + g * G + hh;
+      const float lse2 = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
+      if (p.outer == 1) {
+        uint2 packed;
+        packed.x = pack_bf16(acc.x, acc.y);
+        packed.y = pack_bf16(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(p.out + grow * D + c4 * 4) = packed;
+        if (p.lse && c4 == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
+      } else {
+        const int outer_idx = split / S;
+        *reinterpret_cast<float4*>(p.part_o + (outer_idx * rows_all + grow) * D + c4 * 4) = acc;
+        if (c4 == 0) p.part_lse[outer_idx * rows_all + grow] = lse2;
+      }
+    }
+  }
+  if (S > 1) cluster.sync();  // nobody leaves while a peer's copy may still be reading its staged rows
 }
 
 // ---------------------------------------------------------------------------------------------------
