@@ -532,7 +532,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   // [O (D floats) | m | l | pad] in its own shared memory, then sends each owner its slice with ONE
   // bulk asynchronous shared-to-shared copy that is credited to the owner's mbarrier; the owner
   // reduces its rows over the S sources from local shared memory and stores them.
-  constexpr int RS = D + 8;                         // floats per staged row (16-byte multiple)
+  constexpr int RS = D + 4;                         // floats per staged row: 16-byte multiple, conflict-free
   float* stg = reinterpret_cast<float*>(sQ);        // [128][RS]: Q and the K stages are idle by now
   float* rcv = reinterpret_cast<float*>(sV);        // [S][rows_per][RS]: the V stages + tail
   const int rows_per = ceil_div(TC_BM, S);
@@ -574,51 +574,49 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     __syncthreads();
   }
   {
+    // One warp per row: lane c < S fetches source c's (m, l) and the weights are formed with warp
+    // shuffles; then every lane combines one float4 column group of the row (D/4 <= 32 groups).
     const float* src = S > 1 ? rcv : stg;  // [source][row in my slice][RS]
-    const int Hq_ = Hq;
-    for (int idx = tid; idx < my_rows * (D / 4); idx += TC_THREADS) {
-      const int t = idx / (D / 4), c4 = idx % (D / 4);
+    for (int t = warp; t < my_rows; t += TC_THREADS / 32) {
       const int Rr = row0 + my_first + t;
-      if (Rr >= rows_total) continue;
-      // weights of the S sources for this row (recomputed per thread: broadcast loads, no barrier)
-      float mc[8], lc[8];
+      if (Rr >= rows_total) continue;  // uniform over the warp
+      const float mc = lane < S ? src[((size_t)lane * rows_per + t) * RS + D] : -INFINITY;
+      const float lc = lane < S ? src[((size_t)lane * rows_per + t) * RS + D + 1] : 0.f;
+      float M = mc;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        mc[c] = c < S ? src[((size_t)c * rows_per + t) * RS + D] : -INFINITY;
-        lc[c] = c < S ? src[((size_t)c * rows_per + t) * RS + D + 1] : 0.f;
-      }
-      float M = -INFINITY;
+      for (int sft = 4; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sft));  // S <= 8 lanes
+      const float wl = mc == -INFINITY ? 0.f : fast_exp2(mc - M);
+      float Lsum = wl * lc;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) M = fmaxf(M, mc[c]);
-      float w[8], Lsum = 0.f;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        w[c] = mc[c] == -INFINITY ? 0.f : fast_exp2(mc[c] - M);
-        Lsum += w[c] * lc[c];
-      }
+      for (int sft = 4; sft > 0; sft >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, sft);
+      M = __shfl_sync(0xffffffffu, M, 0);
+      Lsum = __shfl_sync(0xffffffffu, Lsum, 0);
       const float inv = Lsum > 0.f ? __fdividef(1.f, Lsum) : 0.f;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        if (w[c] != 0.f) {  // a source that saw no key for this row left its O unwritten
-          const float4 v = *reinterpret_cast<const float4*>(src + ((size_t)c * rows_per + t) * RS + c4 * 4);
-          acc.x += w[c] * v.x; acc.y += w[c] * v.y; acc.z += w[c] * v.z; acc.w += w[c] * v.w;
+#pragma unroll 1
+      for (int c = 0; c < S; ++c) {
+        const float w = __shfl_sync(0xffffffffu, wl, c);
+        if (w != 0.f && lane < D / 4) {  // a source that saw no key for this row left its O unwritten
+          const float4 v = *reinterpret_cast<const float4*>(src + ((size_t)c * rows_per + t) * RS + lane * 4);
+          acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
         }
       }
       acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
       const int node_l = Rr / G, hh = Rr - node_l * G;
-      const long long grow = (long long)(si.q_off + node_l) * Hq_ + g * G + hh;
+      const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
       const float lse2 = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
-      if (p.outer == 1) {
-        uint2 packed;
-        packed.x = pack_bf16(acc.x, acc.y);
-        packed.y = pack_bf16(acc.z, acc.w);
-        *reinterpret_cast<uint2*>(p.out + grow * D + c4 * 4) = packed;
-        if (p.lse && c4 == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
-      } else {
-        const int outer_idx = split / S;
-        *reinterpret_cast<float4*>(p.part_o + (outer_idx * rows_all + grow) * D + c4 * 4) = acc;
-        if (c4 == 0) p.part_lse[outer_idx * rows_all + grow] = lse2;
+      if (lane < D / 4) {
+        if (p.outer == 1) {
+          uint2 packed;
+          packed.x = pack_bf16(acc.x, acc.y);
+          packed.y = pack_bf16(acc.z, acc.w);
+          *reinterpret_cast<uint2*>(p.out + grow * D + lane * 4) = packed;
+          if (p.lse && lane == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
+        } else {
+          const int outer_idx = split / S;
+          *reinterpret_cast<float4*>(p.part_o + (outer_idx * rows_all + grow) * D + lane * 4) = acc;
+          if (lane == 0) p.part_lse[outer_idx * rows_all + grow] = lse2;
+        }
       }
     }
   }
