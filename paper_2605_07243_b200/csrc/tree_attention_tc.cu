@@ -44,16 +44,16 @@ constexpr int TC_VLOAD_WARP = 10;    // lane 0 issues the V loads; the warp zero
 constexpr int TC_THREADS = 384;      // 12 warps (warp 11 only takes part in the barriers)
 constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_SMALL_BYTES = 8192; // ancestor masks, parents, barriers, softmax exchange
-constexpr int TC_MERGE_TAIL = 8192;  // the merge receive buffer = the V stages + this tail
+constexpr int TC_MERGE_SLOTS = TC_BM + 8;  // receive slots: S * ceil(128 / S) <= 135 for S <= 8
 
 enum TcBar { K_FULL0, K_FULL1, K_EMPTY0, K_EMPTY1, V_FULL0, V_FULL1, V_EMPTY0, V_EMPTY1, S_FULL0, S_FULL1,
-             S_EMPTY0, S_EMPTY1, P_FULL, PV_FULL, V_TMA0, V_TMA1, Q_FULL, MERGE_BAR, TC_NUM_BARS };
+             S_EMPTY0, S_EMPTY1, P_FULL, PV_FULL, V_TMA0, V_TMA1, Q_FULL, MERGE_BAR, ACK_BAR, TC_NUM_BARS };
 
 template <int D>
 constexpr size_t attn_tc_smem_bytes() {
-  // small region + Q + 2 K stages + 2 V stages + tail of the merge receive buffer, plus slack to
-  // align the tiles to 1024 bytes
-  return 1024 + TC_SMALL_BYTES + (size_t)TC_BM * D * 2 + 4 * (size_t)TC_BN * D * 2 + TC_MERGE_TAIL;
+  // small region + Q + 2 K stages + 2 V stages + the merge receive buffer (bf16 rows + m, l), plus
+  // slack to align the tiles to 1024 bytes
+  return 1024 + TC_SMALL_BYTES + (size_t)TC_BM * D * 2 + 4 * (size_t)TC_BN * D * 2 + (size_t)TC_MERGE_SLOTS * (D * 2 + 16);
 }
 
 __device__ inline uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -158,6 +158,10 @@ __device__ inline void dsmem_bulk_copy(uint32_t dst_cluster_addr, uint32_t src_c
                "r"(src_cta_addr), "r"(bytes), "r"(mbar_cluster_addr)
                : "memory");
 }
+// Arrive on an mbarrier that lives in a cluster peer's shared memory.
+__device__ inline void mbar_arrive_remote(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
 __device__ inline void softmax_group_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 // 32 consecutive 32-bit columns of this thread's TMEM lane <- registers.
 __device__ inline void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -227,6 +231,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   uint8_t* sQ = base + TC_SMALL_BYTES;
   uint8_t* sK = sQ + TC_BM * D * 2;
   uint8_t* sV = sK + 2 * TILE_BYTES;
+  uint8_t* sRcv = sV + 2 * TILE_BYTES;  // merge receive buffer: written by cluster peers only
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   cg::cluster_group cluster = cg::this_cluster();
@@ -236,12 +241,44 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const int Hkv = p.tb.n_kv_heads, Hq = p.tb.n_q_heads, G = p.G;
   const int g = blockIdx.y % Hkv, tile = blockIdx.y / Hkv;
   const int b = blockIdx.z;
+  if (tid == 0) {
+    *s_abort = 0;
+    const int n = TC_SOFTMAX_THREADS;
+    const int counts[TC_NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, n, n, n, 1, 1, 1, q_tma ? 1 : n, 1, S};
+    for (int i = 0; i < TC_NUM_BARS; ++i) mbar_init(&s_bar[i], counts[i]);
+    // the merge barrier is armed at once: cluster peers may deliver their rows at any time
+    if (S > 1) {
+      const int rp = ceil_div(TC_BM, S);
+      const int mine = max(0, min(TC_BM, (crank + 1) * rp) - crank * rp);
+      mbar_expect_tx(&s_bar[MERGE_BAR], (uint32_t)(S * mine * (D * 2 + 16)));
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == TC_MMA_WARP) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TC_TMEM_COLS));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  // Non-blocking half of a cluster barrier: "my barriers are initialised".  The matching wait sits
+  // just before this CTA first touches a peer's barrier, microseconds later.
+  if (S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  // Programmatic dependent launch: everything above is independent of earlier kernels' results and
+  // may overlap their tail; from here on their memory is complete and visible.  Dependents of this
+  // kernel are released right away, so at most two consecutive grids are ever in flight.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   const SeqPre pre = plan_lengths(p, b);
   const int rows_total = pre.info.nq * G;
   const int row0 = tile * TC_BM;
   if (!pre.can_write || row0 >= rows_total) {  // uniform over the cluster
     // the designated CTA always owns rows unless the sequence has none; its status is still due
     if (split == 0 && blockIdx.y == 0 && tid == 0) p.status[b] = pre.info.err;
+    if (warp == TC_MMA_WARP)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*s_tmem), "r"(TC_TMEM_COLS));
+    if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // pairs with the arrive above
     return;
   }
   const long long rows_all = (long long)p.total_q * Hq;
@@ -255,20 +292,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const int nb = pre.info.err == 0 ? b_base + (split < b_rem ? 1 : 0) : 0;
   const int chunk_keys = nb == 0 ? 0 : min(nb * TC_BN, ceil_div(L - key_begin, 16) * 16);
 
-  if (tid == 0) {
-    *s_abort = 0;
-    const int n = TC_SOFTMAX_THREADS;
-    const int counts[TC_NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, n, n, n, 1, 1, 1, q_tma ? 1 : n, 1};
-    for (int i = 0; i < TC_NUM_BARS; ++i) mbar_init(&s_bar[i], counts[i]);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == TC_MMA_WARP) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TC_TMEM_COLS));
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
   const uint32_t tmem = *s_tmem;
   // TMEM columns: S buffers [0,128) and [128,256), O [256,256+D), P buffers (packed bf16) [384,448), [448,512)
   const uint32_t tmem_o = tmem + 2 * TC_BN;
@@ -528,13 +551,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   }
 
   // ---- merge the cluster's chunks and store -------------------------------------------------------
-  // Row r of the tile is owned by cluster CTA r / rows_per.  Every CTA stages its 128 rows
-  // [O (D floats) | m | l | pad] in its own shared memory, then sends each owner its slice with ONE
-  // bulk asynchronous shared-to-shared copy that is credited to the owner's mbarrier; the owner
-  // reduces its rows over the S sources from local shared memory and stores them.
-  constexpr int RS = D + 4;                         // floats per staged row: 16-byte multiple, conflict-free
-  float* stg = reinterpret_cast<float*>(sQ);        // [128][RS]: Q and the K stages are idle by now
-  float* rcv = reinterpret_cast<float*>(sV);        // [S][rows_per][RS]: the V stages + tail
+  // Row r of the tile is owned by cluster CTA r / rows_per.  Every CTA stages its 128 rows as
+  // [O / l in bf16 (D) | m | l | pad] (normalised, so bf16 has the range and O(2^-9) relative error
+  // against a 1e-2 tolerance), then sends each owner its slice with ONE bulk asynchronous
+  // shared-to-shared copy credited to the owner's mbarrier.  The receive buffer is written by
+  // peers only and its barrier was armed at kernel start, so nothing has to be awaited before
+  // sending.  The owner reduces its rows over the S sources and stores them; a CTA leaves once
+  // every owner has acknowledged that its slice has arrived.
+  constexpr int ROWB = D * 2 + 16;                  // bytes per staged row (16-byte multiple)
+  uint8_t* stg = sQ;                                // [128][ROWB]: Q and the K stages are idle by now
   const int rows_per = ceil_div(TC_BM, S);
   const int my_first = crank * rows_per;
   const int my_rows = max(0, min(TC_BM, my_first + rows_per) - my_first);
@@ -546,47 +571,58 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   }
   if (tid < TC_SOFTMAX_THREADS) {
     const bool have = nb > 0 && sp.compute;
-    float* dst = stg + row * RS;
-    if (have) {
+    softmax_group_sync();  // both halves' running sums are in s_xl
+    const float l_tot = s_xl[row] + s_xl[TC_BM + row];
+    const float inv_l = (have && l_tot > 0.f) ? __fdividef(1.f, l_tot) : 0.f;
+    uint8_t* dst = stg + row * ROWB;
 #pragma unroll
-      for (int d = 0; d < DH; d += 4)
-        *reinterpret_cast<float4*>(dst + half * DH + d) = make_float4(o_row[d], o_row[d + 1], o_row[d + 2], o_row[d + 3]);
+    for (int d = 0; d < DH; d += 8) {
+      uint4 v;
+      v.x = pack_bf16(o_row[d] * inv_l, o_row[d + 1] * inv_l);
+      v.y = pack_bf16(o_row[d + 2] * inv_l, o_row[d + 3] * inv_l);
+      v.z = pack_bf16(o_row[d + 4] * inv_l, o_row[d + 5] * inv_l);
+      v.w = pack_bf16(o_row[d + 6] * inv_l, o_row[d + 7] * inv_l);
+      *reinterpret_cast<uint4*>(dst + (half * DH + d) * 2) = v;
     }
     if (half == 0) {
-      dst[D] = have ? m_ref : -INFINITY;
-      dst[D + 1] = have ? s_xl[row] + s_xl[TC_BM + row] : 0.f;
+      *reinterpret_cast<float*>(dst + D * 2) = (have && l_tot > 0.f) ? m_ref : -INFINITY;
+      *reinterpret_cast<float*>(dst + D * 2 + 4) = (have && l_tot > 0.f) ? l_tot : 0.f;
     }
   }
+  bool merge_ok = true;
   if (S > 1) {
-    if (tid == 0) mbar_expect_tx(&s_bar[MERGE_BAR], (uint32_t)(S * my_rows * RS * 4));
     fence_async_smem();  // the staged rows are read by the bulk-copy engine
-    cluster.sync();      // all peers are done with their V stages and have armed their barriers
+    __syncthreads();
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // every peer's barriers exist (long since)
     if (tid < S) {       // thread c sends owner c its slice
       const int c = tid;
       const int first = c * rows_per;
       const int n = max(0, min(TC_BM, first + rows_per) - first);
       if (n > 0)
-        dsmem_bulk_copy(mapa_u32(smem_u32(rcv + (size_t)crank * rows_per * RS), c), smem_u32(stg + (size_t)first * RS),
-                        (uint32_t)(n * RS * 4), mapa_u32(smem_u32(&s_bar[MERGE_BAR]), c));
+        dsmem_bulk_copy(mapa_u32(smem_u32(sRcv + (size_t)crank * rows_per * ROWB), c), smem_u32(stg + (size_t)first * ROWB),
+                        (uint32_t)(n * ROWB), mapa_u32(smem_u32(&s_bar[MERGE_BAR]), c));
     }
-    if (!mbar_wait(&s_bar[MERGE_BAR], 0, s_abort) && tid == 0) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
+    merge_ok = mbar_wait(&s_bar[MERGE_BAR], 0, s_abort);
+    // every source's slice has landed here: tell each source that its staging rows are free
+    if (tid < S) mbar_arrive_remote(mapa_u32(smem_u32(&s_bar[ACK_BAR]), tid));
   } else {
     __syncthreads();
   }
   {
-    // One warp per row: lane c < S fetches source c's (m, l) and the weights are formed with warp
-    // shuffles; then every lane combines one float4 column group of the row (D/4 <= 32 groups).
-    const float* src = S > 1 ? rcv : stg;  // [source][row in my slice][RS]
+    // One warp per row: lane c < S fetches source c's (m, l), the weights are formed with warp
+    // shuffles, then every lane combines four columns of the row (D/4 <= 32 lanes).
+    const uint8_t* src = S > 1 ? sRcv : stg;  // [source][row in my slice][ROWB]
     for (int t = warp; t < my_rows; t += TC_THREADS / 32) {
       const int Rr = row0 + my_first + t;
       if (Rr >= rows_total) continue;  // uniform over the warp
-      const float mc = lane < S ? src[((size_t)lane * rows_per + t) * RS + D] : -INFINITY;
-      const float lc = lane < S ? src[((size_t)lane * rows_per + t) * RS + D + 1] : 0.f;
+      const uint8_t* mine = src + ((size_t)(lane < S ? lane : 0) * rows_per + t) * ROWB;
+      const float mc = lane < S ? *reinterpret_cast<const float*>(mine + D * 2) : -INFINITY;
+      const float lc = lane < S ? *reinterpret_cast<const float*>(mine + D * 2 + 4) : 0.f;
       float M = mc;
 #pragma unroll
       for (int sft = 4; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sft));  // S <= 8 lanes
-      const float wl = mc == -INFINITY ? 0.f : fast_exp2(mc - M);
-      float Lsum = wl * lc;
+      const float wl = mc == -INFINITY ? 0.f : fast_exp2(mc - M) * lc;  // weight of source `lane`: 2^(m-M) * l
+      float Lsum = wl;
 #pragma unroll
       for (int sft = 4; sft > 0; sft >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, sft);
       M = __shfl_sync(0xffffffffu, M, 0);
@@ -596,9 +632,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
 #pragma unroll 1
       for (int c = 0; c < S; ++c) {
         const float w = __shfl_sync(0xffffffffu, wl, c);
-        if (w != 0.f && lane < D / 4) {  // a source that saw no key for this row left its O unwritten
-          const float4 v = *reinterpret_cast<const float4*>(src + ((size_t)c * rows_per + t) * RS + lane * 4);
-          acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        if (w != 0.f && lane < D / 4) {
+          const uint2 raw = *reinterpret_cast<const uint2*>(src + ((size_t)c * rows_per + t) * ROWB + lane * 8);
+          acc.x += w * __uint_as_float(raw.x << 16);
+          acc.y += w * __uint_as_float(raw.x & 0xffff0000u);
+          acc.z += w * __uint_as_float(raw.y << 16);
+          acc.w += w * __uint_as_float(raw.y & 0xffff0000u);
         }
       }
       acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
@@ -620,7 +659,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       }
     }
   }
-  if (S > 1) cluster.sync();  // nobody leaves while a peer's copy may still be reading its staged rows
+  if (S > 1) {
+    // do not leave while a peer's copy may still be reading the staged rows
+    if (merge_ok) merge_ok = mbar_wait(&s_bar[ACK_BAR], 0, s_abort);
+    if (!merge_ok && tid == 0) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -690,8 +733,11 @@ static cudaLaunchConfig_t tc_config(dim3 grid, int cluster, cudaStream_t cs, cud
   attr[0].val.clusterDim.x = cluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // the kernel orders itself after its predecessor with griddepcontrol.wait
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = getenv("SB_NO_PDL") ? 1 : 2;
   return cfg;
 }
 
@@ -716,7 +762,7 @@ int attn_tc_max_active_clusters(int D, int cluster) {
   if (cluster < 1 || cluster > 8) return 0;
   if (!have[di][cluster]) {
     int n = 0;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     cudaError_t e = cudaErrorUnknown;
     if (D == 64 && tc_prepare<64>()) {
       cudaLaunchConfig_t cfg = tc_config<64>(dim3(cluster * 64, 1, 1), cluster, nullptr, attr);
@@ -735,7 +781,7 @@ int attn_tc_max_active_clusters(int D, int cluster) {
 template <int D>
 static sb_status launch_tc(const AttnParams& p, dim3 grid, int cluster, cudaStream_t cs) {
   if (!tc_prepare<D>()) return SB_ERR_CUDA;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   cudaLaunchConfig_t cfg = tc_config<D>(grid, cluster, cs, attr);
   if (getenv("SB_DEBUG"))
     fprintf(stderr, "[sb] attn_tc<%d> grid (%u,%u,%u) cluster %d outer %d: max active clusters %d\n", D, grid.x, grid.y,
