@@ -321,23 +321,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
         tma_load_4d(stage_addr + h * (TC_BN * 128) + i * box_rows * 128, map, h * 64, g, c2, c3, bar);
     }
   };
-  // The first loads go out before anything else: they only need the sequence's lengths.
-  if (nb > 0 && lane == 0) {
-    if (warp == TC_KLOAD_WARP) {
-      if (q_tma) {
-        mbar_expect_tx(&s_bar[Q_FULL], (uint32_t)(TC_BM * D * 2));
+  // The first loads go out before anything else: they only need the sequence's lengths.  Only
+  // what the first S product needs (Q and K block 0) is requested at once; the other first-wave
+  // tiles follow when K block 0 has landed, so they do not queue in front of it in the memory system.
+  if (nb > 0 && lane == 0 && warp == TC_KLOAD_WARP) {
+    if (q_tma) {
+      mbar_expect_tx(&s_bar[Q_FULL], (uint32_t)(TC_BM * D * 2));
 #pragma unroll
-        for (int h = 0; h < D / 64; ++h)
-          tma_load_3d(smem_u32(sQ) + h * (TC_BM * 128), &qmap, h * 64, g * G, pre.info.q_off + tile * (TC_BM / G),
-                      &s_bar[Q_FULL]);
-      }
-      issue_block(0, &kmap, smem_u32(sK), &s_bar[K_FULL0]);
-      if (nb > 1) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
-    } else if (warp == TC_VLOAD_WARP) {
-      issue_block(0, &vmap, smem_u32(sV), &s_bar[V_TMA0]);
-      if (nb > 1) issue_block(1, &vmap, smem_u32(sV) + TILE_BYTES, &s_bar[V_TMA1]);
+      for (int h = 0; h < D / 64; ++h)
+        tma_load_3d(smem_u32(sQ) + h * (TC_BM * 128), &qmap, h * 64, g * G, pre.info.q_off + tile * (TC_BM / G),
+                    &s_bar[Q_FULL]);
     }
+    issue_block(0, &kmap, smem_u32(sK), &s_bar[K_FULL0]);
   }
+
   const SeqPlan sp = plan_tree(p, b, split == 0 && blockIdx.y == 0, pre, s_parent, s_anc);
   const SeqInfo& si = sp.info;
 
@@ -514,6 +511,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     // ------------------------------------------------------------------ K loader (blocks 2..)
     if (lane == 0) {
       bool ok = true;
+      if (nb > 1) {
+        ok = mbar_wait(&s_bar[K_FULL0], 0, s_abort);
+        if (ok) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
+      }
       for (int j = 2; j < nb && ok; ++j) {
         ok = mbar_wait(&s_bar[K_EMPTY0 + (j & 1)], ((j >> 1) - 1) & 1, s_abort);
         if (ok) issue_block(j, &kmap, smem_u32(sK) + (j & 1) * TILE_BYTES, &s_bar[K_FULL0 + (j & 1)]);
@@ -523,6 +524,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   } else if (warp == TC_VLOAD_WARP) {
     // ------------------------------------------------------------------ V loader
     bool ok = true;
+    if (nb > 0 && lane == 0) {
+      ok = mbar_wait(&s_bar[K_FULL0], 0, s_abort);
+      if (ok) {
+        issue_block(0, &vmap, smem_u32(sV), &s_bar[V_TMA0]);
+        if (nb > 1) issue_block(1, &vmap, smem_u32(sV) + TILE_BYTES, &s_bar[V_TMA1]);
+      }
+    }
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     for (int j = 0; j < nb && ok; ++j) {
       ok = mbar_wait(&s_bar[V_TMA0 + (j & 1)], (j >> 1) & 1, s_abort);
       if (!ok) break;

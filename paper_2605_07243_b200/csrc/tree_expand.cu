@@ -8,6 +8,8 @@
 //                         elements >= tau (a handful per CTA unless values tie) enter the per-thread
 //                         sorted lists; ids ascend inside a thread, so the order (value descending, id
 //                         ascending) is kept by strict compares.  The CTA then pops its 16 best in order.
+//   topk_partial_reg_kernel: the same result with the chunk held in registers (one HBM pass, no re-read),
+//                         used whenever rows are 16-byte aligned and a chunk has at most 16384 elements.
 //   expand_finish_kernel: one CTA.  A warp per row merges the chunk lists held in registers; then the
 //                         append is done in parallel: a row is alive iff every earlier position of its
 //                         block has width >= 1, its first node id is an exclusive prefix sum of the
@@ -131,6 +133,154 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
   }
 }
 
+// Register-resident variant for 16-byte-aligned rows and chunks of at most TOPK_REG_ELEMS
+// elements: the chunk is read from HBM exactly once into registers (64 values per thread).
+// tau = the smallest of 16 group maxima (16 threads per group; 16 distinct elements reach it), so
+// the chunk's 16 best are among the elements >= tau -- a few dozen unless values tie.  They are
+// collected in shared memory and ranked all-pairs under (value descending, id ascending).  If more
+// than TOPK_CAND of them exist (massive ties) the per-thread sorted-list method takes over, fed
+// from the same registers.
+constexpr int TOPK_VEC_PER_THREAD = 16;
+constexpr int TOPK_REG_ELEMS = TOPK_THREADS * TOPK_VEC_PER_THREAD * 4;  // 16384
+constexpr int TOPK_CAND = 512;
+
+__global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const float* __restrict__ scores,
+                                                                        long long row_stride, int vocab, int chunk,
+                                                                        int n_chunks, float* __restrict__ part_val,
+                                                                        int* __restrict__ part_idx) {
+  __shared__ float s_val[SB_KMAX][TOPK_THREADS];  // fallback lists; the candidate arrays alias them
+  __shared__ int s_idx[SB_KMAX][TOPK_THREADS];
+  __shared__ float s_group[16];
+  __shared__ float s_wv[TOPK_THREADS / 32];
+  __shared__ int s_wi[TOPK_THREADS / 32], s_wt[TOPK_THREADS / 32];
+  __shared__ int s_winner, s_count;
+  float* s_cv = &s_val[0][0];
+  int* s_ci = &s_idx[0][0];
+  const int row = blockIdx.y, c = blockIdx.x, tid = threadIdx.x;
+  const float* base = scores + (long long)row * row_stride;
+  const int begin = c * chunk;
+  const int end = min(vocab, begin + chunk);
+  const int n_elems = max(0, end - begin);
+  const int n_vec = n_elems / 4;  // whole float4s; up to 3 tail elements are handled by thread 0
+  const float4* vb = reinterpret_cast<const float4*>(base + begin);
+  if (tid == 0) s_count = 0;
+
+  float4 x[TOPK_VEC_PER_THREAD];
+  float tmax = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < TOPK_VEC_PER_THREAD; ++i) {
+    const int v = tid + i * TOPK_THREADS;
+    float4 t = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (v < n_vec) {
+      t = __ldg(vb + v);
+      t.x = score_of(t.x); t.y = score_of(t.y); t.z = score_of(t.z); t.w = score_of(t.w);
+    }
+    x[i] = t;
+    tmax = fmaxf(tmax, fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w)));
+  }
+  float gmax = tmax;
+#pragma unroll
+  for (int sft = 8; sft > 0; sft >>= 1) gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, sft));
+  if ((tid & 15) == 0) s_group[tid >> 4] = gmax;
+  __syncthreads();
+  float tau = s_group[0];
+#pragma unroll
+  for (int i = 1; i < 16; ++i) tau = fminf(tau, s_group[i]);
+
+  auto push = [&](float v, int id) {
+    if (v >= tau) {
+      const int pos = atomicAdd(&s_count, 1);
+      if (pos < TOPK_CAND) { s_cv[pos] = v; s_ci[pos] = id; }
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < TOPK_VEC_PER_THREAD; ++i) {
+    const int vi = tid + i * TOPK_THREADS;
+    if (vi < n_vec) {  // padding beyond the chunk is not an element
+      const int id0 = begin + 4 * vi;
+      push(x[i].x, id0); push(x[i].y, id0 + 1); push(x[i].z, id0 + 2); push(x[i].w, id0 + 3);
+    }
+  }
+  if (tid == 0) {  // tail elements are always candidates
+    for (int id = begin + 4 * n_vec; id < end; ++id) {
+      const int pos = atomicAdd(&s_count, 1);
+      if (pos < TOPK_CAND) { s_cv[pos] = score_of(base[id]); s_ci[pos] = id; }
+    }
+  }
+  __syncthreads();
+  const int count = s_count;
+  const long long out0 = ((long long)row * n_chunks + c) * SB_KMAX;
+  if (count <= TOPK_CAND) {
+    for (int a = tid; a < count; a += TOPK_THREADS) {
+      const float v = s_cv[a];
+      const int id = s_ci[a];
+      int r = 0;
+      for (int b2 = 0; b2 < count; ++b2) r += ranks_before(s_cv[b2], s_ci[b2], v, id) ? 1 : 0;
+      if (r < SB_KMAX) { part_val[out0 + r] = v; part_idx[out0 + r] = id; }
+    }
+    if (tid < SB_KMAX && tid >= count) { part_val[out0 + tid] = -INFINITY; part_idx[out0 + tid] = kNoId; }
+    return;
+  }
+  // ---- massive ties: per-thread sorted lists (ids ascend inside a thread), then ordered pops ----
+  __syncthreads();  // the candidate arrays alias the lists
+  float v[SB_KMAX];
+  int id[SB_KMAX];
+#pragma unroll
+  for (int k = 0; k < SB_KMAX; ++k) { v[k] = -INFINITY; id[k] = kNoId; }
+  auto offer = [&](float xv, int xi) {
+    if (xv < tau) return;
+    if (!ranks_before(xv, xi, v[SB_KMAX - 1], id[SB_KMAX - 1])) return;
+    v[SB_KMAX - 1] = xv;
+    id[SB_KMAX - 1] = xi;
+#pragma unroll
+    for (int k = SB_KMAX - 1; k > 0; --k) {
+      if (ranks_before(v[k], id[k], v[k - 1], id[k - 1])) {
+        const float tv = v[k]; v[k] = v[k - 1]; v[k - 1] = tv;
+        const int ti = id[k]; id[k] = id[k - 1]; id[k - 1] = ti;
+      }
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < TOPK_VEC_PER_THREAD; ++i) {
+    const int vi = tid + i * TOPK_THREADS;
+    if (vi < n_vec) {
+      const int id0 = begin + 4 * vi;
+      offer(x[i].x, id0); offer(x[i].y, id0 + 1); offer(x[i].z, id0 + 2); offer(x[i].w, id0 + 3);
+    }
+  }
+  if (tid == 0)
+    for (int i2 = begin + 4 * n_vec; i2 < end; ++i2) offer(score_of(base[i2]), i2);
+#pragma unroll
+  for (int k = 0; k < SB_KMAX; ++k) { s_val[k][tid] = v[k]; s_idx[k][tid] = id[k]; }
+  __syncthreads();
+  int pos = 0;
+  for (int round = 0; round < SB_KMAX; ++round) {
+    float hv = pos < SB_KMAX ? s_val[pos][tid] : -INFINITY;
+    int hi = pos < SB_KMAX ? s_idx[pos][tid] : kNoId;
+    int ht = tid;
+#pragma unroll
+    for (int sft = 16; sft > 0; sft >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, hv, sft);
+      const int oi = __shfl_xor_sync(0xffffffffu, hi, sft);
+      const int ot = __shfl_xor_sync(0xffffffffu, ht, sft);
+      if (ranks_before(ov, oi, hv, hi)) { hv = ov; hi = oi; ht = ot; }
+    }
+    if ((tid & 31) == 0) { s_wv[tid >> 5] = hv; s_wi[tid >> 5] = hi; s_wt[tid >> 5] = ht; }
+    __syncthreads();
+    if (tid == 0) {
+      float bv = s_wv[0];
+      int bi = s_wi[0], bt = s_wt[0];
+      for (int w = 1; w < TOPK_THREADS / 32; ++w)
+        if (ranks_before(s_wv[w], s_wi[w], bv, bi)) { bv = s_wv[w]; bi = s_wi[w]; bt = s_wt[w]; }
+      part_val[out0 + round] = bv;
+      part_idx[out0 + round] = bi;
+      s_winner = bi == kNoId ? -1 : bt;
+    }
+    __syncthreads();
+    if (tid == s_winner) ++pos;
+  }
+}
+
 constexpr int FINISH_THREADS = 1024;
 
 __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
@@ -145,6 +295,20 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
   __shared__ int s_carry;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) s_bad = 0;
+  // Scalars of the first slab of rows are fetched now so that their latency hides under the merge.
+  const int rows_slab0 = (FINISH_THREADS / block_k) * block_k;
+  const bool pre_row = tid < rows_slab0 && tid < n_rows;
+  const int pre_start = pre_row ? start_parent[tid / block_k] : -1;
+  int pre_bucket[4] = {0, 0, 0, 0};  // buckets of this row and of up to three earlier positions of its block
+  if (pre_row) {
+    const int kp = tid % block_k;
+    pre_bucket[0] = bucket[tid];
+    if (kp >= 1) pre_bucket[1] = bucket[tid - 1];
+    if (kp >= 2) pre_bucket[2] = bucket[tid - 2];
+    if (kp >= 3) pre_bucket[3] = bucket[tid - 3];
+  }
+  const int pre_n0 = *n_nodes;
+  const int pre_depth = (pre_row && pre_start >= 0 && pre_start < pre_n0) ? depth[pre_start] : 0;
   __syncthreads();
   // (1) merge the chunk lists of every row: lane c holds chunk c's sorted list in registers and
   //     pops it by shifting
@@ -192,7 +356,7 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
     }
   }
   // (2) argument checks that need device data
-  const int n0 = *n_nodes;
+  const int n0 = pre_n0;
   if (tid == 0 && (n0 < 0 || n0 > node_budget)) s_bad = 1;
   for (int r = tid; r < n_rows; r += FINISH_THREADS)
     if (bucket[r] > 3) s_bad = 1;
@@ -215,15 +379,17 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
     int width = 0, kpos = 0, start = -1;
     if (tid < rows_per_slab && r < n_rows) {
       kpos = r % block_k;
-      start = start_parent[r / block_k];
-      auto width_of = [&](int row) {
-        const int bk = bucket[row];
+      start = slab == 0 ? pre_start : start_parent[r / block_k];
+      auto width_of_bucket = [&](int bk) {
         const int w = bk == 0 ? bmap.x : bk == 1 ? bmap.y : bk == 2 ? bmap.z : bmap.w;
         return w < vocab ? w : vocab;
       };
       bool alive = true;
-      for (int k = 1; k <= kpos; ++k) alive = alive && width_of(r - k) >= 1;
-      width = alive ? width_of(r) : 0;
+      for (int k = 1; k <= kpos; ++k) {
+        const int bk = (slab == 0 && k <= 3) ? (k == 1 ? pre_bucket[1] : k == 2 ? pre_bucket[2] : pre_bucket[3]) : bucket[r - k];
+        alive = alive && width_of_bucket(bk) >= 1;
+      }
+      width = alive ? width_of_bucket(slab == 0 ? pre_bucket[0] : bucket[r]) : 0;
     }
     // exclusive scan of the widths over the slab
     int incl = width;
@@ -250,7 +416,7 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
     __syncthreads();
     if (width > 0) {
       const int par = kpos == 0 ? start : s_first[tid - 1];  // rank-0 node of the previous position
-      const int base_depth = start == -1 ? 0 : depth[start] + 1;
+      const int base_depth = start == -1 ? 0 : (slab == 0 ? pre_depth : depth[start]) + 1;
       for (int j = 0; j < width && first + j < node_budget; ++j) {
         const int n = first + j;
         tok[n] = topk_tok[r * SB_KMAX + j];
@@ -274,6 +440,8 @@ static int topk_chunks(int n_rows, int vocab) {
   int nc = ceil_div(2 * 148, n_rows > 0 ? n_rows : 1);
   const int max_nc = ceil_div(vocab, 2048);
   if (nc > max_nc) nc = max_nc;
+  const int reg_nc = ceil_div(vocab, TOPK_REG_ELEMS);  // chunks that fit the register-resident kernel
+  if (nc < reg_nc) nc = reg_nc;
   if (nc > 32) nc = 32;
   if (nc < 1) nc = 1;
   return nc;
@@ -312,8 +480,11 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
   float* part_val = static_cast<float*>(workspace);
   int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + need / 2);
   dim3 grid(nc, n_rows);
-  topk_partial_kernel<<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
-                                                     part_idx);
+  if (vec_ok && chunk <= TOPK_REG_ELEMS)
+    topk_partial_reg_kernel<<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, part_val, part_idx);
+  else
+    topk_partial_kernel<<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
+                                                       part_idx);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
   expand_finish_kernel<<<1, FINISH_THREADS, 0, cs>>>(n_rows, nc, part_val, part_idx, block_k, bucket,
