@@ -390,13 +390,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       // and only the block's own nj columns
       uint64_t win = k0 + TC_BN > si.P ? visibility_window(anc, k0 + 64 * half - si.P) : ~0ull;
       win &= my_cols >= 64 ? ~0ull : (my_cols <= 0 ? 0ull : ((1ull << my_cols) - 1ull));
+      // row maximum of the raw scores (the softmax scale is positive: it commutes with max)
+      if (win != ~0ull) {  // only blocks that touch the tree or the end of the chunk have masked columns
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (!((win >> i) & 1ull)) sr[i] = 0xff800000u;  // -inf
+      }
       float mx = -INFINITY;
 #pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float sv = ((win >> i) & 1ull) ? __uint_as_float(sr[i]) * p.scale_log2 : -INFINITY;
-        sr[i] = __float_as_uint(sv);
-        mx = fmaxf(mx, sv);
-      }
+      for (int i = 0; i < 64; i += 2) mx = max3(mx, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+      mx *= p.scale_log2;
       s_xmax[((j & 1) * 2 + half) * TC_BM + row] = mx;
       softmax_group_sync();
       mx = fmaxf(mx, s_xmax[((j & 1) * 2 + (half ^ 1)) * TC_BM + row]);
@@ -424,14 +427,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       }
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
       // probabilities -> packed bf16 pairs, written to the block's P buffer in tensor memory
-      float lsum = 0.f;
+      // p = 2^(s * scale - m_ref): the argument and the running sum use packed two-lane arithmetic
+      const unsigned long long scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      const unsigned long long negm2 = pack_f32x2(-m_use, -m_use);
+      unsigned long long lsum2 = pack_f32x2(0.f, 0.f);
       uint32_t packed[32];
 #pragma unroll
       for (int i = 0; i < 64; i += 2) {
-        const float p0 = fast_exp2(__uint_as_float(sr[i]) - m_use), p1 = fast_exp2(__uint_as_float(sr[i + 1]) - m_use);
-        lsum += p0 + p1;
+        float a0, a1;
+        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), scale2, negm2), a0, a1);
+        const float p0 = fast_exp2(a0), p1 = fast_exp2(a1);
+        lsum2 = add_f32x2(lsum2, pack_f32x2(p0, p1));
         packed[i >> 1] = pack_bf16(p0, p1);
       }
+      float lsum, lsum_hi;
+      unpack_f32x2(lsum2, lsum, lsum_hi);
+      lsum += lsum_hi;
       l_run += lsum;
       // Every PV phase is waited for, in order (a parity wait must never lag a whole phase), and
       // late: PV_{j-1} done also means PV_{j-2} has consumed the P buffer about to be overwritten.
