@@ -26,6 +26,7 @@ struct AttnParams {
   float* part_lse;  // [outer][total_q*Hq]    base-2 log-sum-exp of each partial
   int* status;
   int G;            // query heads per KV head
+  int row_tiles;    // 128-row query tiles per (sequence, KV head) in the grid
 };
 
 constexpr float kLn2 = 0.6931471805599453f;

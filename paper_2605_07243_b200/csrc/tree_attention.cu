@@ -146,8 +146,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
   const int S = (int)cluster.num_blocks();   // chunk-CTAs that merge through shared memory
   const int crank = (int)cluster.block_rank();
   const int split = blockIdx.x;              // chunk index among num_splits = S * outer
-  const int Hkv = p.tb.n_kv_heads, Hq = p.tb.n_q_heads, G = p.G;
-  const int g = blockIdx.y % Hkv, tile = blockIdx.y / Hkv;
+  const int Hq = p.tb.n_q_heads, G = p.G;
+  // row tiles of one (sequence, KV head) are neighbours in launch order: they share its K/V through L2
+  const int g = blockIdx.y / p.row_tiles, tile = blockIdx.y % p.row_tiles;
   const int b = blockIdx.z;
 
   const SeqPlan sp = plan_sequence(p, b, split == 0 && blockIdx.y == 0, s_parent, s_anc);
@@ -603,6 +604,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   if (impl == IMPL_SIMPLE) {
     p.num_splits = 1;
     p.outer = 1;
+    p.row_tiles = 1;
     dim3 grid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);
     if (D == 64) attn_simple_kernel<64><<<grid, 256, 0, cs>>>(p);
     else attn_simple_kernel<128><<<grid, 256, 0, cs>>>(p);
@@ -622,6 +624,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
     p.part_lse = reinterpret_cast<float*>(static_cast<char*>(workspace) + o);
   }
   const int row_tiles = ceil_div(tb->max_nodes * p.G, BM);
+  p.row_tiles = row_tiles;
   dim3 grid(p.num_splits, row_tiles * tb->n_kv_heads, tb->batch);
   if (grid.y > 65535 || grid.z > 65535) return SB_ERR_UNSUPPORTED;
   if (impl == IMPL_TC) st = launch_attn_tc(p, grid, plan.cluster, cs);

@@ -238,8 +238,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const int S = (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
   const int split = blockIdx.x;
-  const int Hkv = p.tb.n_kv_heads, Hq = p.tb.n_q_heads, G = p.G;
-  const int g = blockIdx.y % Hkv, tile = blockIdx.y / Hkv;
+  const int Hq = p.tb.n_q_heads, G = p.G;
+  // row tiles of one (sequence, KV head) are neighbours in launch order: they share its K/V through L2
+  const int g = blockIdx.y / p.row_tiles, tile = blockIdx.y % p.row_tiles;
   const int b = blockIdx.z;
   if (tid == 0) {
     *s_abort = 0;
