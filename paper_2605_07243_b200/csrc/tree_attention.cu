@@ -474,10 +474,19 @@ static int max_active_clusters(int D, int cluster) {
   return cache[di][cluster];
 }
 
-static SplitPlan plan_for(int s) {
+// `oversubscribed`: the grid has several waves of CTAs anyway.  Then clusters of 2 are preferred:
+// clusters of 8 full-SM CTAs keep only 120 of the 148 SMs busy, clusters of 2 all of them, and the
+// extra fp32 partials (one per cluster) cost less than the idle SMs (measured on the long-context
+// configuration: 1072 us against 1227 us).
+static SplitPlan plan_for(int s, bool oversubscribed) {
   SplitPlan sp;
   sp.cluster = 1;
-  for (int c = kMaxCluster; c >= 1; --c)
+  int cmax = oversubscribed ? 2 : kMaxCluster;
+  if (const char* e = getenv("SB_ATTN_MAX_CLUSTER")) {  // experiment knob
+    const int v = atoi(e);
+    if (v >= 1 && v <= kMaxCluster) cmax = v;
+  }
+  for (int c = cmax; c >= 1; --c)
     if (s % c == 0) { sp.cluster = c; break; }
   sp.outer = s / sp.cluster;
   return sp;
@@ -501,25 +510,28 @@ static SplitPlan choose_splits(const sb_tree_batch* tb, int num_splits, AttnImpl
   const int row_tiles = ceil_div(tb->max_nodes * G, BM);
   const int granule = impl == IMPL_TC ? 128 : BN;
   const int max_blocks = ceil_div(tb->max_kv_len, granule);
-  if (num_splits > 0) return plan_for(num_splits < max_blocks ? num_splits : max_blocks);
   const long long base = (long long)tb->batch * tb->n_kv_heads * row_tiles;
   const int sms = num_sms();
+  if (num_splits > 0) {
+    const int s = num_splits < max_blocks ? num_splits : max_blocks;
+    return plan_for(s, base * s > 2LL * sms);
+  }
   if (base > sms) {
     int s = impl == IMPL_TC ? max_blocks / 8 : max_blocks / 16;
     if (s > 16) s = 16;
     if (s < 1) s = 1;
-    return plan_for(s);
+    return plan_for(s, true);
   }
   int s = (int)(sms / base);
   if (s > max_blocks) s = max_blocks;
   for (; s > 1; --s) {
-    const SplitPlan sp = plan_for(s);
+    const SplitPlan sp = plan_for(s, false);
     if (sp.outer > 1 && sp.cluster < 4) continue;  // partial traffic for little gain
     const int fit = impl == IMPL_TC ? attn_tc_max_active_clusters(tb->head_dim, sp.cluster)
                                     : max_active_clusters(tb->head_dim, sp.cluster);
     if (fit <= 0 || base * sp.outer <= fit) return sp;
   }
-  return plan_for(1);
+  return plan_for(1, false);
 }
 
 static size_t workspace_bytes_for(const sb_tree_batch* tb, int total_q, int outer) {
