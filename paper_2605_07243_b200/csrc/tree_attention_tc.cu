@@ -323,8 +323,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     }
   };
   // The first loads go out before anything else: they only need the sequence's lengths.  Only
-  // what the first S product needs (Q and K block 0) is requested at once; the other first-wave
-  // tiles follow when K block 0 has landed, so they do not queue in front of it in the memory system.
+  // the K side (Q, K blocks 0 and 1) is requested at once; the V blocks, needed a softmax later,
+  // follow when K block 0 has landed, so they do not queue in front of it in the memory system.
   if (nb > 0 && lane == 0 && warp == TC_KLOAD_WARP) {
     if (q_tma) {
       mbar_expect_tx(&s_bar[Q_FULL], (uint32_t)(TC_BM * D * 2));
@@ -334,6 +334,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
                     &s_bar[Q_FULL]);
     }
     issue_block(0, &kmap, smem_u32(sK), &s_bar[K_FULL0]);
+    if (nb > 1) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
   }
 
   const SeqPlan sp = plan_tree(p, b, split == 0 && blockIdx.y == 0, pre, s_parent, s_anc);
@@ -523,10 +524,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     // ------------------------------------------------------------------ K loader (blocks 2..)
     if (lane == 0) {
       bool ok = true;
-      if (nb > 1) {
-        ok = mbar_wait(&s_bar[K_FULL0], 0, s_abort);
-        if (ok) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
-      }
       for (int j = 2; j < nb && ok; ++j) {
         ok = mbar_wait(&s_bar[K_EMPTY0 + (j & 1)], ((j >> 1) - 1) & 1, s_abort);
         if (ok) issue_block(j, &kmap, smem_u32(sK) + (j & 1) * TILE_BYTES, &s_bar[K_FULL0 + (j & 1)]);
@@ -630,52 +627,68 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     __syncthreads();
   }
   {
-    // One warp per row: lane c < S fetches source c's (m, l), the weights are formed with warp
-    // shuffles, then every lane combines four columns of the row (D/4 <= 32 lanes).
+    // One warp per row, two rows in flight per warp.  Every lane reads all S (m, l) pairs itself
+    // (broadcast loads) and forms the weights redundantly, then loads its four columns from all S
+    // sources at once: no serial chain over the sources and no shuffles.
     const uint8_t* src = S > 1 ? sRcv : stg;  // [source][row in my slice][ROWB]
-    for (int t = warp; t < my_rows; t += TC_THREADS / 32) {
-      const int Rr = row0 + my_first + t;
-      if (Rr >= rows_total) continue;  // uniform over the warp
-      const uint8_t* mine = src + ((size_t)(lane < S ? lane : 0) * rows_per + t) * ROWB;
-      const float mc = lane < S ? *reinterpret_cast<const float*>(mine + D * 2) : -INFINITY;
-      const float lc = lane < S ? *reinterpret_cast<const float*>(mine + D * 2 + 4) : 0.f;
-      float M = mc;
+    constexpr int NW = TC_THREADS / 32;
+    for (int t0 = warp; t0 < my_rows; t0 += 2 * NW) {
+      float w[2][8], M[2], Lsum[2];
+      uint2 raw[2][8];
+      bool live[2];
 #pragma unroll
-      for (int sft = 4; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sft));  // S <= 8 lanes
-      const float wl = mc == -INFINITY ? 0.f : fast_exp2(mc - M) * lc;  // weight of source `lane`: 2^(m-M) * l
-      float Lsum = wl;
+      for (int u = 0; u < 2; ++u) {
+        const int t = t0 + u * NW;
+        live[u] = t < my_rows && row0 + my_first + t < rows_total;
+        float mc[8], lc[8];
 #pragma unroll
-      for (int sft = 4; sft > 0; sft >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, sft);
-      M = __shfl_sync(0xffffffffu, M, 0);
-      Lsum = __shfl_sync(0xffffffffu, Lsum, 0);
-      const float inv = Lsum > 0.f ? __fdividef(1.f, Lsum) : 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 1
-      for (int c = 0; c < S; ++c) {
-        const float w = __shfl_sync(0xffffffffu, wl, c);
-        if (w != 0.f && lane < D / 4) {
-          const uint2 raw = *reinterpret_cast<const uint2*>(src + ((size_t)c * rows_per + t) * ROWB + lane * 8);
-          acc.x += w * __uint_as_float(raw.x << 16);
-          acc.y += w * __uint_as_float(raw.x & 0xffff0000u);
-          acc.z += w * __uint_as_float(raw.y << 16);
-          acc.w += w * __uint_as_float(raw.y & 0xffff0000u);
+        for (int c = 0; c < 8; ++c) {
+          const uint8_t* rowp = src + ((size_t)(c < S ? c : 0) * rows_per + (live[u] ? t : 0)) * ROWB;
+          mc[c] = (c < S && live[u]) ? *reinterpret_cast<const float*>(rowp + D * 2) : -INFINITY;
+          lc[c] = (c < S && live[u]) ? *reinterpret_cast<const float*>(rowp + D * 2 + 4) : 0.f;
+          raw[u][c] = (c < S && live[u] && lane < D / 4) ? *reinterpret_cast<const uint2*>(rowp + lane * 8) : make_uint2(0u, 0u);
         }
+        float m = mc[0];
+#pragma unroll
+        for (int c = 1; c < 8; ++c) m = fmaxf(m, mc[c]);
+        float ls = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          w[u][c] = mc[c] == -INFINITY ? 0.f : fast_exp2(mc[c] - m) * lc[c];  // 2^(m_c - M) * l_c
+          ls += w[u][c];
+        }
+        M[u] = m;
+        Lsum[u] = ls;
       }
-      acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-      const int node_l = Rr / G, hh = Rr - node_l * G;
-      const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
-      const float lse2 = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
-      if (lane < D / 4) {
-        if (p.outer == 1) {
-          uint2 packed;
-          packed.x = pack_bf16(acc.x, acc.y);
-          packed.y = pack_bf16(acc.z, acc.w);
-          *reinterpret_cast<uint2*>(p.out + grow * D + lane * 4) = packed;
-          if (p.lse && lane == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
-        } else {
-          const int outer_idx = split / S;
-          *reinterpret_cast<float4*>(p.part_o + (outer_idx * rows_all + grow) * D + lane * 4) = acc;
-          if (lane == 0) p.part_lse[outer_idx * rows_all + grow] = lse2;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        if (!live[u]) continue;  // uniform over the warp
+        const int Rr = row0 + my_first + t0 + u * NW;
+        const float inv = Lsum[u] > 0.f ? __fdividef(1.f, Lsum[u]) : 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          acc.x += w[u][c] * __uint_as_float(raw[u][c].x << 16);
+          acc.y += w[u][c] * __uint_as_float(raw[u][c].x & 0xffff0000u);
+          acc.z += w[u][c] * __uint_as_float(raw[u][c].y << 16);
+          acc.w += w[u][c] * __uint_as_float(raw[u][c].y & 0xffff0000u);
+        }
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        const int node_l = Rr / G, hh = Rr - node_l * G;
+        const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
+        const float lse2 = Lsum[u] > 0.f ? M[u] + log2f(Lsum[u]) : -INFINITY;
+        if (lane < D / 4) {
+          if (p.outer == 1) {
+            uint2 packed;
+            packed.x = pack_bf16(acc.x, acc.y);
+            packed.y = pack_bf16(acc.z, acc.w);
+            *reinterpret_cast<uint2*>(p.out + grow * D + lane * 4) = packed;
+            if (p.lse && lane == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
+          } else {
+            const int outer_idx = split / S;
+            *reinterpret_cast<float4*>(p.part_o + (outer_idx * rows_all + grow) * D + lane * 4) = acc;
+            if (lane == 0) p.part_lse[outer_idx * rows_all + grow] = lse2;
+          }
         }
       }
     }
