@@ -232,7 +232,6 @@ def run_ours(args):
         g_expand = capture(torch, step.run_expand)
         g_accept = capture(torch, step.run_accept)
         g_compact = capture(torch, step.run_compact)
-        g_layer0 = capture(torch, lambda: step.run_attention([0]))
 
         for _ in range(max(args.warmup, 3)):
             g_step.replay()
@@ -264,9 +263,6 @@ def run_ours(args):
             for _ in range(3):
                 g.replay()
             parts_ms[name] = time_graph(torch, g, 20, False) / 20
-        # one layer alone, cold L2: flush by streaming the other layers' KV between replays is what
-        # g_attn does; here the single layer is replayed back to back (warm L2) for contrast
-        parts_ms["attention_layer_warm_l2"] = time_graph(torch, g_layer0, 50, False) / 50
 
         # end to end: inputs in pinned host memory, results back to pinned host memory
         e2e_steps = 1 if args.quick else max(3, min(args.steps, 5))

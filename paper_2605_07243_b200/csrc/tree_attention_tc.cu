@@ -627,68 +627,65 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     __syncthreads();
   }
   {
-    // One warp per row, two rows in flight per warp.  Every lane reads all S (m, l) pairs itself
-    // (broadcast loads) and forms the weights redundantly, then loads its four columns from all S
-    // sources at once: no serial chain over the sources and no shuffles.
+    // One row per half-warp, eight columns per lane (D <= 128).  Every lane reads all S (m, l)
+    // pairs itself (broadcast loads) and forms the weights redundantly, then loads its columns
+    // from all S sources at once: no serial chain over the sources and no shuffles.
     const uint8_t* src = S > 1 ? sRcv : stg;  // [source][row in my slice][ROWB]
-    constexpr int NW = TC_THREADS / 32;
-    for (int t0 = warp; t0 < my_rows; t0 += 2 * NW) {
-      float w[2][8], M[2], Lsum[2];
-      uint2 raw[2][8];
-      bool live[2];
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int t = t0 + u * NW;
-        live[u] = t < my_rows && row0 + my_first + t < rows_total;
+    const int sub = lane >> 4, col8 = lane & 15;
+    for (int t = 2 * warp + sub; t < my_rows; t += 2 * (TC_THREADS / 32)) {
+      const int Rr = row0 + my_first + t;
+      if (Rr >= rows_total) continue;
+      const bool has_cols = col8 < D / 8;
+      float w[8];
+      uint4 raw[8];
+      float M = -INFINITY, Lsum = 0.f;
+      {
         float mc[8], lc[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-          const uint8_t* rowp = src + ((size_t)(c < S ? c : 0) * rows_per + (live[u] ? t : 0)) * ROWB;
-          mc[c] = (c < S && live[u]) ? *reinterpret_cast<const float*>(rowp + D * 2) : -INFINITY;
-          lc[c] = (c < S && live[u]) ? *reinterpret_cast<const float*>(rowp + D * 2 + 4) : 0.f;
-          raw[u][c] = (c < S && live[u] && lane < D / 4) ? *reinterpret_cast<const uint2*>(rowp + lane * 8) : make_uint2(0u, 0u);
+          const uint8_t* rowp = src + ((size_t)(c < S ? c : 0) * rows_per + t) * ROWB;
+          mc[c] = c < S ? *reinterpret_cast<const float*>(rowp + D * 2) : -INFINITY;
+          lc[c] = c < S ? *reinterpret_cast<const float*>(rowp + D * 2 + 4) : 0.f;
+          raw[c] = (c < S && has_cols) ? *reinterpret_cast<const uint4*>(rowp + col8 * 16) : make_uint4(0u, 0u, 0u, 0u);
+          M = fmaxf(M, mc[c]);
         }
-        float m = mc[0];
-#pragma unroll
-        for (int c = 1; c < 8; ++c) m = fmaxf(m, mc[c]);
-        float ls = 0.f;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-          w[u][c] = mc[c] == -INFINITY ? 0.f : fast_exp2(mc[c] - m) * lc[c];  // 2^(m_c - M) * l_c
-          ls += w[u][c];
+          w[c] = mc[c] == -INFINITY ? 0.f : fast_exp2(mc[c] - M) * lc[c];  // 2^(m_c - M) * l_c
+          Lsum += w[c];
         }
-        M[u] = m;
-        Lsum[u] = ls;
       }
+      const float inv = Lsum > 0.f ? __fdividef(1.f, Lsum) : 0.f;
+      float acc[8];
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        if (!live[u]) continue;  // uniform over the warp
-        const int Rr = row0 + my_first + t0 + u * NW;
-        const float inv = Lsum[u] > 0.f ? __fdividef(1.f, Lsum[u]) : 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          acc.x += w[u][c] * __uint_as_float(raw[u][c].x << 16);
-          acc.y += w[u][c] * __uint_as_float(raw[u][c].x & 0xffff0000u);
-          acc.z += w[u][c] * __uint_as_float(raw[u][c].y << 16);
-          acc.w += w[u][c] * __uint_as_float(raw[u][c].y & 0xffff0000u);
+      for (int c = 0; c < 8; ++c) {
+        const uint32_t q4[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          acc[2 * e] += w[c] * __uint_as_float(q4[e] << 16);
+          acc[2 * e + 1] += w[c] * __uint_as_float(q4[e] & 0xffff0000u);
         }
-        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        const int node_l = Rr / G, hh = Rr - node_l * G;
-        const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
-        const float lse2 = Lsum[u] > 0.f ? M[u] + log2f(Lsum[u]) : -INFINITY;
-        if (lane < D / 4) {
-          if (p.outer == 1) {
-            uint2 packed;
-            packed.x = pack_bf16(acc.x, acc.y);
-            packed.y = pack_bf16(acc.z, acc.w);
-            *reinterpret_cast<uint2*>(p.out + grow * D + lane * 4) = packed;
-            if (p.lse && lane == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
-          } else {
-            const int outer_idx = split / S;
-            *reinterpret_cast<float4*>(p.part_o + (outer_idx * rows_all + grow) * D + lane * 4) = acc;
-            if (lane == 0) p.part_lse[outer_idx * rows_all + grow] = lse2;
-          }
+      }
+      const int node_l = Rr / G, hh = Rr - node_l * G;
+      const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
+      const float lse2 = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
+      if (has_cols) {
+        if (p.outer == 1) {
+          uint4 packed;
+          packed.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+          packed.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+          packed.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+          packed.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+          *reinterpret_cast<uint4*>(p.out + grow * D + col8 * 8) = packed;
+          if (p.lse && col8 == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
+        } else {
+          const int outer_idx = split / S;
+          float* po = p.part_o + (outer_idx * rows_all + grow) * D + col8 * 8;
+          *reinterpret_cast<float4*>(po) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+          *reinterpret_cast<float4*>(po + 4) = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);
+          if (col8 == 0) p.part_lse[outer_idx * rows_all + grow] = lse2;
         }
       }
     }
