@@ -10,6 +10,7 @@ from .oracle import (  # noqa: F401
     tree_attention,
     row_argmax,
     row_topk,
+    rank_features,
     verify_accept,
     accept_from_amax,
     kv_compact,

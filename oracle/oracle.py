@@ -129,6 +129,16 @@ def row_topk(scores, vocab=None):
     return tok, val
 
 
+def rank_features(scores, vocab=None):
+    """-> float64 [n_rows, 15]: top-10 log-probs, 3 logit gaps, top probability, entropy."""
+    scores = np.ascontiguousarray(scores, np.float32)
+    n_rows, stride = scores.shape
+    vocab = stride if vocab is None else vocab
+    feats = np.zeros((n_rows, 15), np.float64)
+    _load().sbo_rank_features(_p(scores), C.c_int64(stride), C.c_int(n_rows), C.c_int(vocab), _p(feats))
+    return feats
+
+
 def verify_accept(logits, node_offsets, parent, tok, max_depth, vocab=None):
     """-> dict(amax, accept_len, path_nodes, out_tokens, bonus, status)."""
     logits, dt = _logits_arg(logits)

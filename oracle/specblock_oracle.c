@@ -17,6 +17,7 @@
  *   sbo_verify_accept   : exhaustive comparison with an independent recurrence on all small
  *                         trees; planted paths; the case-study tree (4 accepted + bonus).
  *   sbo_kv_compact      : numpy fancy-index gather; attention over the compacted cache.
+ *   sbo_rank_features   : scipy log_softmax / entropy; closed forms (uniform row, one dominant token).
  *   sbo_tree_expand     : hand-derived trees for the two printed branching maps; chain special
  *                         case; structural invariants.  The attach point of siblings, the cut
  *                         order at the node budget and the treatment of b = 0 are readings of
@@ -444,6 +445,52 @@ int sbo_tree_expand(const float* scores, int64_t row_stride, int n_rows, int voc
   }
   *n_nodes = n;
   return 0;
+}
+
+/* ---- psi(p): the rank head's 15-dimensional summary of a draft distribution (App. B) ----------- */
+
+/*
+ * For every row of drafter scores (logits), with p = softmax(row) (NaN scores count as -inf):
+ *   features[0..9]  natural-log probabilities of the ten most likely tokens, most likely first
+ *                   (value descending, id ascending; -inf where the vocabulary has fewer than ten);
+ *   features[10..12] logit gaps between the top token and the tokens of rank 2, 3 and 5
+ *                   (+inf where that rank does not exist);
+ *   features[13]    probability of the top token;
+ *   features[14]    entropy -sum p ln p in nats (terms with p = 0 contribute nothing).
+ * Plain definition: exact maximum, fp64 log-sum-exp over the whole row, full sort.
+ */
+void sbo_rank_features(const float* scores, int64_t row_stride, int n_rows, int vocab, double* features) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int r = 0; r < n_rows; ++r) {
+    scored* e = (scored*)malloc(sizeof(scored) * (size_t)vocab);
+    double m = -INFINITY;
+    for (int v = 0; v < vocab; ++v) {
+      e[v].val = score_of((double)scores[(int64_t)r * row_stride + v]);
+      e[v].id = v;
+      if (e[v].val > m) m = e[v].val;
+    }
+    double* f = features + (int64_t)r * 15;
+    if (m == -INFINITY) { /* no finite score: the distribution is undefined; report a flat one */
+      m = 0.0;
+      for (int v = 0; v < vocab; ++v) e[v].val = 0.0;
+    }
+    double z = 0.0;
+    for (int v = 0; v < vocab; ++v) z += exp(e[v].val - m);
+    const double log_z = m + log(z);
+    double entropy = 0.0;
+    for (int v = 0; v < vocab; ++v) {
+      const double lp = e[v].val - log_z;
+      if (lp > -INFINITY) entropy -= exp(lp) * lp;
+    }
+    qsort(e, (size_t)vocab, sizeof(scored), by_score_desc_id_asc);
+    for (int j = 0; j < 10; ++j) f[j] = j < vocab ? e[j].val - log_z : -INFINITY;
+    f[10] = vocab > 1 ? e[0].val - e[1].val : INFINITY;
+    f[11] = vocab > 2 ? e[0].val - e[2].val : INFINITY;
+    f[12] = vocab > 4 ? e[0].val - e[4].val : INFINITY;
+    f[13] = exp(e[0].val - log_z);
+    f[14] = entropy;
+    free(e);
+  }
 }
 
 /* Threads the OpenMP loops above use (1 when built without OpenMP). */

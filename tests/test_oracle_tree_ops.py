@@ -340,3 +340,42 @@ def test_expand_rejects_bad_arguments():
     assert oracle.tree_expand(c.scores, 4, [0, 1, 4, 0], c.bmap, [-1], 20)["status"] == 1
     assert oracle.tree_expand(c.scores, 4, c.bucket, [2, 4, 17, 0], [-1], 20)["status"] == 1
     assert oracle.tree_expand(c.scores, 4, c.bucket, c.bmap, [0], 20)["status"] == 1
+
+
+# ---- rank-head distribution summary psi(p) (App. B) --------------------------------------------------------
+
+def test_rank_features_match_scipy_and_closed_forms():
+    from scipy.special import log_softmax
+    from scipy.stats import entropy as scipy_entropy
+    rng = W.rng_for(33)
+    x = (rng.standard_normal((5, 3000), dtype=np.float32) * 3).astype(np.float32)
+    x[1] = np.round(x[1])                       # ties among the leaders
+    x[2, ::7] = np.nan                          # NaN counts as -inf
+    x[3, 5:] = -np.inf                          # only five finite scores
+    f = oracle.rank_features(x)
+    clean = np.where(np.isnan(x), -np.inf, x).astype(np.float64)
+    lsm = log_softmax(clean, axis=1)            # library routine
+    order = np.argsort(-clean, axis=1, kind="stable")
+    top = np.take_along_axis(clean, order[:, :10], 1)
+    np.testing.assert_allclose(f[:, :10], np.take_along_axis(lsm, order[:, :10], 1), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(f[:, 10], top[:, 0] - top[:, 1], atol=1e-12)
+    np.testing.assert_allclose(f[:, 11], top[:, 0] - top[:, 2], atol=1e-12)
+    np.testing.assert_allclose(f[:, 12], top[:, 0] - top[:, 4], atol=1e-12)
+    np.testing.assert_allclose(f[:, 13], np.exp(lsm.max(axis=1)), rtol=1e-12)
+    np.testing.assert_allclose(f[:, 14], [scipy_entropy(np.exp(r)) for r in lsm], rtol=1e-10)
+    assert np.isneginf(f[3, 5:10]).all()          # row 3 has only five finite scores
+    # closed forms: a uniform row has entropy ln V, zero gaps and log-probs -ln V ...
+    V = 1000
+    u = oracle.rank_features(np.full((1, V), 2.5, np.float32))[0]
+    np.testing.assert_allclose(u[:10], -np.log(V), rtol=1e-12)
+    np.testing.assert_allclose(u[10:13], 0.0, atol=1e-12)
+    np.testing.assert_allclose(u[13:], [1.0 / V, np.log(V)], rtol=1e-12)
+    # ... and one token 50 above the rest owns the distribution: entropy ~ 0, top probability ~ 1
+    d = np.zeros((1, V), np.float32)
+    d[0, 123] = 50.0
+    o = oracle.rank_features(d)[0]
+    assert abs(o[0]) < 1e-18 and abs(o[13] - 1.0) < 1e-15 and o[14] < 1e-15
+    np.testing.assert_allclose(o[10:13], 50.0)
+    # fewer than ten / five tokens
+    s = oracle.rank_features(np.asarray([[1.0, 3.0, 2.0]], np.float32))[0]
+    assert np.isneginf(s[3:10]).all() and s[10] == 1.0 and s[11] == 2.0 and np.isposinf(s[12])
