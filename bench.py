@@ -232,6 +232,8 @@ def run_ours(args):
         g_expand = capture(torch, step.run_expand)
         g_accept = capture(torch, step.run_accept)
         g_compact = capture(torch, step.run_compact)
+        step.run_rank_features()
+        g_features = capture(torch, step.run_rank_features)
 
         for _ in range(max(args.warmup, 3)):
             g_step.replay()
@@ -259,7 +261,8 @@ def run_ours(args):
         keep_busy(0.4)
         clocks = sampler.stop()
         parts_ms = {}
-        for name, g in (("expand", g_expand), ("accept", g_accept), ("compact", g_compact)):
+        for name, g in (("expand", g_expand), ("accept", g_accept), ("compact", g_compact),
+                        ("rank_features_not_in_step", g_features)):
             for _ in range(3):
                 g.replay()
             parts_ms[name] = time_graph(torch, g, 20, False) / 20

@@ -10,6 +10,7 @@
  *   sb_tree_ancestors  ancestor bitmask / depth of every tree node      (Sec. 3.1, App. A.2, Fig. 4)
  *   sb_tree_attention  tree-masked attention over prefix KV + ancestors (Sec. 3.1, App. A.2, Alg. 1 "verify")
  *   sb_tree_expand     per-row top-k + bucket-driven branching          (Sec. 3.2, App. A.5, Alg. 1 "attach")
+ *   sb_rank_features   15-dim summary of each draft distribution        (Sec. 3.2, App. B)
  *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
  *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
  *
@@ -163,6 +164,26 @@ sb_status sb_tree_expand(const float* scores, int64_t row_stride, int32_t n_rows
                          int32_t* node_rank, int32_t* topk_tok, float* topk_val, void* workspace,
                          size_t workspace_bytes, int32_t* status, void* stream);
 size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab);
+
+/*
+ * sb_rank_features -- the rank head's 15-dimensional summary psi(p) of every draft distribution
+ * (Sec. 3.2 "rank head"; App. B "distribution summary features").
+ *
+ *   scores fp32 [n_rows][row_stride >= vocab] are the drafter's logits; p = softmax(row), NaN read
+ *   as -inf.  features fp32 [n_rows][15], in the order the appendix lists them:
+ *     [0..9]   natural-log probabilities of the ten most likely tokens, most likely first
+ *              (-inf where the vocabulary has fewer than ten tokens);
+ *     [10..12] logit gaps between the top token and the tokens of rank 2, 3 and 5 (+inf where
+ *              that rank does not exist);
+ *     [13]     probability of the top token;   [14] entropy -sum p ln p in nats.
+ *   A row without any finite score is reported as the uniform distribution.
+ *   The scores are streamed once (the same scan as sb_tree_expand's top-k, which also yields the
+ *   chunk maxima and the two exponential sums); accuracy is that of fp32 sums over the row.
+ *   workspace : sb_rank_features_workspace_bytes(n_rows, vocab) bytes, 256-byte aligned.
+ */
+sb_status sb_rank_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                           float* features, void* workspace, size_t workspace_bytes, void* stream);
+size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
 
 /*
  * sb_verify_accept -- greedy (temperature 0) verification (App. A.5 "the longest accepted

@@ -62,10 +62,10 @@ def load(build_if_missing: bool = True):
     lib.sb_version.restype = C.c_int32
     lib.sb_kernel_launch_count.restype = C.c_int64
     for name in ("sb_tree_attention_workspace_bytes", "sb_tree_expand_workspace_bytes",
-                 "sb_verify_accept_workspace_bytes"):
+                 "sb_verify_accept_workspace_bytes", "sb_rank_features_workspace_bytes"):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
-                 "sb_verify_accept_static", "sb_kv_compact"):
+                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -74,7 +74,7 @@ def load(build_if_missing: bool = True):
 EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspace_bytes",
             "sb_tree_expand", "sb_tree_expand_workspace_bytes", "sb_verify_accept",
             "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
-            "sb_status_string", "sb_version",
+            "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_status_string", "sb_version",
             "sb_kernel_launch_count")
 
 
@@ -228,6 +228,26 @@ def sb_verify_accept(logits, node_offsets, parent, tok, max_depth, *, vocab=None
                               C.c_size_t(workspace.numel()), _ptr(out["status"]), _stream())
     _check(rc, "sb_verify_accept")
     return out
+
+
+def sb_rank_features_workspace_bytes(n_rows: int, vocab: int) -> int:
+    return int(load().sb_rank_features_workspace_bytes(C.c_int32(n_rows), C.c_int32(vocab)))
+
+
+def sb_rank_features(scores, *, vocab=None, features=None, workspace=None):
+    """scores fp32 [R, stride] -> features fp32 [R, 15] (top-10 log-probs, 3 logit gaps, top
+    probability, entropy)."""
+    n_rows, stride = scores.shape
+    vocab = stride if vocab is None else vocab
+    dev = scores.device
+    features = torch.empty((n_rows, 15), dtype=torch.float32, device=dev) if features is None else features
+    if workspace is None:
+        workspace = torch.empty(max(sb_rank_features_workspace_bytes(n_rows, vocab), 256), dtype=torch.uint8, device=dev)
+    rc = load().sb_rank_features(_ptr(scores, torch.float32), C.c_int64(stride), C.c_int32(n_rows), C.c_int32(vocab),
+                                 _ptr(features, torch.float32), _ptr(workspace), C.c_size_t(workspace.numel()),
+                                 _stream())
+    _check(rc, "sb_rank_features")
+    return features
 
 
 SB_STATIC_SCRATCH_BYTES = 256 * 1024

@@ -24,11 +24,42 @@ constexpr int kNoId = 0x7fffffff;
 
 __device__ inline bool ranks_before(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
 
+// Softmax statistics of a chunk for the rank head's distribution summary (App. B): with m the
+// chunk maximum, s = sum exp(x - m) and t = sum exp(x - m) * x.  `tmax`, `s`, `t` are this thread's
+// share (s, t relative to the CTA maximum returned through *cta_max by the first call).
+__device__ inline float cta_reduce_max(float v, float* s_red) {
+#pragma unroll
+  for (int sft = 16; sft > 0; sft >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, sft));
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = s_red[0];
+  for (int w = 1; w < (int)(blockDim.x >> 5); ++w) r = fmaxf(r, s_red[w]);
+  __syncthreads();
+  return r;
+}
+__device__ inline float cta_reduce_sum(float v, float* s_red) {
+#pragma unroll
+  for (int sft = 16; sft > 0; sft >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sft);
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = 0.f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) r += s_red[w];
+  __syncthreads();
+  return r;
+}
+__device__ inline void stats_term(float x, float m, float& s, float& t) {
+  const float e = exp2f((x - m) * 1.4426950408889634f);  // x = -inf gives 0
+  s += e;
+  t += e > 0.f ? e * x : 0.f;
+}
+
+template <bool STATS>
 __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float* __restrict__ scores,
                                                                     long long row_stride, int vocab, int chunk,
                                                                     int n_chunks, bool vec_ok,
                                                                     float* __restrict__ part_val,
-                                                                    int* __restrict__ part_idx) {
+                                                                    int* __restrict__ part_idx,
+                                                                    float* __restrict__ part_stats) {
   __shared__ float s_val[SB_KMAX][TOPK_THREADS];  // [rank][thread]: conflict-free per-thread lists
   __shared__ int s_idx[SB_KMAX][TOPK_THREADS];
   __shared__ float s_wv[TOPK_THREADS / 32];
@@ -65,6 +96,27 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
   __syncthreads();
   const float tau = s_tau;
   __syncthreads();  // s_max (aliasing the lists) is dead from here on
+  if (STATS) {  // chunk maximum, then one more pass (L1/L2 hits) for the two sums
+    __shared__ float s_red[TOPK_THREADS / 32];
+    const float cmax = cta_reduce_max(tmax, s_red);
+    float ss = 0.f, tt = 0.f;
+    if (cmax > -INFINITY) {
+      for (int t = tid; t < n_vec; t += TOPK_THREADS) {
+        const float4 x = __ldg(vb + t);
+        stats_term(score_of(x.x), cmax, ss, tt);
+        stats_term(score_of(x.y), cmax, ss, tt);
+        stats_term(score_of(x.z), cmax, ss, tt);
+        stats_term(score_of(x.w), cmax, ss, tt);
+      }
+      for (int i = begin + n_vec * 4 + tid; i < end; i += TOPK_THREADS) stats_term(score_of(base[i]), cmax, ss, tt);
+    }
+    ss = cta_reduce_sum(ss, s_red);
+    tt = cta_reduce_sum(tt, s_red);
+    if (tid == 0) {
+      float* o = part_stats + ((long long)row * n_chunks + c) * 3;
+      o[0] = cmax; o[1] = ss; o[2] = tt;
+    }
+  }
 
   float v[SB_KMAX];
   int id[SB_KMAX];
@@ -144,10 +196,12 @@ constexpr int TOPK_VEC_PER_THREAD = 16;
 constexpr int TOPK_REG_ELEMS = TOPK_THREADS * TOPK_VEC_PER_THREAD * 4;  // 16384
 constexpr int TOPK_CAND = 512;
 
+template <bool STATS>
 __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const float* __restrict__ scores,
                                                                         long long row_stride, int vocab, int chunk,
                                                                         int n_chunks, float* __restrict__ part_val,
-                                                                        int* __restrict__ part_idx) {
+                                                                        int* __restrict__ part_idx,
+                                                                        float* __restrict__ part_stats) {
   __shared__ float s_val[SB_KMAX][TOPK_THREADS];  // fallback lists; the candidate arrays alias them
   __shared__ int s_idx[SB_KMAX][TOPK_THREADS];
   __shared__ float s_group[16];
@@ -177,6 +231,33 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
     }
     x[i] = t;
     tmax = fmaxf(tmax, fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w)));
+  }
+  if (STATS) {  // softmax statistics of the chunk from the values already in registers
+    __shared__ float s_red[TOPK_THREADS / 32];
+    float tail_max = -INFINITY;
+    if (tid == 0)
+      for (int id2 = begin + 4 * n_vec; id2 < end; ++id2) tail_max = fmaxf(tail_max, score_of(base[id2]));
+    const float cmax = cta_reduce_max(fmaxf(tmax, tail_max), s_red);
+    float ss = 0.f, tt = 0.f;
+    if (cmax > -INFINITY) {
+#pragma unroll
+      for (int i = 0; i < TOPK_VEC_PER_THREAD; ++i) {
+        if (tid + i * TOPK_THREADS < n_vec) {
+          stats_term(x[i].x, cmax, ss, tt);
+          stats_term(x[i].y, cmax, ss, tt);
+          stats_term(x[i].z, cmax, ss, tt);
+          stats_term(x[i].w, cmax, ss, tt);
+        }
+      }
+      if (tid == 0)
+        for (int id2 = begin + 4 * n_vec; id2 < end; ++id2) stats_term(score_of(base[id2]), cmax, ss, tt);
+    }
+    ss = cta_reduce_sum(ss, s_red);
+    tt = cta_reduce_sum(tt, s_red);
+    if (tid == 0) {
+      float* o = part_stats + ((long long)row * n_chunks + c) * 3;
+      o[0] = cmax; o[1] = ss; o[2] = tt;
+    }
   }
   float gmax = tmax;
 #pragma unroll
@@ -436,6 +517,85 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
   }
 }
 
+// psi(p) of every row from the chunk partials: a warp per row merges the chunk lists (value
+// descending, id ascending) and the chunk statistics (m, s, t):  M = max m_c,
+// S = sum s_c e^(m_c - M), T = sum t_c e^(m_c - M); ln Z = M + ln S; entropy = ln Z - T / S.
+__global__ void __launch_bounds__(256) rank_features_finish_kernel(int n_rows, int n_chunks, int vocab,
+                                                                   const float* __restrict__ part_val,
+                                                                   const int* __restrict__ part_idx,
+                                                                   const float* __restrict__ part_stats,
+                                                                   float* __restrict__ features) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * 8 + warp;
+  if (r >= n_rows) return;
+  float lv[SB_KMAX];
+  int li[SB_KMAX];
+  float m = -INFINITY, sc = 0.f, tc = 0.f;
+  if (lane < n_chunks) {
+    const float4* pv = reinterpret_cast<const float4*>(part_val + ((long long)r * n_chunks + lane) * SB_KMAX);
+    const int4* pi = reinterpret_cast<const int4*>(part_idx + ((long long)r * n_chunks + lane) * SB_KMAX);
+#pragma unroll
+    for (int q = 0; q < SB_KMAX / 4; ++q) {
+      const float4 a = pv[q];
+      const int4 c = pi[q];
+      lv[4 * q] = a.x; lv[4 * q + 1] = a.y; lv[4 * q + 2] = a.z; lv[4 * q + 3] = a.w;
+      li[4 * q] = c.x; li[4 * q + 1] = c.y; li[4 * q + 2] = c.z; li[4 * q + 3] = c.w;
+    }
+    const float* st = part_stats + ((long long)r * n_chunks + lane) * 3;
+    m = st[0]; sc = st[1]; tc = st[2];
+  } else {
+#pragma unroll
+    for (int k = 0; k < SB_KMAX; ++k) { lv[k] = -INFINITY; li[k] = kNoId; }
+  }
+  float M = m;
+#pragma unroll
+  for (int sft = 16; sft > 0; sft >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sft));
+  const float wgt = m > -INFINITY ? exp2f((m - M) * 1.4426950408889634f) : 0.f;
+  float S = sc * wgt, T = tc * wgt;
+#pragma unroll
+  for (int sft = 16; sft > 0; sft >>= 1) {
+    S += __shfl_xor_sync(0xffffffffu, S, sft);
+    T += __shfl_xor_sync(0xffffffffu, T, sft);
+  }
+  // the ten best values of the row, in order (lane k keeps rank k)
+  float keep = -INFINITY;
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    float hv = lv[0];
+    int hi = li[0], hl = lane;
+#pragma unroll
+    for (int sft = 16; sft > 0; sft >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, hv, sft);
+      const int oi = __shfl_xor_sync(0xffffffffu, hi, sft);
+      const int ol = __shfl_xor_sync(0xffffffffu, hl, sft);
+      if (ranks_before(ov, oi, hv, hi)) { hv = ov; hi = oi; hl = ol; }
+    }
+    if (lane == round) keep = hi == kNoId ? NAN : hv;  // NaN marks "no such rank"
+    if (hi != kNoId && lane == hl) {
+#pragma unroll
+      for (int k = 0; k + 1 < SB_KMAX; ++k) { lv[k] = lv[k + 1]; li[k] = li[k + 1]; }
+      lv[SB_KMAX - 1] = -INFINITY;
+      li[SB_KMAX - 1] = kNoId;
+    }
+  }
+  const bool flat = !(M > -INFINITY);  // no finite score: reported as the uniform distribution
+  const float log_z = flat ? logf((float)vocab) : M + logf(S);
+  const float v0 = __shfl_sync(0xffffffffu, keep, 0);
+  const float v1 = __shfl_sync(0xffffffffu, keep, 1);
+  const float v2 = __shfl_sync(0xffffffffu, keep, 2);
+  const float v4 = __shfl_sync(0xffffffffu, keep, 4);
+  float* f = features + (long long)r * 15;
+  if (lane < 10) {
+    const bool exists = keep == keep;
+    f[lane] = !exists ? -INFINITY : (flat ? -log_z : keep - log_z);
+  }
+  if (lane == 10) f[10] = v1 == v1 ? (flat ? 0.f : v0 - v1) : INFINITY;
+  if (lane == 11) f[11] = v2 == v2 ? (flat ? 0.f : v0 - v2) : INFINITY;
+  if (lane == 12) f[12] = v4 == v4 ? (flat ? 0.f : v0 - v4) : INFINITY;
+  if (lane == 13) f[13] = flat ? 1.f / (float)vocab : expf(v0 - log_z);
+  if (lane == 14) f[14] = flat ? log_z : log_z - T / S;
+}
+
 static int topk_chunks(int n_rows, int vocab) {
   int nc = ceil_div(2 * 148, n_rows > 0 ? n_rows : 1);
   const int max_nc = ceil_div(vocab, 2048);
@@ -481,15 +641,52 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
   int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + need / 2);
   dim3 grid(nc, n_rows);
   if (vec_ok && chunk <= TOPK_REG_ELEMS)
-    topk_partial_reg_kernel<<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, part_val, part_idx);
+    topk_partial_reg_kernel<false><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, part_val,
+                                                                  part_idx, nullptr);
   else
-    topk_partial_kernel<<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
-                                                       part_idx);
+    topk_partial_kernel<false><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
+                                                              part_idx, nullptr);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
   expand_finish_kernel<<<1, FINISH_THREADS, 0, cs>>>(n_rows, nc, part_val, part_idx, block_k, bucket,
                                                      make_int4(bmap[0], bmap[1], bmap[2], bmap[3]),
                                                      start_parent, node_budget, vocab, n_nodes, tok, parent,
                                                      depth, node_row, node_rank, topk_tok, topk_val, status);
+  return launch_check();
+}
+
+extern "C" size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab) {
+  if (n_rows < 1 || vocab < 1) return 0;
+  const size_t nc = (size_t)sb::topk_chunks(n_rows, vocab);
+  return sb_tree_expand_workspace_bytes(n_rows, vocab) + (((size_t)n_rows * nc * 3 * 4 + 255) & ~(size_t)255);
+}
+
+extern "C" sb_status sb_rank_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                                      float* features, void* workspace, size_t workspace_bytes, void* stream) {
+  using namespace sb;
+  if (!scores || !features || n_rows < 1 || vocab < 1 || row_stride < vocab) return SB_ERR_INVALID_ARG;
+  if (n_rows > 65535) return SB_ERR_UNSUPPORTED;
+  const size_t need = sb_rank_features_workspace_bytes(n_rows, vocab);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SB_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int nc = topk_chunks(n_rows, vocab);
+  int chunk = ceil_div(vocab, nc);
+  chunk = ceil_div(chunk, 4) * 4;
+  const bool vec_ok = (reinterpret_cast<uintptr_t>(scores) & 15) == 0 && row_stride % 4 == 0;
+  const size_t lists = sb_tree_expand_workspace_bytes(n_rows, vocab);
+  float* part_val = static_cast<float*>(workspace);
+  int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + lists / 2);
+  float* part_stats = reinterpret_cast<float*>(static_cast<char*>(workspace) + lists);
+  dim3 grid(nc, n_rows);
+  if (vec_ok && chunk <= TOPK_REG_ELEMS)
+    topk_partial_reg_kernel<true><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, part_val,
+                                                                 part_idx, part_stats);
+  else
+    topk_partial_kernel<true><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
+                                                             part_idx, part_stats);
+  sb_status st = launch_check();
+  if (st != SB_OK) return st;
+  rank_features_finish_kernel<<<ceil_div(n_rows, 8), 256, 0, cs>>>(n_rows, nc, vocab, part_val, part_idx, part_stats,
+                                                                   features);
   return launch_check();
 }

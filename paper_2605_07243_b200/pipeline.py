@@ -115,6 +115,18 @@ class VerifyStep:
                           tree, workspace=e["ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"],
                           status=e["status"])
 
+    def run_rank_features(self):
+        """psi(p) of every drafter row (not part of run_device(): a 'next' row, timed on its own)."""
+        e = self.expand
+        if e is None:
+            return None
+        if "features" not in e:
+            R, V = e["scores"].shape
+            e["features"] = torch.empty((R, 15), dtype=torch.float32, device=self.device)
+            e["features_ws"] = torch.empty(max(256, sb.sb_rank_features_workspace_bytes(R, V)), dtype=torch.uint8,
+                                           device=self.device)
+        return sb.sb_rank_features(e["scores"], features=e["features"], workspace=e["features_ws"])
+
     def run_attention(self, layers=None):
         for l in range(self.n_layers) if layers is None else layers:
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,

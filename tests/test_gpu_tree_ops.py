@@ -273,3 +273,41 @@ def test_accept_then_compact_chain_on_device():
     got_k = tb.k_cache.view(torch.int16).cpu().numpy().view(np.uint16)
     for j, node in enumerate(path):
         np.testing.assert_array_equal(got_k[0, 200 + j], case.k[0, 200 + node])
+
+
+# ---- rank-head distribution summary -------------------------------------------------------------------
+
+# fp32 sums over rows of up to 128256 terms: |err| <= 2e-5 * max(1, |ref|)
+FEAT_TOL = 2e-5
+
+
+def _check_features(scores, vocab=None):
+    got = sb.sb_rank_features(torch.from_numpy(np.ascontiguousarray(scores)).cuda(), vocab=vocab)
+    torch.cuda.synchronize()
+    got = got.cpu().numpy().astype(np.float64)
+    ref = oracle.rank_features(scores, vocab=vocab)
+    inf = np.isinf(ref)
+    np.testing.assert_array_equal(got[inf], ref[inf])
+    err = np.abs(got[~inf] - ref[~inf]) / np.maximum(1.0, np.abs(ref[~inf]))
+    assert err.max() <= FEAT_TOL, f"feature error {err.max():.2e}"
+    return got
+
+
+def test_rank_features_config3_full_vocab():
+    _, exp = W.config3_drafter()
+    got = _check_features(exp.scores)
+    assert (np.diff(got[:, :10], axis=1) <= 0).all()          # log-probs are listed in descending order
+
+
+@pytest.mark.parametrize("vocab", [3, 17, 1000, 4099, 32000])
+def test_rank_features_vocab_sizes_ties_nan_inf(vocab):
+    rng = W.rng_for(90 + vocab)
+    x = (rng.standard_normal((7, vocab + 5), dtype=np.float32) * 3).astype(np.float32)
+    x[:, vocab:] = 1e9                      # padding beyond vocab
+    x[1, :vocab] = np.round(x[1, :vocab])    # ties among the leaders
+    x[2, :vocab:3] = np.nan
+    x[3, :vocab] = -np.inf                   # no finite score: reported as uniform
+    x[4, 2:vocab] = -np.inf                  # two finite scores only
+    x[5, :vocab] = 4.0                       # exactly uniform
+    x[6, 1] = 60.0                           # one token owns the distribution
+    _check_features(x, vocab=vocab)
