@@ -292,12 +292,19 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
   const int count = s_count;
   const long long out0 = ((long long)row * n_chunks + c) * SB_KMAX;
   if (count <= TOPK_CAND) {
-    for (int a = tid; a < count; a += TOPK_THREADS) {
-      const float v = s_cv[a];
-      const int id = s_ci[a];
+    // rank of candidate a = number of candidates that come before it; four threads share one
+    // candidate (a quarter of the comparisons each, combined by shuffles)
+    for (int a0 = 0; a0 < count; a0 += TOPK_THREADS / 4) {
+      const int a = a0 + (tid >> 2);
+      const bool live = a < count;
+      const float v = live ? s_cv[a] : 0.f;
+      const int id = live ? s_ci[a] : 0;
       int r = 0;
-      for (int b2 = 0; b2 < count; ++b2) r += ranks_before(s_cv[b2], s_ci[b2], v, id) ? 1 : 0;
-      if (r < SB_KMAX) { part_val[out0 + r] = v; part_idx[out0 + r] = id; }
+      if (live)
+        for (int b2 = tid & 3; b2 < count; b2 += 4) r += ranks_before(s_cv[b2], s_ci[b2], v, id) ? 1 : 0;
+      r += __shfl_xor_sync(0xffffffffu, r, 1);
+      r += __shfl_xor_sync(0xffffffffu, r, 2);
+      if (live && (tid & 3) == 0 && r < SB_KMAX) { part_val[out0 + r] = v; part_idx[out0 + r] = id; }
     }
     if (tid < SB_KMAX && tid >= count) { part_val[out0 + tid] = -INFINITY; part_idx[out0 + tid] = kNoId; }
     return;
@@ -597,7 +604,8 @@ __global__ void __launch_bounds__(256) rank_features_finish_kernel(int n_rows, i
 }
 
 static int topk_chunks(int n_rows, int vocab) {
-  int nc = ceil_div(2 * 148, n_rows > 0 ? n_rows : 1);
+  // two CTAs of the partial kernels are resident per SM: keep rows * chunks within one wave
+  int nc = (2 * 148) / (n_rows > 0 ? n_rows : 1);
   const int max_nc = ceil_div(vocab, 2048);
   if (nc > max_nc) nc = max_nc;
   const int reg_nc = ceil_div(vocab, TOPK_REG_ELEMS);  // chunks that fit the register-resident kernel
