@@ -517,10 +517,25 @@ static SplitPlan choose_splits(const sb_tree_batch* tb, int num_splits, AttnImpl
     return plan_for(s, base * s > 2LL * sms);
   }
   if (base > sms) {
-    int s = impl == IMPL_TC ? max_blocks / 8 : max_blocks / 16;
-    if (s > 16) s = 16;
-    if (s < 1) s = 1;
-    return plan_for(s, true);
+    if (impl != IMPL_TC) {
+      int s = max_blocks / 16;
+      if (s > 16) s = 16;
+      if (s < 1) s = 1;
+      return plan_for(s, true);
+    }
+    // More tiles than SMs: CTAs run in waves, and every CTA pays a fixed start-up and merge cost
+    // worth about five blocks.  Take the chunk count with the fewest waves x (blocks + fixed cost).
+    int best = 1;
+    long long best_cost = 0;
+    for (int s = 1; s <= 8 && s <= max_blocks; ++s) {
+      const long long waves = (base * s + sms - 1) / sms;
+      const long long cost = waves * (ceil_div(max_blocks, s) + 5 + (s > 1 ? 1 : 0));
+      if (s == 1 || cost < best_cost) {
+        best = s;
+        best_cost = cost;
+      }
+    }
+    return plan_for(best, true);
   }
   int s = (int)(sms / base);
   if (s > max_blocks) s = max_blocks;

@@ -94,19 +94,16 @@ __device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thr
 __device__ inline void tc_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate, issued by one thread.
-__device__ inline void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
+// Shared-memory matrix descriptor, 128-byte swizzle: start address (bits 0-13), leading (16-29) and
+// stride (32-45) byte offsets, all in 16-byte units, descriptor version 1 (bit 46), layout type 2
+// (bits 61-63) -- kept as two 32-bit halves.  Only the low half depends on the address, and a byte
+// offset inside the tile is added to it as offset >> 4 (shared memory addresses stay below 2^18,
+// so the 14-bit field cannot overflow): the issuing thread forms each operand with one add.
+__device__ inline uint32_t tc_desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr >> 4) & 0x3FFF) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
 }
-// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading / stride byte offsets
-// (all in 16-byte units), descriptor version 1, layout type 2.
-__device__ inline uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16) |
-         ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+__device__ inline uint32_t tc_desc_hi(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFF) | (1u << 14) | (2u << 29);
 }
 // Instruction descriptor: fp32 accumulator, bf16 A and B, N>>3 at bit 17, M>>4 at bit 24,
 // bit 16 = B is MN-major.
@@ -192,12 +189,25 @@ __device__ inline void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
         : "r"(taddr + 32 * h));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]: A is read from tensor memory (row = lane, bf16 pairs along columns).
-__device__ inline void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A * B, bf16 inputs, fp32 accumulate, issued by one thread; the shared memory
+// descriptors are given as (low, high) halves.  First form: A and B in shared memory.  Second form:
+// A is read from tensor memory (row = lane, bf16 pairs along columns).
+__device__ inline void tc_mma_h(uint32_t d_tmem, uint32_t alo, uint32_t blo, uint32_t hi, uint32_t idesc,
+                                uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 ad, {%1, %3};\n\tmov.b64 bd, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %4, p;\n\t}\n" ::"r"(d_tmem),
+      "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ inline void tc_mma_ts_h(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, uint32_t hi, uint32_t idesc,
+                                   uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 bd, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(blo), "r"(hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ inline void cp_async_16_tc(uint32_t smem_dst, const void* gmem_src, int src_bytes) {
@@ -298,23 +308,34 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const uint32_t tmem_o = tmem + 2 * TC_BN;
   const uint32_t tmem_p = tmem + 3 * TC_BN;
 
-  // One TMA box per page piece of a block: box_rows keys x 64 columns, per 64-column half.
-  auto issue_block = [&](int j, const CUtensorMap* map, uint32_t stage_addr, uint64_t* bar) {
+  // One TMA box per page piece of a block: box_rows keys x 64 columns, per 64-column half.  The
+  // page ids of a block are looked up separately (page sizes are powers of two >= 16: at most 8
+  // pieces), so that a loader can have them in registers before the stage it waits for is free.
+  constexpr int MAX_PIECES = TC_BN / 16;
+  auto lookup_pages = [&](int j, int (&pg)[MAX_PIECES]) {
+    if (p.tb.page_size == 0) return;
+    const int nj = min(TC_BN, chunk_keys - j * TC_BN);
+    const int k0 = key_begin + j * TC_BN;
+    const int pieces = ceil_div(nj, box_rows);
+#pragma unroll
+    for (int i = 0; i < MAX_PIECES; ++i)
+      if (i < pieces) pg[i] = p.tb.page_table[(long long)b * p.tb.max_pages + (k0 + i * box_rows) / p.tb.page_size];
+  };
+  auto issue_pieces = [&](int j, const int (&pg)[MAX_PIECES], const CUtensorMap* map, uint32_t stage_addr,
+                          uint64_t* bar) {
     const int nj = min(TC_BN, chunk_keys - j * TC_BN);
     const int k0 = key_begin + j * TC_BN;
     const int pieces = ceil_div(nj, box_rows);
     mbar_expect_tx(bar, (uint32_t)(pieces * box_rows * D * 2));
-    for (int i = 0; i < pieces; ++i) {
+#pragma unroll
+    for (int i = 0; i < MAX_PIECES; ++i) {
+      if (i >= pieces) break;
       const int key = k0 + i * box_rows;
-      int c2, c3;
-      if (p.tb.page_size == 0) {
-        c2 = key;
-        c3 = b;
-      } else {
-        const int lp = key / p.tb.page_size;
-        int page = p.tb.page_table[(long long)b * p.tb.max_pages + lp];
+      int c2 = key, c3 = b;
+      if (p.tb.page_size != 0) {
+        int page = pg[i];
         if (page < 0 || page >= p.tb.num_pages) page = 0;  // reported by the designated CTA
-        c2 = key - lp * p.tb.page_size;
+        c2 = key & (p.tb.page_size - 1);
         c3 = page;
       }
 #pragma unroll
@@ -322,6 +343,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
         tma_load_4d(stage_addr + h * (TC_BN * 128) + i * box_rows * 128, map, h * 64, g, c2, c3, bar);
     }
   };
+  auto issue_block = [&](int j, const CUtensorMap* map, uint32_t stage_addr, uint64_t* bar) {
+    int pg[MAX_PIECES];
+    lookup_pages(j, pg);
+    issue_pieces(j, pg, map, stage_addr, bar);
+  };
+  // A V block whose rows reach past the end of the sequence holds stale cache rows there; they
+  // meet zero probabilities, but must not be NaN or infinite: such a block (only the last one of
+  // the sequence can be) lands on a barrier of its own and is cleaned before the MMA may read it.
+  // Every other V block completes the barrier the MMA warp waits on directly.
+  auto v_needs_fix = [&](int j) { return L - (key_begin + j * TC_BN) < min(TC_BN, chunk_keys - j * TC_BN); };
+  auto v_bar = [&](int j) { return &s_bar[(v_needs_fix(j) ? V_TMA0 : V_FULL0) + (j & 1)]; };
   // The first loads go out before anything else: they only need the sequence's lengths.  Only
   // the K side (Q, K blocks 0 and 1) is requested at once; the V blocks, needed a softmax later,
   // follow when K block 0 has landed, so they do not queue in front of it in the memory system.
@@ -475,17 +507,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   } else if (warp == TC_MMA_WARP) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && nb > 0) {
-      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+      // Every operand descriptor is a constant plus a small offset: the halves are formed once, so
+      // that each MMA costs the issuing thread a couple of integer adds.
+      const uint32_t hi = tc_desc_hi(1024);
+      const uint32_t q_lo = tc_desc_lo(smem_u32(sQ), 16), k_lo = tc_desc_lo(smem_u32(sK), 16);
+      const uint32_t v_lo = tc_desc_lo(smem_u32(sV), TC_BN * 128);
+      const uint32_t idesc_s_full = tc_idesc(TC_BM, TC_BN, 0), idesc_pv = tc_idesc(TC_BM, D, 1);
       bool ok = true;
       auto issue_s = [&](int j) {
         const int nj = min(TC_BN, chunk_keys - j * TC_BN);
-        const uint32_t idesc = tc_idesc(TC_BM, nj, 0);
-        const uint32_t kb = k_addr + (j & 1) * TILE_BYTES;
+        const uint32_t idesc = nj == TC_BN ? idesc_s_full : tc_idesc(TC_BM, nj, 0);
+        const uint32_t kb = k_lo + (j & 1) * (TILE_BYTES >> 4);
+        const uint32_t d = tmem + (j & 1) * TC_BN;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t koff = (ks >> 2) * (TC_BM * 128) + (ks & 3) * 32;
-          tc_mma(tmem + (j & 1) * TC_BN, tc_smem_desc(q_addr + koff, 16, 1024), tc_smem_desc(kb + koff, 16, 1024), idesc,
-                 ks > 0);
+          const uint32_t koff = ((ks >> 2) * (TC_BM * 128) + (ks & 3) * 32) >> 4;
+          tc_mma_h(d, q_lo + koff, kb + koff, hi, idesc, ks > 0);
         }
         tc_commit(&s_bar[S_FULL0 + (j & 1)]);
         tc_commit(&s_bar[K_EMPTY0 + (j & 1)]);
@@ -510,11 +547,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
         if (!ok) break;
         tc_fence_after();
         const int nj = min(TC_BN, chunk_keys - j * TC_BN);
-        const uint32_t idesc = tc_idesc(TC_BM, D, 1);
-        const uint32_t vb = v_addr + (j & 1) * TILE_BYTES;
-        for (int ks = 0; ks < nj / 16; ++ks)  // 16 keys = 8 packed columns of P per step
-          tc_mma_ts(tmem_o, tmem_p + (j & 1) * 64 + ks * 8, tc_smem_desc(vb + ks * 2048, TC_BN * 128, 1024), idesc,
-                    (j > 0 || ks > 0) ? 1u : 0u);
+        const uint32_t vb = v_lo + (j & 1) * (TILE_BYTES >> 4);
+        const uint32_t pb = tmem_p + (j & 1) * 64;
+        // 16 keys = 8 packed columns of P = 2048 bytes of the V stage per step
+        if (nj == TC_BN) {
+#pragma unroll
+          for (int ks = 0; ks < TC_BN / 16; ++ks)
+            tc_mma_ts_h(tmem_o, pb + ks * 8, vb + ks * (2048 >> 4), hi, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+        } else {
+          for (int ks = 0; ks < nj / 16; ++ks)
+            tc_mma_ts_h(tmem_o, pb + ks * 8, vb + ks * (2048 >> 4), hi, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+        }
         tc_commit(&s_bar[PV_FULL]);
         tc_commit(&s_bar[V_EMPTY0 + (j & 1)]);
       }
@@ -524,43 +567,50 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     // ------------------------------------------------------------------ K loader (blocks 2..)
     if (lane == 0) {
       bool ok = true;
+      int pg[MAX_PIECES];
+      if (nb > 2) lookup_pages(2, pg);
       for (int j = 2; j < nb && ok; ++j) {
         ok = mbar_wait(&s_bar[K_EMPTY0 + (j & 1)], ((j >> 1) - 1) & 1, s_abort);
-        if (ok) issue_block(j, &kmap, smem_u32(sK) + (j & 1) * TILE_BYTES, &s_bar[K_FULL0 + (j & 1)]);
+        if (!ok) break;
+        issue_pieces(j, pg, &kmap, smem_u32(sK) + (j & 1) * TILE_BYTES, &s_bar[K_FULL0 + (j & 1)]);
+        if (j + 1 < nb) lookup_pages(j + 1, pg);  // in flight while the next stage is awaited
       }
       if (!ok) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
     }
   } else if (warp == TC_VLOAD_WARP) {
     // ------------------------------------------------------------------ V loader
     bool ok = true;
+    int pg[MAX_PIECES];
     if (nb > 0 && lane == 0) {
       ok = mbar_wait(&s_bar[K_FULL0], 0, s_abort);
       if (ok) {
-        issue_block(0, &vmap, smem_u32(sV), &s_bar[V_TMA0]);
-        if (nb > 1) issue_block(1, &vmap, smem_u32(sV) + TILE_BYTES, &s_bar[V_TMA1]);
+        issue_block(0, &vmap, smem_u32(sV), v_bar(0));
+        if (nb > 1) issue_block(1, &vmap, smem_u32(sV) + TILE_BYTES, v_bar(1));
+        if (nb > 2) lookup_pages(2, pg);
       }
     }
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     for (int j = 0; j < nb && ok; ++j) {
-      ok = mbar_wait(&s_bar[V_TMA0 + (j & 1)], (j >> 1) & 1, s_abort);
-      if (!ok) break;
-      // rows of this block that lie past the end of the sequence: zero them (at most 15)
-      const int nj = min(TC_BN, chunk_keys - j * TC_BN);
-      const int first_bad = L - (key_begin + j * TC_BN);
-      if (first_bad < nj) {
+      if (v_needs_fix(j)) {  // warp-uniform; at most once per sequence, so the barrier's phase is 0
+        ok = mbar_wait(&s_bar[V_TMA0 + (j & 1)], 0, s_abort);
+        if (!ok) break;
+        // rows of this block that lie past the end of the sequence: zero them (at most 15)
+        const int nj = min(TC_BN, chunk_keys - j * TC_BN);
+        const int first_bad = L - (key_begin + j * TC_BN);
         uint8_t* stage = sV + (j & 1) * TILE_BYTES;
         for (int c = lane; c < (nj - first_bad) * CH; c += 32) {
           const int r = first_bad + c / CH, ch = c % CH;
           *reinterpret_cast<uint4*>(stage + sw128_chunk_off(r, ch, TC_BN)) = make_uint4(0, 0, 0, 0);
         }
         fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_bar[V_FULL0 + (j & 1)]);
       }
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&s_bar[V_FULL0 + (j & 1)]);
-        if (j + 2 < nb) {
-          ok = mbar_wait(&s_bar[V_EMPTY0 + (j & 1)], (j >> 1) & 1, s_abort);
-          if (ok) issue_block(j + 2, &vmap, smem_u32(sV) + (j & 1) * TILE_BYTES, &s_bar[V_TMA0 + (j & 1)]);
+      if (lane == 0 && j + 2 < nb) {
+        ok = mbar_wait(&s_bar[V_EMPTY0 + (j & 1)], (j >> 1) & 1, s_abort);
+        if (ok) {
+          issue_pieces(j + 2, pg, &vmap, smem_u32(sV) + (j & 1) * TILE_BYTES, v_bar(j + 2));
+          if (j + 3 < nb) lookup_pages(j + 3, pg);
         }
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;

@@ -1,6 +1,6 @@
 """Times sb_tree_attention on the five benchmark configurations and prints one JSON line each.
 
-    python -m paper_2605_07243_b200.time_configs [--configs 1,2,3,4,5] [--iters 30]
+    python -m paper_2605_07243_b200.time_configs [--configs 1,2,3,4,5] [--iters 30] [--num-splits S]
 
 For every configuration: CUDA-event time per call (a CUDA graph walks buffer sets whose total
 exceeds L2, so K/V come from HBM; median over `iters` replays), algorithmic bytes and flops,
@@ -46,8 +46,10 @@ def _cases(which):
     raise ValueError(which)
 
 
-def time_config(which, iters):
+def time_config(which, iters, num_splits=None):
     case, splits = _cases(which)
+    if num_splits is not None:
+        splits = num_splits
     kv_bytes = case.k.nbytes + case.v.nbytes
     # enough distinct KV copies to exceed L2 (126 MB) between two uses of the same copy
     n_sets = max(2, min(32, int(np.ceil(2 * 134e6 / kv_bytes))))
@@ -99,12 +101,14 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--iters", type=int, default=30)
+    ap.add_argument("--num-splits", type=int, default=None,
+                    help="override the number of KV chunks (0 = the library's choice)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("needs a CUDA device")
     sb.load()
     for c in [int(x) for x in args.configs.split(",")]:
-        print(json.dumps(time_config(c, args.iters)), flush=True)
+        print(json.dumps(time_config(c, args.iters, args.num_splits)), flush=True)
 
 
 if __name__ == "__main__":
