@@ -19,6 +19,32 @@ inline sb_status launch_check() {
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Programmatic dependent launch.  A kernel started with launch_dependent() may begin while its
+// predecessor in the stream is still running; it must execute pdl_wait() before it reads anything
+// the predecessor writes (and always before it ends, so that completion stays transitive along
+// the stream).  The predecessor lets it start early with pdl_release().
+__device__ inline void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ inline void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline sb_status launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t cs, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = cs;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) != cudaSuccess) {
+    cudaGetLastError();
+    return SB_ERR_CUDA;
+  }
+  return launch_check();
+}
+
 // Per-sequence facts every CTA of a sequence derives identically from device data.
 struct SeqInfo {
   int n;       // tree nodes

@@ -69,6 +69,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
   const float* base = scores + (long long)row * row_stride;
   const int begin = c * chunk;
   const int end = min(vocab, begin + chunk);
+  pdl_release();  // the finishing kernel may start its prologue
 
   // pass 1: thread maxima -> threshold tau = 16th largest of them
   const int n_vec = vec_ok ? max(0, (end - begin) / 4) : 0;
@@ -214,6 +215,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
   const float* base = scores + (long long)row * row_stride;
   const int begin = c * chunk;
   const int end = min(vocab, begin + chunk);
+  pdl_release();  // the finishing kernel may start its prologue
   const int n_elems = max(0, end - begin);
   const int n_vec = n_elems / 4;  // whole float4s; up to 3 tail elements are handled by thread 0
   const float4* vb = reinterpret_cast<const float4*>(base + begin);
@@ -397,6 +399,7 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
   }
   const int pre_n0 = *n_nodes;
   const int pre_depth = (pre_row && pre_start >= 0 && pre_start < pre_n0) ? depth[pre_start] : 0;
+  pdl_wait();  // the chunk lists of the scan kernel are complete from here on
   __syncthreads();
   // (1) merge the chunk lists of every row: lane c holds chunk c's sorted list in registers and
   //     pops it by shifting
@@ -534,6 +537,7 @@ __global__ void __launch_bounds__(256) rank_features_finish_kernel(int n_rows, i
                                                                    float* __restrict__ features) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * 8 + warp;
+  pdl_wait();  // the chunk lists and statistics of the scan kernel are complete from here on
   if (r >= n_rows) return;
   float lv[SB_KMAX];
   int li[SB_KMAX];
@@ -656,11 +660,9 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
                                                               part_idx, nullptr);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
-  expand_finish_kernel<<<1, FINISH_THREADS, 0, cs>>>(n_rows, nc, part_val, part_idx, block_k, bucket,
-                                                     make_int4(bmap[0], bmap[1], bmap[2], bmap[3]),
-                                                     start_parent, node_budget, vocab, n_nodes, tok, parent,
-                                                     depth, node_row, node_rank, topk_tok, topk_val, status);
-  return launch_check();
+  return launch_dependent(expand_finish_kernel, dim3(1), dim3(FINISH_THREADS), cs, n_rows, nc, part_val, part_idx,
+                          block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
+                          vocab, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val, status);
 }
 
 extern "C" size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab) {
@@ -694,7 +696,6 @@ extern "C" sb_status sb_rank_features(const float* scores, int64_t row_stride, i
                                                              part_idx, part_stats);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
-  rank_features_finish_kernel<<<ceil_div(n_rows, 8), 256, 0, cs>>>(n_rows, nc, vocab, part_val, part_idx, part_stats,
-                                                                   features);
-  return launch_check();
+  return launch_dependent(rank_features_finish_kernel, dim3(ceil_div(n_rows, 8)), dim3(256), cs, n_rows, nc, vocab,
+                          part_val, part_idx, part_stats, features);
 }

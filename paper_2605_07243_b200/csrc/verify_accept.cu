@@ -49,46 +49,41 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) row_argmax_kernel(const T* __r
   const T* base = logits + (long long)row * row_stride;
   const int begin = c * chunk;
   const int end = min(vocab, begin + chunk);
+  pdl_release();  // the path kernel may start its prologue
   Best best = {-INFINITY, 0x7fffffff};
   if (vec_ok) {
     // chunk is a multiple of VEC and rows are 16-byte aligned
     const int n_vec = max(0, (end - begin) / VEC);
     const uint4* vb = reinterpret_cast<const uint4*>(base + begin);
-    constexpr int UNROLL = 4;  // independent 16-byte loads in flight per thread
-    int t = threadIdx.x;
-    for (; t + (UNROLL - 1) * ARGMAX_THREADS < n_vec; t += UNROLL * ARGMAX_THREADS) {
+    // All of a thread's loads of one sweep are issued before any is used: a chunk of up to
+    // UNROLL * 256 vectors (32 KB) costs one trip to memory.
+    constexpr int UNROLL = 8;
+    for (int t0 = threadIdx.x; t0 < n_vec; t0 += UNROLL * ARGMAX_THREADS) {
       uint4 raw[UNROLL];
 #pragma unroll
-      for (int q = 0; q < UNROLL; ++q) raw[q] = __ldg(vb + t + q * ARGMAX_THREADS);
+      for (int q = 0; q < UNROLL; ++q)
+        if (t0 + q * ARGMAX_THREADS < n_vec) raw[q] = __ldg(vb + t0 + q * ARGMAX_THREADS);
 #pragma unroll
       for (int q = 0; q < UNROLL; ++q) {
-        const T* e = reinterpret_cast<const T*>(&raw[q]);
+        if (t0 + q * ARGMAX_THREADS < n_vec) {
+          const T* e = reinterpret_cast<const T*>(&raw[q]);
 #pragma unroll
-        for (int u = 0; u < VEC; ++u) {
-          const float x = logit_to_float<T>(e[u]);
-          const int id = begin + (t + q * ARGMAX_THREADS) * VEC + u;
-          if (x > best.v) { best.v = x; best.i = id; }  // ids ascend inside a thread: strict keeps the first
+          for (int u = 0; u < VEC; ++u) {
+            const float x = logit_to_float<T>(e[u]);
+            const int id = begin + (t0 + q * ARGMAX_THREADS) * VEC + u;
+            if (x > best.v) { best.v = x; best.i = id; }  // ids ascend inside a thread: strict keeps the first
+          }
         }
-      }
-    }
-    for (; t < n_vec; t += ARGMAX_THREADS) {
-      const uint4 raw = __ldg(vb + t);
-      const T* e = reinterpret_cast<const T*>(&raw);
-#pragma unroll
-      for (int u = 0; u < VEC; ++u) {
-        const float x = logit_to_float<T>(e[u]);
-        const int id = begin + t * VEC + u;
-        if (better(x, id, best.v, best.i)) { best.v = x; best.i = id; }
       }
     }
     for (int id = begin + n_vec * VEC + threadIdx.x; id < end; id += ARGMAX_THREADS) {
       const float x = logit_to_float<T>(base[id]);
-      if (better(x, id, best.v, best.i)) { best.v = x; best.i = id; }
+      if (x > best.v) { best.v = x; best.i = id; }
     }
   } else {
     for (int id = begin + threadIdx.x; id < end; id += ARGMAX_THREADS) {
       const float x = logit_to_float<T>(base[id]);
-      if (better(x, id, best.v, best.i)) { best.v = x; best.i = id; }
+      if (x > best.v) { best.v = x; best.i = id; }
     }
   }
   best = warp_best(best);
@@ -101,6 +96,9 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) row_argmax_kernel(const T* __r
     if (threadIdx.x < ARGMAX_THREADS / 32) { x.v = s_v[threadIdx.x]; x.i = s_i[threadIdx.x]; }
     x = warp_best(x);
     if (threadIdx.x == 0) {
+      // Every thread keeps the first of its maxima by strict compares over ascending ids, so a chunk
+      // that holds nothing above -inf (NaN counts as -inf) records no id at all: its first element wins.
+      if (x.i == 0x7fffffff && begin < end) x.i = begin;
       part_val[(long long)row * n_chunks + c] = x.v;
       part_idx[(long long)row * n_chunks + c] = x.i;
     }
@@ -127,6 +125,7 @@ __global__ void __launch_bounds__(SB_MAX_NODES) accept_kernel(int n_chunks, cons
   for (int t = i; t <= max_depth; t += blockDim.x) { path[t] = -1; otok[t] = -1; }
   if (i == 0) { s_bad = 0; s_best = -1; accept_len[b] = 0; bonus[b] = -1; }
   __syncthreads();
+  pdl_wait();  // the chunk partials of the scan kernel are complete from here on
   if (n < 1 || n > SB_MAX_NODES || o < 0 || (long long)o + n > total_nodes) {
     if (i == 0) status[b] = SB_ERR_INVALID_TREE;
     return;
@@ -230,10 +229,9 @@ extern "C" sb_status sb_verify_accept(const void* logits, sb_dtype dtype, int64_
                                                               vocab, chunk, nc, vec_ok, part_val, part_idx);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
-  accept_kernel<<<batch, SB_MAX_NODES, 0, cs>>>(nc, part_val, part_idx, node_offsets, parent, tok,
-                                                total_nodes, max_depth, amax, accept_len, path_nodes,
-                                                out_tokens, bonus, status);
-  return launch_check();
+  return launch_dependent(accept_kernel, dim3(batch), dim3(SB_MAX_NODES), cs, nc, part_val, part_idx, node_offsets,
+                          parent, tok, total_nodes, max_depth, amax, accept_len, path_nodes, out_tokens, bonus,
+                          status);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -294,8 +292,7 @@ extern "C" sb_status sb_verify_accept_static(const void* logits, sb_dtype dtype,
                                                               vocab, chunk, nc, vec_ok, part_val, part_idx);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
-  accept_kernel<<<batch, SB_MAX_NODES, 0, cs>>>(nc, part_val, part_idx, node_offsets, parent, tok,
-                                                total_nodes, max_depth, amax, accept_len, path_nodes,
-                                                out_tokens, bonus, status);
-  return launch_check();
+  return launch_dependent(accept_kernel, dim3(batch), dim3(SB_MAX_NODES), cs, nc, part_val, part_idx, node_offsets,
+                          parent, tok, total_nodes, max_depth, amax, accept_len, path_nodes, out_tokens, bonus,
+                          status);
 }

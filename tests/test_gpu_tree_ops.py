@@ -94,6 +94,30 @@ def test_accept_row_stride_padding_nan_inf_and_ties():
     assert got["amax"][3] == 0 and got["amax"][5] == 77 and got["amax"][6] == 0 and got["amax"][7] == 0
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_accept_degenerate_rows_large_vocab(dtype):
+    """Rows with nothing above -inf, over a vocabulary that spans many chunks and many vectors per thread."""
+    rng = W.rng_for(63)
+    vocab = 128256
+    parents = [W.chain_tree(8)]
+    x = np.round(rng.standard_normal((8, vocab), dtype=np.float32) * 2)
+    x[1, :] = -np.inf                        # -> id 0
+    x[2, :] = np.nan                         # NaN reads as -inf -> id 0
+    x[3, :] = -np.inf
+    x[3, vocab - 1] = -7.0                   # the only finite value sits in the last chunk's tail
+    x[4, :] = -np.inf
+    x[4, 40000:40003] = np.nan               # still nothing above -inf -> id 0
+    x[5, :] = 3.0                            # all equal -> id 0
+    x[6, :] = -np.inf
+    x[6, 70001] = -np.inf
+    x[6, 70002] = -1e30
+    logits = W.f32_to_bf16_bits(x) if dtype == "bf16" else x
+    case = W.VerifyCase(logits, rng.integers(0, vocab, 8).astype(np.int32), np.asarray([0, 8], np.int32),
+                        parents[0], 8, None, None, None)
+    got = _check_accept(case)
+    np.testing.assert_array_equal(got["amax"][1:7], [0, 0, vocab - 1, 0, 0, 70002])
+
+
 def test_accept_depth_cut_duplicates_and_invalid_trees():
     rng = W.rng_for(62)
     # duplicate sibling tokens and a tiny alphabet -> many equally long accepted paths
