@@ -12,6 +12,7 @@ from .oracle import (  # noqa: F401
     row_topk,
     rank_features,
     verify_accept,
+    verifier_signal,
     accept_from_amax,
     kv_compact,
     tree_expand,

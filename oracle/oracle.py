@@ -139,6 +139,24 @@ def rank_features(scores, vocab=None):
     return feats
 
 
+def verifier_signal(scores, node_offsets, child_row, path_nodes, accept_len, bonus, max_depth, signal=None,
+                    vocab=None):
+    """-> dict(r_prob f64 [B], signal f64 [B] (= signal in + 1 - r), status int32 [B])."""
+    scores = np.ascontiguousarray(scores, np.float32)
+    n_rows, stride = scores.shape
+    vocab = stride if vocab is None else vocab
+    node_offsets, child_row = _i32(node_offsets), _i32(child_row)
+    path_nodes, accept_len, bonus = _i32(path_nodes), _i32(accept_len), _i32(bonus)
+    batch = node_offsets.shape[0] - 1
+    r_prob = np.zeros(batch, np.float64)
+    sig = np.zeros(batch, np.float64) if signal is None else np.array(signal, np.float64)
+    status = np.zeros(batch, np.int32)
+    _load().sbo_verifier_signal(_p(scores), C.c_int64(stride), C.c_int(n_rows), C.c_int(vocab), C.c_int(batch),
+                                _p(node_offsets), _p(child_row), _p(path_nodes), _p(accept_len), _p(bonus),
+                                C.c_int(max_depth), _p(r_prob), _p(sig), _p(status))
+    return dict(r_prob=r_prob, signal=sig, status=status)
+
+
 def verify_accept(logits, node_offsets, parent, tok, max_depth, vocab=None):
     """-> dict(amax, accept_len, path_nodes, out_tokens, bonus, status)."""
     logits, dt = _logits_arg(logits)

@@ -18,6 +18,8 @@
  *                         trees; planted paths; the case-study tree (4 accepted + bonus).
  *   sbo_kv_compact      : numpy fancy-index gather; attention over the compacted cache.
  *   sbo_rank_features   : scipy log_softmax / entropy; closed forms (uniform row, one dominant token).
+ *   sbo_verifier_signal : scipy softmax; closed forms (flat row, one raised token); probabilities of
+ *                         all tokens of a row sum to one; the sum over iterations of a query.
  *   sbo_tree_expand     : hand-derived trees for the two printed branching maps; chain special
  *                         case; structural invariants.  The attach point of siblings, the cut
  *                         order at the node budget and the treatment of b = 0 are readings of
@@ -490,6 +492,58 @@ void sbo_rank_features(const float* scores, int64_t row_stride, int n_rows, int 
     f[13] = exp(e[0].val - log_z);
     f[14] = entropy;
     free(e);
+  }
+}
+
+/* ---- verifier-derived update signal (Sec. 3.4, the equation for s; Alg. 2 line 2) ------------- */
+
+/*
+ * s = sum over rejected positions of (1 - r), r = the drafter's probability of the token the
+ * target chose at that position.  One verify iteration rejects at most one position per sequence:
+ * the one right after the last accepted node `best` = path_nodes[b][accept_len[b]], where the
+ * target chose bonus[b].  child_row[node] names the row of `scores` (drafter logits) that
+ * predicted the token following `node`, or -1 when nothing was drafted there (then nothing was
+ * rejected: r_prob = -1 and the sum is left alone).
+ *   r = softmax(scores[row])[bonus] by the plain definition in fp64 (NaN scores count as -inf; a
+ *   row without a finite score is flat; a token outside [0, vocab) has probability 0);
+ *   r_prob[b] = r;  signal[b] += 1 - r   (signal is in/out: the caller zeroes it per query).
+ * status[b] = 5 (and r_prob = -1, signal untouched) when accept_len, the path node or the row
+ * index is out of range.
+ */
+void sbo_verifier_signal(const float* scores, int64_t row_stride, int n_rows, int vocab, int batch,
+                         const int32_t* node_offsets, const int32_t* child_row, const int32_t* path_nodes,
+                         const int32_t* accept_len, const int32_t* bonus, int max_depth, double* r_prob,
+                         double* signal, int32_t* status) {
+  for (int b = 0; b < batch; ++b) {
+    const int o = node_offsets[b], n = node_offsets[b + 1] - o;
+    const int a = accept_len[b];
+    status[b] = 0;
+    r_prob[b] = -1.0;
+    if (a < 0 || a > max_depth) { status[b] = 5; continue; }
+    const int best = path_nodes[(int64_t)b * (max_depth + 1) + a];
+    if (best < 0 || best >= n) { status[b] = 5; continue; }
+    const int row = child_row[o + best];
+    if (row < 0) continue; /* nothing drafted after the last accepted node */
+    if (row >= n_rows) { status[b] = 5; continue; }
+    const float* x = scores + (int64_t)row * row_stride;
+    const int t = bonus[b];
+    double m = -INFINITY;
+    for (int v = 0; v < vocab; ++v) {
+      const double xv = score_of((double)x[v]);
+      if (xv > m) m = xv;
+    }
+    double r;
+    if (t < 0 || t >= vocab) {
+      r = 0.0;
+    } else if (m == -INFINITY) {
+      r = 1.0 / (double)vocab;
+    } else {
+      double z = 0.0;
+      for (int v = 0; v < vocab; ++v) z += exp(score_of((double)x[v]) - m);
+      r = exp(score_of((double)x[t]) - m) / z;
+    }
+    r_prob[b] = r;
+    signal[b] += 1.0 - r;
   }
 }
 

@@ -379,3 +379,80 @@ def test_rank_features_match_scipy_and_closed_forms():
     # fewer than ten / five tokens
     s = oracle.rank_features(np.asarray([[1.0, 3.0, 2.0]], np.float32))[0]
     assert np.isneginf(s[3:10]).all() and s[10] == 1.0 and s[11] == 2.0 and np.isposinf(s[12])
+
+
+# ---- verifier-derived update signal s = sum (1 - r) (Sec. 3.4; Alg. 2 line 2) ---------------------------------
+
+def _signal_inputs(best_nodes, bonus, child_row, n_nodes, max_depth=4):
+    """One sequence per entry; the accepted path is only needed at its last node."""
+    B = len(best_nodes)
+    node_offsets = np.arange(B + 1, dtype=np.int32) * n_nodes
+    path = np.full((B, max_depth + 1), -1, np.int32)
+    accept_len = np.zeros(B, np.int32)
+    for b, node in enumerate(best_nodes):
+        accept_len[b] = b % (max_depth + 1)
+        path[b, accept_len[b]] = node
+    return dict(node_offsets=node_offsets, child_row=np.tile(np.asarray(child_row, np.int32), B), path_nodes=path,
+                accept_len=accept_len, bonus=np.asarray(bonus, np.int32), max_depth=max_depth)
+
+
+def test_verifier_signal_matches_scipy_softmax_and_closed_forms():
+    from scipy.special import softmax
+    rng = W.rng_for(34)
+    V, R = 777, 6
+    x = (rng.standard_normal((R, V), dtype=np.float32) * 3).astype(np.float32)
+    x[2, ::5] = np.nan                           # NaN counts as -inf
+    x[3, 10:] = -np.inf
+    child_row = [4, 2, -1, 0, 3, 5, 1]           # node -> drafter row that predicted its successor
+    best = [0, 1, 3, 4, 5, 6, 2]
+    bonus = [5, 10, 700, 3, V - 1, 0, 9]
+    got = oracle.verifier_signal(x, **_signal_inputs(best, bonus, child_row, 7))
+    p = softmax(np.where(np.isnan(x), -np.inf, x).astype(np.float64), axis=1)   # library routine
+    want_r = np.asarray([p[child_row[n], t] if child_row[n] >= 0 else -1.0 for n, t in zip(best, bonus)])
+    np.testing.assert_allclose(got["r_prob"], want_r, rtol=1e-12, atol=1e-300)
+    np.testing.assert_allclose(got["signal"], np.where(want_r >= 0, 1.0 - want_r, 0.0), rtol=1e-12)
+    assert (got["status"] == 0).all()
+    assert got["r_prob"][6] == -1.0 and got["signal"][6] == 0.0    # nothing drafted after node 2: nothing rejected
+    assert got["r_prob"][1] == 0.0                                  # token 10 sits on a NaN score of row 2
+
+    # closed forms: a flat row gives r = 1/V; one token raised by c gives e^c / (e^c + V - 1)
+    flat = np.full((1, V), -1.25, np.float32)
+    g = oracle.verifier_signal(flat, **_signal_inputs([0], [123], [0], 1))
+    np.testing.assert_allclose(g["signal"], 1.0 - 1.0 / V, rtol=1e-15)
+    c = 6.5
+    raised = np.zeros((1, V), np.float32)
+    raised[0, 40] = c
+    g = oracle.verifier_signal(raised, **_signal_inputs([0, 0], [40, 41], [0], 1))
+    np.testing.assert_allclose(g["r_prob"], [np.exp(c) / (np.exp(c) + V - 1), 1.0 / (np.exp(c) + V - 1)], rtol=1e-13)
+    # a row with no finite score is read as flat; a token outside the vocabulary has probability 0
+    dead = np.full((1, V), -np.inf, np.float32)
+    assert oracle.verifier_signal(dead, **_signal_inputs([0], [7], [0], 1))["r_prob"][0] == 1.0 / V
+    out = oracle.verifier_signal(flat, **_signal_inputs([0, 0], [V, -1], [0], 1))
+    assert (out["r_prob"] == 0.0).all() and (out["signal"] == 1.0).all()
+
+
+def test_verifier_signal_invariants_accumulation_and_bounds():
+    rng = W.rng_for(35)
+    V = 50
+    x = (rng.standard_normal((3, V), dtype=np.float32) * 2).astype(np.float32)
+    # the probabilities of all tokens of one row sum to one
+    r = oracle.verifier_signal(x, **_signal_inputs([0] * V, list(range(V)), [1], 1))["r_prob"]
+    np.testing.assert_allclose(r.sum(), 1.0, rtol=1e-14)
+    # adding a constant to a row changes nothing (values chosen exactly representable)
+    y = np.round(x * 8) / 8
+    a = oracle.verifier_signal(y, **_signal_inputs([0, 0], [3, 4], [2], 1))
+    b = oracle.verifier_signal(y + np.float32(16.0), **_signal_inputs([0, 0], [3, 4], [2], 1))
+    np.testing.assert_allclose(a["r_prob"], b["r_prob"], rtol=1e-13)
+    # the query-level signal is the sum over iterations: feed the running value back in
+    args = _signal_inputs([0, 0], [3, 4], [2], 1)
+    s1 = oracle.verifier_signal(x, **args)
+    s2 = oracle.verifier_signal(x, signal=s1["signal"], **_signal_inputs([0, 0], [5, 6], [0], 1))
+    np.testing.assert_allclose(s2["signal"], (1 - s1["r_prob"]) + (1 - s2["r_prob"]), rtol=1e-14)
+    assert (0 <= s1["signal"]).all() and (s1["signal"] <= 1).all()
+    # out-of-range accept_len / path node / row are reported per sequence and change nothing
+    bad = _signal_inputs([0, 0, 0], [1, 1, 1], [7], 1)      # row 7 of a 3-row matrix
+    bad["accept_len"][1] = 9
+    g = oracle.verifier_signal(x, signal=[0.5, 0.5, 0.5], **bad)
+    assert (g["status"] == 5).all() and (g["signal"] == 0.5).all() and (g["r_prob"] == -1).all()
+    bad = _signal_inputs([4], [1], [0], 1)                  # path node 4 of a 1-node tree
+    assert oracle.verifier_signal(x, **bad)["status"][0] == 5
