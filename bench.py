@@ -234,6 +234,8 @@ def run_ours(args):
         g_compact = capture(torch, step.run_compact)
         step.run_rank_features()
         g_features = capture(torch, step.run_rank_features)
+        step.run_signal()
+        g_signal = capture(torch, step.run_signal)
 
         for _ in range(max(args.warmup, 3)):
             g_step.replay()
@@ -262,7 +264,7 @@ def run_ours(args):
         clocks = sampler.stop()
         parts_ms = {}
         for name, g in (("expand", g_expand), ("accept", g_accept), ("compact", g_compact),
-                        ("rank_features_not_in_step", g_features)):
+                        ("rank_features_not_in_step", g_features), ("verifier_signal_not_in_step", g_signal)):
             for _ in range(3):
                 g.replay()
             parts_ms[name] = time_graph(torch, g, 20, False) / 20

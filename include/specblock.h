@@ -11,6 +11,7 @@
  *   sb_tree_attention  tree-masked attention over prefix KV + ancestors (Sec. 3.1, App. A.2, Alg. 1 "verify")
  *   sb_tree_expand     per-row top-k + bucket-driven branching          (Sec. 3.2, App. A.5, Alg. 1 "attach")
  *   sb_rank_features   15-dim summary of each draft distribution        (Sec. 3.2, App. B)
+ *   sb_verifier_signal verifier-derived update signal s = sum (1 - r)   (Sec. 3.4, Alg. 2)
  *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
  *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
  *
@@ -184,6 +185,32 @@ size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab);
 sb_status sb_rank_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
                            float* features, void* workspace, size_t workspace_bytes, void* stream);
 size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
+
+/*
+ * sb_verifier_signal -- one iteration's term of the verifier-derived update signal
+ * s = sum over rejected positions of (1 - r), r = the drafter's probability of the token the
+ * target chose there (Sec. 3.4 "Verifier-derived update signal"; Alg. 2 line 2).
+ *
+ *   A verify iteration rejects at most one position per sequence: the one right after the last
+ *   accepted node best = path_nodes[b][accept_len[b]], where the target chose bonus[b] (all three
+ *   as sb_verify_accept leaves them on the device).
+ *   child_row int32 [total_nodes]: for every tree node the row of `scores` (drafter logits, fp32
+ *       [n_rows][row_stride >= vocab]) that predicted the token following it, or -1 when nothing
+ *       was drafted after it.
+ *   r = softmax(scores[child_row[best]])[bonus]; NaN scores read as -inf, a row without a finite
+ *       score as flat, a token outside [0, vocab) as probability 0 (not in the drafter's vocabulary).
+ *   r_prob fp32 [batch]: out, r, or -1 when nothing was rejected (child_row = -1) or on an error.
+ *   signal fp32 [batch]: in/out, signal[b] += 1 - r; the caller zeroes it at the start of a query
+ *       and reads the query-level s after its last iteration.
+ *   status int32 [batch]: SB_OK, or SB_ERR_BOUNDS when accept_len, the path node or the row index
+ *       is out of range (r_prob = -1, signal untouched).
+ *   One pass over one score row per sequence (vocab * 4 bytes); fp32 sums.  No workspace.
+ */
+sb_status sb_verifier_signal(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                             int32_t batch, int32_t total_nodes, const int32_t* node_offsets,
+                             const int32_t* child_row, const int32_t* path_nodes, const int32_t* accept_len,
+                             const int32_t* bonus, int32_t max_depth, float* r_prob, float* signal,
+                             int32_t* status, void* stream);
 
 /*
  * sb_verify_accept -- greedy (temperature 0) verification (App. A.5 "the longest accepted

@@ -65,7 +65,7 @@ def load(build_if_missing: bool = True):
                  "sb_verify_accept_workspace_bytes", "sb_rank_features_workspace_bytes"):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
-                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features"):
+                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -74,7 +74,8 @@ def load(build_if_missing: bool = True):
 EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspace_bytes",
             "sb_tree_expand", "sb_tree_expand_workspace_bytes", "sb_verify_accept",
             "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
-            "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_status_string", "sb_version",
+            "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_verifier_signal", "sb_status_string",
+            "sb_version",
             "sb_kernel_launch_count")
 
 
@@ -248,6 +249,26 @@ def sb_rank_features(scores, *, vocab=None, features=None, workspace=None):
                                  _stream())
     _check(rc, "sb_rank_features")
     return features
+
+
+def sb_verifier_signal(scores, node_offsets, child_row, path_nodes, accept_len, bonus, max_depth, signal, *,
+                       vocab=None, r_prob=None, status=None):
+    """One iteration's term of s = sum (1 - r): signal fp32 [B] is updated in place.
+    -> dict(r_prob, signal, status)."""
+    n_rows, stride = scores.shape
+    vocab = stride if vocab is None else vocab
+    batch = node_offsets.numel() - 1
+    dev = scores.device
+    r_prob = torch.empty(batch, dtype=torch.float32, device=dev) if r_prob is None else r_prob
+    status = torch.empty(batch, dtype=torch.int32, device=dev) if status is None else status
+    rc = load().sb_verifier_signal(
+        _ptr(scores, torch.float32), C.c_int64(stride), C.c_int32(n_rows), C.c_int32(vocab), C.c_int32(batch),
+        C.c_int32(child_row.numel()), _ptr(node_offsets, torch.int32), _ptr(child_row, torch.int32),
+        _ptr(path_nodes, torch.int32), _ptr(accept_len, torch.int32), _ptr(bonus, torch.int32),
+        C.c_int32(max_depth), _ptr(r_prob, torch.float32), _ptr(signal, torch.float32), _ptr(status, torch.int32),
+        _stream())
+    _check(rc, "sb_verifier_signal")
+    return dict(r_prob=r_prob, signal=signal, status=status)
 
 
 SB_STATIC_SCRATCH_BYTES = 256 * 1024

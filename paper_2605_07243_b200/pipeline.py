@@ -127,6 +127,24 @@ class VerifyStep:
                                            device=self.device)
         return sb.sb_rank_features(e["scores"], features=e["features"], workspace=e["features_ws"])
 
+    def run_signal(self):
+        """One iteration's term of the verifier-derived update signal, chained after run_accept() (not
+        part of run_device(): a 'next' row, timed on its own).  The benchmark's tree and drafter rows
+        are separate synthetic pieces, so node i is mapped to drafter row i mod R."""
+        e = self.expand
+        if e is None:
+            return None
+        if "signal" not in e:
+            R = e["scores"].shape[0]
+            n = int(self.tb.total_nodes)
+            e["child_row"] = (torch.arange(n, dtype=torch.int32, device=self.device) % R).contiguous()
+            e["signal"] = torch.zeros(self.tb.prefix_len.numel(), dtype=torch.float32, device=self.device)
+            e["r_prob"] = torch.empty(self.tb.prefix_len.numel(), dtype=torch.float32, device=self.device)
+            e["signal_status"] = torch.empty(self.tb.prefix_len.numel(), dtype=torch.int32, device=self.device)
+        return sb.sb_verifier_signal(e["scores"], self.tb.node_offsets, e["child_row"], self.accept["path_nodes"],
+                                     self.accept["accept_len"], self.accept["bonus"], self.max_depth, e["signal"],
+                                     r_prob=e["r_prob"], status=e["signal_status"])
+
     def run_attention(self, layers=None):
         for l in range(self.n_layers) if layers is None else layers:
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,

@@ -335,3 +335,102 @@ def test_rank_features_vocab_sizes_ties_nan_inf(vocab):
     x[5, :vocab] = 4.0                       # exactly uniform
     x[6, 1] = 60.0                           # one token owns the distribution
     _check_features(x, vocab=vocab)
+
+
+# ---- verifier-derived update signal (Sec. 3.4; Alg. 2 line 2) -----------------------------------------------
+
+SIGNAL_TOL = 2e-5      # |r - r_ref| <= tol * max(r_ref, 1e-3) and |s - s_ref| <= tol: fp32 sums over the row
+
+
+def _check_signal(scores, node_offsets, child_row, path_nodes, accept_len, bonus, max_depth, signal0, vocab=None):
+    sig = torch.from_numpy(np.asarray(signal0, np.float32)).cuda()
+    got = sb.sb_verifier_signal(torch.from_numpy(np.ascontiguousarray(scores)).cuda(), dev.i32_tensor(node_offsets),
+                                dev.i32_tensor(child_row), dev.i32_tensor(path_nodes), dev.i32_tensor(accept_len),
+                                dev.i32_tensor(bonus), max_depth, sig, vocab=vocab)
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in got.items()}
+    ref = oracle.verifier_signal(scores, node_offsets, child_row, path_nodes, accept_len, bonus, max_depth,
+                                 signal=np.asarray(signal0, np.float32), vocab=vocab)
+    np.testing.assert_array_equal(got["status"], ref["status"])
+    none = ref["r_prob"] < 0
+    np.testing.assert_array_equal(got["r_prob"][none], -1.0)
+    err_r = np.abs(got["r_prob"][~none] - ref["r_prob"][~none]) / np.maximum(ref["r_prob"][~none], 1e-3)
+    assert err_r.size == 0 or err_r.max() <= SIGNAL_TOL, f"r error {err_r.max():.2e}"
+    assert np.abs(got["signal"] - ref["signal"]).max() <= SIGNAL_TOL
+    return got, ref
+
+
+def test_verifier_signal_after_accept_config2_and_config3_scores():
+    """The signal chained on the device after sb_verify_accept, over full-vocabulary drafter rows."""
+    par = W.config2_tree()
+    ver = W.config2_logits(par=par, accept_len=3)
+    _, exp = W.config3_drafter()                       # fp32 [32][128256] drafter scores
+    rng = W.rng_for(95)
+    child_row = rng.integers(-1, exp.scores.shape[0], len(par)).astype(np.int32)
+    acc = sb.sb_verify_accept(_logits_tensor(ver.logits), dev.i32_tensor(ver.node_offsets), dev.i32_tensor(ver.parent),
+                              dev.i32_tensor(ver.tok), ver.max_depth)
+    best = int(acc["path_nodes"].cpu().numpy()[0, int(acc["accept_len"].cpu().numpy()[0])])
+    child_row[best] = 7                                  # the row that predicted the rejected position
+    sig = torch.full((1,), 0.25, dtype=torch.float32, device="cuda")
+    got = sb.sb_verifier_signal(torch.from_numpy(exp.scores).cuda(), dev.i32_tensor(ver.node_offsets),
+                                dev.i32_tensor(child_row), acc["path_nodes"], acc["accept_len"], acc["bonus"],
+                                ver.max_depth, sig)
+    torch.cuda.synchronize()
+    ref_acc = oracle.verify_accept(ver.logits, ver.node_offsets, ver.parent, ver.tok, ver.max_depth)
+    ref = oracle.verifier_signal(exp.scores, ver.node_offsets, child_row, ref_acc["path_nodes"], ref_acc["accept_len"],
+                                 ref_acc["bonus"], ver.max_depth, signal=[0.25])
+    assert int(got["status"].cpu()[0]) == 0 and ref["status"][0] == 0
+    r, r_ref = float(got["r_prob"].cpu()[0]), ref["r_prob"][0]
+    assert abs(r - r_ref) <= SIGNAL_TOL * max(r_ref, 1e-3)
+    assert abs(float(got["signal"].cpu()[0]) - ref["signal"][0]) <= SIGNAL_TOL
+
+
+@pytest.mark.parametrize("vocab", [1, 5, 1000, 4099, 32000, 128256])
+def test_verifier_signal_vocab_sizes_batch_and_degenerate_rows(vocab):
+    rng = W.rng_for(96 + vocab)
+    R, B, n, max_depth = 9, 11, 6, 5
+    x = (rng.standard_normal((R, vocab + 3), dtype=np.float32) * 3).astype(np.float32)
+    x[:, vocab:] = 1e9                       # padding beyond vocab must be ignored
+    x[1, :vocab:3] = np.nan
+    x[2, :vocab] = -np.inf                   # no finite score: flat
+    x[3, :vocab] = 2.0                       # exactly flat
+    x[4, :vocab] = -np.inf
+    x[4, vocab // 2] = 1.0                   # one finite score
+    x[5, vocab - 1] = 70.0                   # one token owns the row, in the last CTA's tail
+    node_offsets = np.arange(B + 1, dtype=np.int32) * n
+    child_row = rng.integers(0, R, B * n).astype(np.int32)
+    accept_len = rng.integers(0, max_depth + 1, B).astype(np.int32)
+    path = rng.integers(0, n, (B, max_depth + 1)).astype(np.int32)
+    bonus = rng.integers(0, vocab, B).astype(np.int32)
+    for b in range(min(B, R)):               # sequence b reads row b, so every special row is used
+        child_row[b * n + path[b, accept_len[b]]] = b
+    bonus[4] = vocab // 2
+    bonus[5] = vocab - 1
+    bonus[6] = vocab + 2                     # outside the drafter's vocabulary: r = 0
+    child_row[7 * n + path[7, accept_len[7]]] = -1      # nothing drafted there
+    child_row[9 * n + path[9, accept_len[9]]] = R       # row out of range
+    accept_len[10] = max_depth + 1                      # accept length out of range
+    got, ref = _check_signal(x, node_offsets, child_row, path, accept_len, bonus, max_depth,
+                             rng.random(B).astype(np.float32), vocab=vocab)
+    assert list(got["status"][[9, 10]]) == [5, 5] and got["r_prob"][7] == -1.0
+    if vocab > 1:
+        assert got["r_prob"][6] == 0.0 and abs(got["r_prob"][5] - 1.0) < 1e-6
+
+
+def test_verifier_signal_unaligned_rows_and_host_errors():
+    rng = W.rng_for(97)
+    x = (rng.standard_normal((4, 1001), dtype=np.float32)).astype(np.float32)   # odd stride: rows 1..3 unaligned
+    node_offsets = np.asarray([0, 3, 6], np.int32)
+    child_row = np.asarray([1, 2, 3, 3, 2, 1], np.int32)
+    path = np.asarray([[0, 1, 2], [2, 1, 0]], np.int32)
+    accept_len = np.asarray([2, 1], np.int32)
+    _check_signal(x, node_offsets, child_row, path, accept_len, np.asarray([5, 999], np.int32), 2, [0.0, 1.5],
+                  vocab=999)
+    t = torch.from_numpy(x).cuda()
+    sig = torch.zeros(2, dtype=torch.float32, device="cuda")
+    with pytest.raises(sb.SbError):
+        sb.sb_verifier_signal(t, dev.i32_tensor(node_offsets), dev.i32_tensor(child_row), dev.i32_tensor(path),
+                              dev.i32_tensor(accept_len), dev.i32_tensor([1, 1]), 2, sig, vocab=2000)
+    with pytest.raises(sb.SbError):
+        sb.sb_verifier_signal(t, dev.i32_tensor(node_offsets), dev.i32_tensor(child_row), dev.i32_tensor(path),
+                              dev.i32_tensor(accept_len), dev.i32_tensor([1, 1]), 99, sig)
