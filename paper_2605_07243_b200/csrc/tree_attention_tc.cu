@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     const int nj = min(TC_BN, chunk_keys - j * TC_BN);
     const int k0 = key_begin + j * TC_BN;
     const int pieces = ceil_div(nj, box_rows);
-#pragma unroll
+#pragma unroll 1
     for (int i = 0; i < MAX_PIECES; ++i)
       if (i < pieces) pg[i] = p.tb.page_table[(long long)b * p.tb.max_pages + (k0 + i * box_rows) / p.tb.page_size];
   };
@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     const int k0 = key_begin + j * TC_BN;
     const int pieces = ceil_div(nj, box_rows);
     mbar_expect_tx(bar, (uint32_t)(pieces * box_rows * D * 2));
-#pragma unroll
+#pragma unroll 1
     for (int i = 0; i < MAX_PIECES; ++i) {
       if (i >= pieces) break;
       const int key = k0 + i * box_rows;
