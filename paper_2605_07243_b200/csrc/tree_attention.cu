@@ -28,6 +28,7 @@ namespace sb {
 // tcgen05 kernel (tree_attention_tc.cu)
 sb_status launch_attn_tc(const AttnParams& p, dim3 grid, int cluster, cudaStream_t cs);
 int attn_tc_max_active_clusters(int D, int cluster);
+sb_status launch_attn_tc2(const AttnParams& p, dim3 grid, cudaStream_t cs);
 
 // ----------------------------------------------------------------------------------------------
 // Simple kernel: one warp per (node, head) row.
@@ -434,8 +435,9 @@ static sb_status check_batch(const sb_tree_batch* tb) {
 constexpr int kMaxCluster = 8;  // portable thread-block cluster size
 
 struct SplitPlan {
-  int cluster;  // chunk-CTAs merged through distributed shared memory
-  int outer;    // clusters per (sequence, KV head, row tile)
+  int cluster;     // chunk-CTAs merged through distributed shared memory
+  int outer;       // clusters per (sequence, KV head, row tile)
+  bool two_tiles;  // the two-tiles-per-CTA tcgen05 kernel (no clusters: outer = chunks)
 };
 
 // How many clusters of `cluster` CTAs of the attention kernel can be resident at once (0 when the
@@ -480,6 +482,7 @@ static int max_active_clusters(int D, int cluster) {
 // configuration: 1072 us against 1227 us).
 static SplitPlan plan_for(int s, bool oversubscribed) {
   SplitPlan sp;
+  sp.two_tiles = false;
   sp.cluster = 1;
   int cmax = oversubscribed ? 2 : kMaxCluster;
   if (const char* e = getenv("SB_ATTN_MAX_CLUSTER")) {  // experiment knob
@@ -505,13 +508,45 @@ static AttnImpl attn_impl() {
 // largest count whose clusters are all resident at once when the batch is small, otherwise
 // chunks of a few KV blocks to even out ragged prefix lengths.  The chunks are grouped into
 // clusters of the largest divisor <= 8.  `granule` is the kernel's key-block size.
-static SplitPlan choose_splits(const sb_tree_batch* tb, int num_splits, AttnImpl impl) {
+static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_splits, AttnImpl impl) {
   const int G = tb->n_q_heads / tb->n_kv_heads;
   const int row_tiles = ceil_div(tb->max_nodes * G, BM);
   const int granule = impl == IMPL_TC ? 128 : BN;
   const int max_blocks = ceil_div(tb->max_kv_len, granule);
   const long long base = (long long)tb->batch * tb->n_kv_heads * row_tiles;
   const int sms = num_sms();
+  // More (sequence, KV head, row tile) units than SMs and at least two row tiles per KV head: the
+  // tcgen05 kernel that gives one CTA two tiles (each K/V block is pulled from L2 once for both).
+  // (With three tiles the second CTA of a KV head would hold a single one, and ragged batches whose
+  // largest tree has three tiles mostly hold one or two: measured slower than the one-tile kernel.)
+  bool two_tiles = impl == IMPL_TC && row_tiles >= 2 && row_tiles != 3 && base > sms;
+  if (const char* e = getenv("SB_ATTN_TWO_TILES")) two_tiles = impl == IMPL_TC && row_tiles >= 2 && atoi(e) != 0;
+  if (two_tiles) {
+    SplitPlan sp;
+    sp.two_tiles = true;
+    sp.cluster = 1;
+    if (num_splits > 0) {
+      sp.outer = num_splits < max_blocks ? num_splits : max_blocks;
+      return sp;
+    }
+    // CTAs run in waves; a CTA costs its blocks (two tiles each) plus a fixed start-up worth about
+    // five, and every chunk beyond the first writes and re-reads an fp32 partial of all rows, here
+    // in units of one block-time (1.2 us) at 6 TB/s.
+    const long long units = (long long)tb->batch * tb->n_kv_heads * ceil_div(row_tiles, 2);
+    const double partial = 2.0 * (double)total_q * tb->n_q_heads * tb->head_dim * 4.0 / 6e12 / 1.2e-6;
+    int best = 1;
+    double best_cost = 0.0;
+    for (int s = 1; s <= 8 && s <= max_blocks; ++s) {
+      const long long waves = (units * s + sms - 1) / sms;
+      const double cost = (double)waves * (2 * ceil_div(max_blocks, s) + 5) + (s > 1 ? partial * s + 3.0 : 0.0);
+      if (s == 1 || cost < best_cost) {
+        best = s;
+        best_cost = cost;
+      }
+    }
+    sp.outer = best;
+    return sp;
+  }
   if (num_splits > 0) {
     const int s = num_splits < max_blocks ? num_splits : max_blocks;
     return plan_for(s, base * s > 2LL * sms);
@@ -596,7 +631,7 @@ static sb_status launch_attn_mma(const AttnParams& p, dim3 grid, int cluster, cu
 extern "C" size_t sb_tree_attention_workspace_bytes(const sb_tree_batch* tb, int32_t total_q,
                                                     int32_t num_splits) {
   if (sb::check_batch(tb) != SB_OK || total_q < 0 || num_splits < 0) return 0;
-  return sb::workspace_bytes_for(tb, total_q, sb::choose_splits(tb, num_splits, sb::attn_impl()).outer);
+  return sb::workspace_bytes_for(tb, total_q, sb::choose_splits(tb, total_q, num_splits, sb::attn_impl()).outer);
 }
 
 extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q_node_begin,
@@ -638,7 +673,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
     return launch_check();
   }
 
-  const SplitPlan plan = choose_splits(tb, num_splits, impl);
+  const SplitPlan plan = choose_splits(tb, total_q, num_splits, impl);
   p.num_splits = plan.cluster * plan.outer;
   p.outer = plan.outer;
   if (plan.outer > 1) {
@@ -652,9 +687,10 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   }
   const int row_tiles = ceil_div(tb->max_nodes * p.G, BM);
   p.row_tiles = row_tiles;
-  dim3 grid(p.num_splits, row_tiles * tb->n_kv_heads, tb->batch);
+  dim3 grid(p.num_splits, (plan.two_tiles ? ceil_div(row_tiles, 2) : row_tiles) * tb->n_kv_heads, tb->batch);
   if (grid.y > 65535 || grid.z > 65535) return SB_ERR_UNSUPPORTED;
-  if (impl == IMPL_TC) st = launch_attn_tc(p, grid, plan.cluster, cs);
+  if (plan.two_tiles) st = launch_attn_tc2(p, grid, cs);
+  else if (impl == IMPL_TC) st = launch_attn_tc(p, grid, plan.cluster, cs);
   else st = D == 64 ? launch_attn_mma<64>(p, grid, plan.cluster, cs) : launch_attn_mma<128>(p, grid, plan.cluster, cs);
   if (st != SB_OK || plan.outer == 1) return st;
   dim3 mgrid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);

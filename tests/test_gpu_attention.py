@@ -267,3 +267,39 @@ def test_config5_long_context_full_size_sampled():
     attn, _ = W.config5_long(with_logits=False)
     sel = sample_rows(attn, 96, seed=5)
     check_attention(attn, "config 5 sampled, 16 chunks", sel=sel, num_splits=16)
+
+
+def test_two_tiles_per_cta_kernel(monkeypatch):
+    """The throughput kernel (two row tiles per CTA, P written over S in tensor memory, chunks merged
+    from fp32 partials), forced on shapes that would otherwise take the one-tile kernel."""
+    monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
+    check_attention(W.config2_verify_layer(prefix=777), "two tiles: 8B-shaped, P=777, 1 chunk", num_splits=1)
+    check_attention(W.config2_verify_layer(prefix=777), "two tiles: 8B-shaped, P=777, 3 chunks", num_splits=3)
+    check_attention(W.config2_verify_layer(prefix=2048), "two tiles: 8B-shaped, library's chunks")
+    check_attention(W.config2_verify_layer(prefix=300), "two tiles: more chunks than blocks", num_splits=16)
+    rng = W.rng_for(70)
+    # ragged trees: 1, 2, 3 and 8 row tiles in one batch (a last pair with a single tile), paged, G = 8
+    parents = [W.random_tree(rng, 128, 12), W.chain_tree(5), W.random_tree(rng, 40, 6), W.random_tree(rng, 24, 4)]
+    case = W.make_attn_case(rng, parents=parents, prefix_lens=[333, 0, 2000, 129], n_q_heads=64, n_kv_heads=8,
+                            head_dim=128, page_size=64)
+    check_attention(case, "two tiles: ragged paged G=8", num_splits=5)
+    check_attention(case, "two tiles: ragged paged G=8, one chunk", num_splits=1)
+    # G = 3 does not divide 128: Q tiles are gathered; head_dim 64; page 16
+    case = W.make_attn_case(rng, parents=[W.random_tree(rng, 100, 9), W.random_tree(rng, 50, 5)], prefix_lens=[700, 64],
+                            n_q_heads=6, n_kv_heads=2, head_dim=64, page_size=16, scale=0.2)
+    check_attention(case, "two tiles: G=3, D=64, page 16", num_splits=2)
+    # no prefix at all: every block is masked
+    case = W.make_attn_case(rng, parents=[W.random_tree(rng, 128, 10)], prefix_lens=[0], n_q_heads=8, n_kv_heads=2,
+                            head_dim=128)
+    check_attention(case, "two tiles: P=0")
+
+
+def test_two_tiles_per_cta_long_chunks(monkeypatch):
+    """Many blocks per CTA (the steady state of the two-tile pipeline), peaky scores so that the
+    reference maximum moves and accumulators are rescaled."""
+    monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
+    rng = W.rng_for(71)
+    case = W.make_attn_case(rng, parents=[W.random_tree(rng, 96, 10), W.random_tree(rng, 33, 10)],
+                            prefix_lens=[6000, 3001], n_q_heads=32, n_kv_heads=8, head_dim=128, page_size=64, q_std=4.0)
+    check_attention(case, "two tiles: long chunks, peaky", num_splits=1)
+    check_attention(case, "two tiles: long chunks, peaky, 2 chunks", num_splits=2)
