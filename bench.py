@@ -34,7 +34,7 @@ N_LAYERS = 32
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on this workload, from the
 # ncu capture summarised in profiles/attn_tc_kernel_c2_verify_layer.md
-ATTN_DRAM_TRAFFIC_BYTES = 9230336
+ATTN_DRAM_TRAFFIC_BYTES = 9209856
 FALLBACK_HBM_GBS = 6650.0
 
 
