@@ -13,6 +13,7 @@ from .oracle import (  # noqa: F401
     rank_features,
     verify_accept,
     verifier_signal,
+    verify_sample,
     accept_from_amax,
     kv_compact,
     tree_expand,

@@ -176,6 +176,29 @@ def verify_accept(logits, node_offsets, parent, tok, max_depth, vocab=None):
     return r
 
 
+def verify_sample(logits, scores, node_offsets, parent, tok, child_row, temperature, u_accept, u_bonus, max_depth,
+                  vocab=None):
+    """Stochastic tree verification.  -> dict(accept_len, path_nodes, out_tokens, bonus, status)."""
+    logits, dt = _logits_arg(logits)
+    scores = np.ascontiguousarray(scores, np.float32)
+    total, stride = logits.shape
+    n_rows, sstride = scores.shape
+    vocab = stride if vocab is None else vocab
+    node_offsets, parent, tok, child_row = _i32(node_offsets), _i32(parent), _i32(tok), _i32(child_row)
+    u_accept = np.ascontiguousarray(u_accept, np.float32)
+    u_bonus = np.ascontiguousarray(u_bonus, np.float32)
+    batch = node_offsets.shape[0] - 1
+    r = dict(accept_len=np.zeros(batch, np.int32), path_nodes=np.zeros((batch, max_depth + 1), np.int32),
+             out_tokens=np.zeros((batch, max_depth + 1), np.int32), bonus=np.zeros(batch, np.int32),
+             status=np.zeros(batch, np.int32))
+    _load().sbo_verify_sample(_p(logits), C.c_int(dt), C.c_int64(stride), C.c_int(vocab), _p(scores),
+                              C.c_int64(sstride), C.c_int(n_rows), C.c_int(batch), _p(node_offsets), _p(parent),
+                              _p(tok), _p(child_row), C.c_double(temperature), _p(u_accept), _p(u_bonus),
+                              C.c_int(max_depth), _p(r["accept_len"]), _p(r["path_nodes"]), _p(r["out_tokens"]),
+                              _p(r["bonus"]), _p(r["status"]))
+    return r
+
+
 def accept_from_amax(parent, tok, amax, max_depth):
     parent, tok, amax = _i32(parent), _i32(tok), _i32(amax)
     n = parent.shape[0]

@@ -20,6 +20,14 @@
  *   sbo_rank_features   : scipy log_softmax / entropy; closed forms (uniform row, one dominant token).
  *   sbo_verifier_signal : scipy softmax; closed forms (flat row, one raised token); probabilities of
  *                         all tokens of a row sum to one; the sum over iterations of a query.
+ *   sbo_verify_sample   : the textbook identity of speculative sampling -- with the candidate drawn from
+ *                         the draft distribution (one candidate, and two drawn without replacement) the
+ *                         committed token is distributed exactly as the target -- checked by exact
+ *                         integration over the uniforms (acceptance thresholds and bonus intervals found
+ *                         by bisection on the oracle); T -> 0 reduces to greedy acceptance.  The paper
+ *                         names the procedure only as "rejection sampling": the order in which siblings
+ *                         are tried and the treatment of the draft distribution after a rejection are
+ *                         readings -- for those PARITY IS UNPINNED by the paper.
  *   sbo_tree_expand     : hand-derived trees for the two printed branching maps; chain special
  *                         case; structural invariants.  The attach point of siblings, the cut
  *                         order at the node budget and the treatment of b = 0 are readings of
@@ -493,6 +501,128 @@ void sbo_rank_features(const float* scores, int64_t row_stride, int n_rows, int 
     f[14] = entropy;
     free(e);
   }
+}
+
+/* ---- stochastic verification of a draft tree (Sec. 4.1 "temperature 0 and 1.0"; Sec. 4.2) ------- */
+
+/*
+ * The paper verifies at temperature 1 by "rejection sampling against the target" without giving
+ * the procedure; this is the multi-candidate rejection sampling of tree-based speculative decoding
+ * (the systems it compares with), taken in the order below.  All random numbers are inputs.
+ *
+ *   node a = root (0), depth 0, p = softmax(logits[a] / T).
+ *   repeat:
+ *     children of a = the nodes c with parent[c] == a, in increasing index (= emission order).
+ *     no children, or depth == max_depth: stop.
+ *     q = softmax(scores[child_row[a]] / T)   (the draft distribution that proposed them).
+ *     for each child c in order, x = tok[c]:
+ *         accept c iff  u_accept[c] < p(x) / q(x)   (q(x) = 0: accepted iff p(x) > 0);
+ *         accepted: a = c, depth += 1, p = softmax(logits[c] / T), next round;
+ *         rejected: p <- max(p - q, 0) renormalised (left as it is if nothing remains),
+ *                   q(x) <- 0 and q renormalised (x was drawn without replacement).
+ *     every child rejected: stop.
+ *   bonus = the smallest v with  sum_{w <= v} p(w) > u_bonus * sum_w p(w)  (the last v with
+ *   p(v) > 0 if rounding leaves none), p being the (possibly residual) distribution at the stop.
+ * Outputs as sbo_verify_accept: accept_len = depth, path_nodes, out_tokens = accepted tokens then
+ * bonus.  status 4: invalid tree; 5: child_row of an inner node on the walk outside [0, n_rows).
+ * NaN logits/scores count as -inf; a row without a finite value is flat.
+ */
+static void softmax_row_f64(const void* row, int dtype, int64_t base, int vocab, double inv_t, double* out) {
+  double m = -INFINITY;
+  for (int v = 0; v < vocab; ++v) {
+    const double x = score_of(logit_at(row, dtype, base + v));
+    if (x > m) m = x;
+  }
+  double z = 0.0;
+  for (int v = 0; v < vocab; ++v) {
+    const double x = score_of(logit_at(row, dtype, base + v));
+    out[v] = m == -INFINITY ? 1.0 : exp((x - m) * inv_t);
+    z += out[v];
+  }
+  for (int v = 0; v < vocab; ++v) out[v] /= z;
+}
+
+void sbo_verify_sample(const void* logits, int dtype, int64_t row_stride, int vocab, const float* scores,
+                       int64_t score_stride, int n_rows, int batch, const int32_t* node_offsets,
+                       const int32_t* parent, const int32_t* tok, const int32_t* child_row, double temperature,
+                       const float* u_accept, const float* u_bonus, int max_depth, int32_t* accept_len,
+                       int32_t* path_nodes, int32_t* out_tokens, int32_t* bonus, int32_t* status) {
+  const double inv_t = 1.0 / temperature;
+  double* p = (double*)malloc(sizeof(double) * (size_t)vocab);
+  double* q = (double*)malloc(sizeof(double) * (size_t)vocab);
+  for (int b = 0; b < batch; ++b) {
+    const int o = node_offsets[b], n = node_offsets[b + 1] - o;
+    const int32_t *par = parent + o, *tk = tok + o;
+    int32_t* path = path_nodes + (int64_t)b * (max_depth + 1);
+    int32_t* otok = out_tokens + (int64_t)b * (max_depth + 1);
+    for (int t = 0; t <= max_depth; ++t) { path[t] = -1; otok[t] = -1; }
+    accept_len[b] = 0;
+    bonus[b] = -1;
+    status[b] = 0;
+    int valid = n >= 1 && tree_is_valid(par, n) && par[0] == -1;
+    for (int i = 1; valid && i < n; ++i)
+      if (par[i] == -1) valid = 0;
+    if (!valid) { status[b] = 4; continue; }
+    int a = 0, depth = 0;
+    path[0] = 0;
+    softmax_row_f64(logits, dtype, (int64_t)(o + a) * row_stride, vocab, inv_t, p);
+    for (;;) {
+      int first_child = -1;
+      for (int c = a + 1; c < n; ++c)
+        if (par[c] == a) { first_child = c; break; }
+      if (first_child < 0 || depth == max_depth) break;
+      const int row = child_row[o + a];
+      if (row < 0 || row >= n_rows) { status[b] = 5; break; }
+      softmax_row_f64(scores, 1, (int64_t)row * score_stride, vocab, inv_t, q);
+      int accepted = -1;
+      for (int c = first_child; c < n; ++c) {
+        if (par[c] != a) continue;
+        const int x = tk[c];
+        const double px = (x >= 0 && x < vocab) ? p[x] : 0.0;
+        const double qx = (x >= 0 && x < vocab) ? q[x] : 0.0;
+        const int take = qx > 0.0 ? ((double)u_accept[o + c] < px / qx) : (px > 0.0);
+        if (take) { accepted = c; break; }
+        /* rejected: residual target, and the token leaves the draft distribution */
+        double z = 0.0;
+        for (int v = 0; v < vocab; ++v) z += p[v] > q[v] ? p[v] - q[v] : 0.0;
+        if (z > 0.0)
+          for (int v = 0; v < vocab; ++v) p[v] = (p[v] > q[v] ? p[v] - q[v] : 0.0) / z;
+        if (x >= 0 && x < vocab) {
+          q[x] = 0.0;
+          double zq = 0.0;
+          for (int v = 0; v < vocab; ++v) zq += q[v];
+          if (zq > 0.0)
+            for (int v = 0; v < vocab; ++v) q[v] /= zq;
+        }
+      }
+      if (accepted < 0) break;
+      a = accepted;
+      ++depth;
+      path[depth] = a;
+      otok[depth - 1] = tk[a];
+      softmax_row_f64(logits, dtype, (int64_t)(o + a) * row_stride, vocab, inv_t, p);
+    }
+    if (status[b]) {
+      for (int t = 0; t <= max_depth; ++t) { path[t] = -1; otok[t] = -1; }
+      continue;
+    }
+    double total = 0.0;
+    for (int v = 0; v < vocab; ++v) total += p[v];
+    const double target = (double)u_bonus[b] * total;
+    double cum = 0.0;
+    int pick = -1, last_pos = -1;
+    for (int v = 0; v < vocab; ++v) {
+      if (p[v] > 0.0) last_pos = v;
+      cum += p[v];
+      if (cum > target) { pick = v; break; }
+    }
+    if (pick < 0) pick = last_pos;
+    accept_len[b] = depth;
+    bonus[b] = pick;
+    otok[depth] = pick;
+  }
+  free(p);
+  free(q);
 }
 
 /* ---- verifier-derived update signal (Sec. 3.4, the equation for s; Alg. 2 line 2) ------------- */

@@ -456,3 +456,135 @@ def test_verifier_signal_invariants_accumulation_and_bounds():
     assert (g["status"] == 5).all() and (g["signal"] == 0.5).all() and (g["r_prob"] == -1).all()
     bad = _signal_inputs([4], [1], [0], 1)                  # path node 4 of a 1-node tree
     assert oracle.verifier_signal(x, **bad)["status"][0] == 5
+
+
+# ---- stochastic verification (temperature > 0): multi-candidate rejection sampling on the tree -----------------
+
+def _one_level_case(rng, V, cand):
+    """Root with len(cand) leaf children carrying the tokens `cand`; one drafter row."""
+    n = 1 + len(cand)
+    logits = (rng.standard_normal((n, V)) * 1.5).astype(np.float32)
+    scores = (rng.standard_normal((1, V)) * 1.5).astype(np.float32)
+    parent = np.asarray([-1] + [0] * len(cand), np.int32)
+    tok = np.asarray([0] + list(cand), np.int32)
+    child_row = np.asarray([0] + [-1] * len(cand), np.int32)
+    return logits, scores, parent, tok, child_row
+
+
+def _run_sample(case, u_accept, u_bonus, T=1.0, max_depth=4):
+    logits, scores, parent, tok, child_row = case
+    r = oracle.verify_sample(logits, scores, [0, len(parent)], parent, tok, child_row, T, u_accept, [u_bonus], max_depth)
+    assert r["status"][0] == 0
+    return int(r["accept_len"][0]), int(r["out_tokens"][0, 0]), int(r["bonus"][0])
+
+
+def _threshold(f):
+    """sup{u in [0,1]: f(u)} for a predicate that is true on [0, theta) (float32 resolution)."""
+    if not f(0.0):
+        return 0.0
+    if f(np.nextafter(np.float32(1.0), np.float32(0.0))):
+        return 1.0
+    lo, hi = 0.0, 1.0
+    for _ in range(30):
+        mid = 0.5 * (lo + hi)
+        lo, hi = (mid, hi) if f(mid) else (lo, mid)
+    return 0.5 * (lo + hi)
+
+
+def _bonus_distribution(run_with_u_bonus, V):
+    """Measure of the u_bonus interval that yields each token (the bonus is monotone in u)."""
+    edges = [0.0] + [_threshold(lambda u, v=v: run_with_u_bonus(u) <= v) for v in range(V - 1)] + [1.0]
+    return np.diff(np.asarray(edges))
+
+
+def test_verify_sample_one_candidate_from_q_commits_exactly_the_target_distribution():
+    """Speculative sampling's identity: x ~ q accepted with probability min(1, p/q), else a draw from
+    norm(max(p - q, 0)), is distributed as p.  Checked by exact integration over both uniforms."""
+    from scipy.special import softmax
+    rng = W.rng_for(36)
+    V = 6
+    first = np.zeros(V)
+    base = None
+    for x in range(V):
+        rng_x = W.rng_for(360)                      # the same p and q for every candidate
+        case = _one_level_case(rng_x, V, [x])
+        if base is None:
+            base = case
+            p = softmax(case[0][0].astype(np.float64))
+            q = softmax(case[1][0].astype(np.float64))
+        theta = _threshold(lambda u: _run_sample(case, [0.0, u], 0.5)[0] == 1)
+        np.testing.assert_allclose(theta, min(1.0, p[x] / q[x]), atol=2e-7)      # the acceptance rule itself
+        first[x] += q[x] * theta
+        if theta < 1.0:
+            res = _bonus_distribution(lambda u: _run_sample(case, [0.0, 1.0], u)[2], V)
+            want = np.maximum(p - q, 0.0)
+            np.testing.assert_allclose(res, want / want.sum(), atol=5e-7)         # the residual distribution
+            first += q[x] * (1.0 - theta) * res
+    np.testing.assert_allclose(first, p, atol=2e-6)
+    del rng
+
+
+def test_verify_sample_two_candidates_without_replacement_is_still_exact():
+    from scipy.special import softmax
+    V = 5
+    first = np.zeros(V)
+    for x1 in range(V):
+        for x2 in range(V):
+            if x2 == x1:
+                continue
+            case = _one_level_case(W.rng_for(361), V, [x1, x2])
+            p = softmax(case[0][0].astype(np.float64))
+            q = softmax(case[1][0].astype(np.float64))
+            q2 = q.copy()
+            q2[x1] = 0.0
+            q2 /= q2.sum()
+            w = q[x1] * q2[x2]                        # probability of drawing (x1, x2) without replacement
+            th1 = _threshold(lambda u: _run_sample(case, [0.0, u, 0.0], 0.5)[1] == x1 and
+                             _run_sample(case, [0.0, u, 0.0], 0.5)[0] == 1)
+            first[x1] += w * th1
+            if th1 >= 1.0:
+                continue
+            th2 = _threshold(lambda u: _run_sample(case, [0.0, 1.0, u], 0.5)[0] == 1)
+            first[x2] += w * (1.0 - th1) * th2
+            if th2 >= 1.0:
+                continue
+            res = _bonus_distribution(lambda u: _run_sample(case, [0.0, 1.0, 1.0], u)[2], V)
+            first += w * (1.0 - th1) * (1.0 - th2) * res
+    p = softmax(_one_level_case(W.rng_for(361), V, [0, 1])[0][0].astype(np.float64))
+    np.testing.assert_allclose(first, p, atol=5e-6)
+
+
+def test_verify_sample_low_temperature_is_greedy_and_walks_the_tree():
+    rng = W.rng_for(37)
+    par = W.random_tree(rng, 30, 6)
+    ver = W.make_verify_case(rng, parents=[par], vocab=300, dtype="f32", std=2.0, accept_lens=[4], max_depth=6)
+    n = len(par)
+    scores = (rng.standard_normal((n, 300)) * 2).astype(np.float32)
+    child_row = np.arange(n, dtype=np.int32)
+    greedy = oracle.verify_accept(ver.logits, ver.node_offsets, ver.parent, ver.tok, ver.max_depth)
+    # T -> 0 against a flat draft distribution (which no temperature sharpens): the target becomes
+    # one-hot at its argmax, a child is accepted iff it carries that token, whatever the uniforms
+    flat = np.zeros_like(scores)
+    for rep in range(5):
+        u_a = rng.random(n).astype(np.float32)
+        got = oracle.verify_sample(ver.logits, flat, ver.node_offsets, ver.parent, ver.tok, child_row, 0.02, u_a,
+                                   [rng.random()], ver.max_depth)
+        for key in ("accept_len", "path_nodes", "out_tokens", "bonus"):
+            np.testing.assert_array_equal(got[key], greedy[key], err_msg=key)
+    # at temperature 1 the result is a root-to-node path whose tokens are the path's, followed by the bonus
+    for rep in range(20):
+        got = oracle.verify_sample(ver.logits, scores, ver.node_offsets, ver.parent, ver.tok, child_row, 1.0,
+                                   rng.random(n).astype(np.float32), [rng.random()], 3)
+        a = int(got["accept_len"][0])
+        path = got["path_nodes"][0]
+        assert 0 <= a <= 3 and path[0] == 0 and (path[a + 1:] == -1).all()
+        for t in range(1, a + 1):
+            assert ver.parent[path[t]] == path[t - 1] and got["out_tokens"][0, t - 1] == ver.tok[path[t]]
+        assert got["out_tokens"][0, a] == got["bonus"][0] and 0 <= got["bonus"][0] < 300
+    # invalid trees and a missing drafter row are reported
+    bad = oracle.verify_sample(ver.logits, scores, ver.node_offsets, np.full(n, -1, np.int32), ver.tok, child_row, 1.0,
+                               np.zeros(n, np.float32), [0.5], 3)
+    assert bad["status"][0] == 4
+    no_row = oracle.verify_sample(ver.logits, scores, ver.node_offsets, ver.parent, ver.tok, np.full(n, -1, np.int32),
+                                  1.0, np.zeros(n, np.float32), [0.5], 3)
+    assert no_row["status"][0] == 5
