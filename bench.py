@@ -236,6 +236,8 @@ def run_ours(args):
         g_features = capture(torch, step.run_rank_features)
         step.run_signal()
         g_signal = capture(torch, step.run_signal)
+        step.run_sample()
+        g_sample = capture(torch, step.run_sample)
 
         for _ in range(max(args.warmup, 3)):
             g_step.replay()
@@ -264,7 +266,8 @@ def run_ours(args):
         clocks = sampler.stop()
         parts_ms = {}
         for name, g in (("expand", g_expand), ("accept", g_accept), ("compact", g_compact),
-                        ("rank_features_not_in_step", g_features), ("verifier_signal_not_in_step", g_signal)):
+                        ("rank_features_not_in_step", g_features), ("verifier_signal_not_in_step", g_signal),
+                        ("verify_sample_T1_not_in_step", g_sample)):
             for _ in range(3):
                 g.replay()
             parts_ms[name] = time_graph(torch, g, 20, False) / 20

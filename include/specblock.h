@@ -12,6 +12,7 @@
  *   sb_tree_expand     per-row top-k + bucket-driven branching          (Sec. 3.2, App. A.5, Alg. 1 "attach")
  *   sb_rank_features   15-dim summary of each draft distribution        (Sec. 3.2, App. B)
  *   sb_verifier_signal verifier-derived update signal s = sum (1 - r)   (Sec. 3.4, Alg. 2)
+ *   sb_verify_sample   stochastic (temperature > 0) tree verification   (Sec. 4.1, Sec. 4.2)
  *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
  *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
  *
@@ -185,6 +186,44 @@ size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab);
 sb_status sb_rank_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
                            float* features, void* workspace, size_t workspace_bytes, void* stream);
 size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
+
+/*
+ * sb_verify_sample -- verification at temperature T > 0 by multi-candidate rejection sampling over
+ * the draft tree (Sec. 4.1 evaluates temperature 0 and 1.0; Sec. 4.2 "rejection sampling against a
+ * high-entropy target").  The paper names the procedure without listing it; the steps are:
+ *
+ *   a = root (node 0), depth 0, p = softmax(logits[a] / T).  Repeat:
+ *     children of a = the nodes c with parent[c] == a, in increasing index (emission order);
+ *     stop if there are none or depth == max_depth;
+ *     q = softmax(scores[child_row[a]] / T), the draft distribution that proposed them;
+ *     for each child c in order, x = tok[c]: accept c iff u_accept[c] < p(x) / q(x)
+ *       (q(x) = 0: iff p(x) > 0).  Accepted: a = c, depth += 1, p = softmax(logits[c] / T), next round.
+ *       Rejected: p <- max(p - q, 0) renormalised (unchanged if nothing remains); q(x) <- 0 and q
+ *       renormalised (siblings are distinct tokens: drawn without replacement).
+ *     stop if every child was rejected.
+ *   bonus = the smallest v whose inclusive prefix sum of p exceeds u_bonus * sum(p) (p is the residual
+ *   distribution when the walk stopped on a rejection).
+ *
+ *   logits [total_nodes][row_stride >= vocab] bf16 or fp32 (target), scores fp32
+ *   [n_rows][score_stride >= vocab] (drafter, over the same vocabulary), child_row int32 [total_nodes]
+ *   as for sb_verifier_signal, u_accept fp32 [total_nodes] and u_bonus fp32 [batch] uniform in [0, 1)
+ *   supplied by the caller (the library draws no random numbers).  NaN counts as -inf; a row without a
+ *   finite value is flat.  Outputs as sb_verify_accept (accept_len = depth reached, path_nodes,
+ *   out_tokens = accepted tokens then the bonus, bonus).
+ *   status int32 [batch]: SB_OK, SB_ERR_INVALID_TREE, or SB_ERR_BOUNDS when an inner node of the walk
+ *   has no valid child_row (outputs of that sequence: accept_len 0, -1 elsewhere).
+ *   workspace: sb_verify_sample_workspace_bytes(batch, vocab) = batch * 2 * vocab floats, 16-byte aligned.
+ *   Probabilities and sums are fp32; a decision whose two sides differ by less than about 1e-5
+ *   relative may fall either way.
+ */
+sb_status sb_verify_sample(const void* logits, sb_dtype dtype, int64_t row_stride, int32_t vocab,
+                           const float* scores, int64_t score_stride, int32_t n_rows, int32_t batch,
+                           int32_t total_nodes, const int32_t* node_offsets, const int32_t* parent,
+                           const int32_t* tok, const int32_t* child_row, float temperature,
+                           const float* u_accept, const float* u_bonus, int32_t max_depth, int32_t* accept_len,
+                           int32_t* path_nodes, int32_t* out_tokens, int32_t* bonus, void* workspace,
+                           size_t workspace_bytes, int32_t* status, void* stream);
+size_t sb_verify_sample_workspace_bytes(int32_t batch, int32_t vocab);
 
 /*
  * sb_verifier_signal -- one iteration's term of the verifier-derived update signal

@@ -62,10 +62,11 @@ def load(build_if_missing: bool = True):
     lib.sb_version.restype = C.c_int32
     lib.sb_kernel_launch_count.restype = C.c_int64
     for name in ("sb_tree_attention_workspace_bytes", "sb_tree_expand_workspace_bytes",
-                 "sb_verify_accept_workspace_bytes", "sb_rank_features_workspace_bytes"):
+                 "sb_verify_accept_workspace_bytes", "sb_rank_features_workspace_bytes",
+                 "sb_verify_sample_workspace_bytes"):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
-                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal"):
+                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal", "sb_verify_sample"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -74,7 +75,8 @@ def load(build_if_missing: bool = True):
 EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspace_bytes",
             "sb_tree_expand", "sb_tree_expand_workspace_bytes", "sb_verify_accept",
             "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
-            "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_verifier_signal", "sb_status_string",
+            "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_verifier_signal", "sb_verify_sample",
+            "sb_verify_sample_workspace_bytes", "sb_status_string",
             "sb_version",
             "sb_kernel_launch_count")
 
@@ -269,6 +271,38 @@ def sb_verifier_signal(scores, node_offsets, child_row, path_nodes, accept_len, 
         _stream())
     _check(rc, "sb_verifier_signal")
     return dict(r_prob=r_prob, signal=signal, status=status)
+
+
+def sb_verify_sample_workspace_bytes(batch: int, vocab: int) -> int:
+    return int(load().sb_verify_sample_workspace_bytes(C.c_int32(batch), C.c_int32(vocab)))
+
+
+def sb_verify_sample(logits, scores, node_offsets, parent, tok, child_row, temperature, u_accept, u_bonus, max_depth,
+                     *, vocab=None, workspace=None, out=None):
+    """Stochastic tree verification (temperature > 0); the uniforms are inputs.
+    -> dict(accept_len, path_nodes, out_tokens, bonus, status)."""
+    total, stride = logits.shape
+    n_rows, sstride = scores.shape
+    vocab = stride if vocab is None else vocab
+    batch = node_offsets.numel() - 1
+    dev = logits.device
+    dt = {torch.bfloat16: SB_BF16, torch.float32: SB_F32}[logits.dtype]
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=dev)
+        out = dict(accept_len=torch.empty(batch, **i32), path_nodes=torch.empty((batch, max_depth + 1), **i32),
+                   out_tokens=torch.empty((batch, max_depth + 1), **i32), bonus=torch.empty(batch, **i32),
+                   status=torch.empty(batch, **i32))
+    if workspace is None:
+        workspace = torch.empty(max(sb_verify_sample_workspace_bytes(batch, vocab), 16), dtype=torch.uint8, device=dev)
+    rc = load().sb_verify_sample(
+        _ptr(logits), C.c_int(dt), C.c_int64(stride), C.c_int32(vocab), _ptr(scores, torch.float32), C.c_int64(sstride),
+        C.c_int32(n_rows), C.c_int32(batch), C.c_int32(total), _ptr(node_offsets, torch.int32),
+        _ptr(parent, torch.int32), _ptr(tok, torch.int32), _ptr(child_row, torch.int32), C.c_float(temperature),
+        _ptr(u_accept, torch.float32), _ptr(u_bonus, torch.float32), C.c_int32(max_depth), _ptr(out["accept_len"]),
+        _ptr(out["path_nodes"]), _ptr(out["out_tokens"]), _ptr(out["bonus"]), _ptr(workspace),
+        C.c_size_t(workspace.numel()), _ptr(out["status"]), _stream())
+    _check(rc, "sb_verify_sample")
+    return out
 
 
 SB_STATIC_SCRATCH_BYTES = 256 * 1024

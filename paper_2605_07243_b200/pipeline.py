@@ -145,6 +145,30 @@ class VerifyStep:
                                      self.accept["accept_len"], self.accept["bonus"], self.max_depth, e["signal"],
                                      r_prob=e["r_prob"], status=e["signal_status"])
 
+    def run_sample(self, temperature=1.0):
+        """Stochastic (temperature > 0) verification of the same tree and logits (not part of run_device():
+        a 'next' row, timed on its own); drafter rows are mapped as in run_signal(), the uniforms are fixed."""
+        e = self.expand
+        if e is None:
+            return None
+        if "sample_out" not in e:
+            self.run_signal()
+            n, B = int(self.tb.total_nodes), self.tb.prefix_len.numel()
+            gen = torch.Generator(device="cpu").manual_seed(1234)
+            e["u_accept"] = torch.rand(n, generator=gen).to(self.device)
+            e["u_bonus"] = torch.rand(B, generator=gen).to(self.device)
+            V = self.logits.shape[1]
+            e["sample_ws"] = torch.empty(max(16, sb.sb_verify_sample_workspace_bytes(B, V)), dtype=torch.uint8,
+                                         device=self.device)
+            i32 = dict(dtype=torch.int32, device=self.device)
+            e["sample_out"] = dict(accept_len=torch.empty(B, **i32),
+                                   path_nodes=torch.empty((B, self.max_depth + 1), **i32),
+                                   out_tokens=torch.empty((B, self.max_depth + 1), **i32),
+                                   bonus=torch.empty(B, **i32), status=torch.empty(B, **i32))
+        return sb.sb_verify_sample(self.logits, e["scores"], self.tb.node_offsets, self.tb.parent, self.tok,
+                                   e["child_row"], temperature, e["u_accept"], e["u_bonus"], self.max_depth,
+                                   workspace=e["sample_ws"], out=e["sample_out"])
+
     def run_attention(self, layers=None):
         for l in range(self.n_layers) if layers is None else layers:
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,

@@ -434,3 +434,134 @@ def test_verifier_signal_unaligned_rows_and_host_errors():
     with pytest.raises(sb.SbError):
         sb.sb_verifier_signal(t, dev.i32_tensor(node_offsets), dev.i32_tensor(child_row), dev.i32_tensor(path),
                               dev.i32_tensor(accept_len), dev.i32_tensor([1, 1]), 99, sig)
+
+
+# ---- stochastic verification (temperature > 0) ---------------------------------------------------------------
+
+def _robust_uniforms(rng, case_args, temperature, max_depth, total, batch, vocab=None, eps=2e-3, tries=40):
+    """Acceptance uniforms whose every decision in the oracle has a relative margin of eps: the walk is
+    the same with all of them scaled by 1 - eps and 1 + eps (acceptance is monotone in u, so the three
+    runs follow the same path and every comparison on it holds with that margin).  The GPU decides
+    in fp32 (about 1e-5 relative on a ratio of sums over the vocabulary)."""
+    u_b = rng.random(batch).astype(np.float32) * np.float32(0.98) + np.float32(0.01)
+    for _ in range(tries):
+        u_a = rng.random(total).astype(np.float32) * np.float32(0.98) + np.float32(0.01)
+        runs = [oracle.verify_sample(*case_args, temperature, (u_a * np.float32(s)).astype(np.float32), u_b,
+                                     max_depth, vocab=vocab) for s in (1.0, 1.0 - eps, 1.0 + eps)]
+        if all(np.array_equal(runs[0][k], r[k]) for r in runs[1:] for k in ("status", "accept_len", "path_nodes")):
+            return u_a, u_b, runs[0]
+    raise AssertionError("no robust uniforms found")
+
+
+def _check_sample(rng, logits, scores, node_offsets, parent, tok, child_row, temperature, max_depth, vocab=None,
+                  delta=1e-3):
+    """The walk (status, accept_len, path, accepted tokens) must equal the oracle's.  The bonus token is
+    an inverse-CDF draw whose cell can be far narrower than fp32 sums over the vocabulary resolve, so it
+    is checked as a draw: it must lie between the oracle's draws for u_bonus (1 - delta) and (1 + delta)
+    (the draw is monotone in u_bonus)."""
+    total = len(parent)
+    batch = len(node_offsets) - 1
+    args = (logits, scores, node_offsets, parent, tok, child_row)
+    u_a, u_b, ref = _robust_uniforms(rng, args, temperature, max_depth, total, batch, vocab=vocab)
+    got = sb.sb_verify_sample(_logits_tensor(logits), torch.from_numpy(np.ascontiguousarray(scores)).cuda(),
+                              dev.i32_tensor(node_offsets), dev.i32_tensor(parent), dev.i32_tensor(tok),
+                              dev.i32_tensor(child_row), temperature, torch.from_numpy(u_a).cuda(),
+                              torch.from_numpy(u_b).cuda(), max_depth, vocab=vocab)
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in got.items()}
+    for key in ("status", "accept_len", "path_nodes"):
+        np.testing.assert_array_equal(got[key], ref[key], err_msg=key)
+    lo = oracle.verify_sample(*args, temperature, u_a, (u_b * np.float32(1 - delta)).astype(np.float32), max_depth,
+                              vocab=vocab)["bonus"]
+    hi = oracle.verify_sample(*args, temperature, u_a, (u_b * np.float32(1 + delta)).astype(np.float32), max_depth,
+                              vocab=vocab)["bonus"]
+    for b in range(batch):
+        a = int(ref["accept_len"][b])
+        if ref["status"][b] != 0:
+            np.testing.assert_array_equal(got["out_tokens"][b], ref["out_tokens"][b])
+            assert got["bonus"][b] == ref["bonus"][b] == -1
+            continue
+        np.testing.assert_array_equal(got["out_tokens"][b, :a], ref["out_tokens"][b, :a])
+        assert lo[b] <= got["bonus"][b] <= hi[b], (b, lo[b], got["bonus"][b], hi[b])
+        assert got["out_tokens"][b, a] == got["bonus"][b] and (got["out_tokens"][b, a + 1:] == -1).all()
+    return ref, got
+
+
+def _sample_case(rng, parents, vocab, dtype, std=2.0, stride_pad=0):
+    """Target logits that favour the drafted tokens (so that walks go deep) and drafter scores that
+    favour them too; child_row = the node's own index."""
+    n_nodes = [len(p) for p in parents]
+    total = sum(n_nodes)
+    node_offsets = np.concatenate([[0], np.cumsum(n_nodes)]).astype(np.int32)
+    parent = np.concatenate(parents).astype(np.int32)
+    tok = np.zeros(total, np.int32)
+    logits = (rng.standard_normal((total, vocab + stride_pad), dtype=np.float32) * std).astype(np.float32)
+    scores = (rng.standard_normal((total, vocab + stride_pad), dtype=np.float32) * std).astype(np.float32)
+    if stride_pad:
+        logits[:, vocab:] = 1e9
+        scores[:, vocab:] = 1e9
+    for b, par in enumerate(parents):
+        o = node_offsets[b]
+        for a in range(len(par)):
+            kids = [c for c in range(len(par)) if par[c] == a]
+            toks = rng.choice(vocab, size=len(kids), replace=False) if kids else []
+            for c, t in zip(kids, toks):
+                tok[o + c] = t
+                logits[o + a, t] += 6.0 + rng.random() * 2          # the target likes its children ...
+                scores[o + a, t] += 5.0 + rng.random() * 3          # ... and so does the drafter
+    child_row = np.arange(total, dtype=np.int32)
+    if dtype == "bf16":
+        logits = W.f32_to_bf16_bits(logits)
+    return logits, scores, node_offsets, parent, tok, child_row
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_verify_sample_matches_oracle_small_vocab(dtype):
+    rng = W.rng_for(110)
+    parents = [W.random_tree(rng, 40, 7), W.chain_tree(6), np.asarray([-1], np.int32), W.random_tree(rng, 128, 12)]
+    case = _sample_case(rng, parents, 1000, dtype, stride_pad=3)
+    depths = set()
+    exact = 0
+    for rep in range(6):
+        ref, got = _check_sample(rng, *case, temperature=1.0, max_depth=8, vocab=1000)
+        depths.update(int(a) for a in ref["accept_len"])
+        exact += int((got["bonus"] == ref["bonus"]).sum())
+    assert len(depths) >= 3, depths          # the walks really differ: rejections, residual draws, deep accepts
+    assert exact >= 20, exact                # and almost every bonus draw is the oracle's own (24 draws)
+    _check_sample(rng, *case, temperature=0.5, max_depth=3, vocab=1000)
+    _check_sample(rng, *case, temperature=2.0, max_depth=8, vocab=1000)
+
+
+def test_verify_sample_full_vocabulary_config2_tree():
+    rng = W.rng_for(111)
+    par = W.config2_tree()
+    case = _sample_case(rng, [par], 128256, "bf16")
+    for rep in range(2):
+        _check_sample(rng, *case, temperature=1.0, max_depth=8)
+
+
+def test_verify_sample_errors_and_degenerate_rows():
+    rng = W.rng_for(112)
+    parents = [W.random_tree(rng, 12, 4), W.random_tree(rng, 9, 3), W.chain_tree(4)]
+    logits, scores, node_offsets, parent, tok, child_row = _sample_case(rng, parents, 257, "f32")
+    bad_parent = parent.copy()
+    bad_parent[node_offsets[1] + 3] = 5                  # parent index not below its child
+    child_row2 = child_row.copy()
+    child_row2[node_offsets[2]] = -1                     # the chain's root has children but no drafter row
+    logits2 = logits.copy()
+    logits2[0, :] = np.nan                               # a target row without a finite value: flat
+    scores2 = scores.copy()
+    scores2[0, :] = -np.inf
+    ref, _ = _check_sample(rng, logits2, scores2, node_offsets, bad_parent, tok, child_row2, temperature=1.0, max_depth=6)
+    assert list(ref["status"]) == [0, 4, 5]
+    t = torch.from_numpy(logits).cuda()
+    s = torch.from_numpy(scores).cuda()
+    u = torch.zeros(len(parent), dtype=torch.float32, device="cuda")
+    ub = torch.zeros(3, dtype=torch.float32, device="cuda")
+    with pytest.raises(sb.SbError):
+        sb.sb_verify_sample(t, s, dev.i32_tensor(node_offsets), dev.i32_tensor(parent), dev.i32_tensor(tok),
+                            dev.i32_tensor(child_row), 0.0, u, ub, 6)
+    with pytest.raises(sb.SbError):
+        sb.sb_verify_sample(t, s, dev.i32_tensor(node_offsets), dev.i32_tensor(parent), dev.i32_tensor(tok),
+                            dev.i32_tensor(child_row), 1.0, u, ub, 6,
+                            workspace=torch.empty(64, dtype=torch.uint8, device="cuda"))
