@@ -303,3 +303,30 @@ def test_two_tiles_per_cta_long_chunks(monkeypatch):
                             prefix_lens=[6000, 3001], n_q_heads=32, n_kv_heads=8, head_dim=128, page_size=64, q_std=4.0)
     check_attention(case, "two tiles: long chunks, peaky", num_splits=1)
     check_attention(case, "two tiles: long chunks, peaky, 2 chunks", num_splits=2)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_shapes_against_oracle(seed, monkeypatch):
+    """Seeded random shapes: batch, head layout, head_dim, page size, tree sizes, prefix lengths, query
+    range, chunk count and kernel variant all drawn at random; element-wise parity on every one."""
+    rng = W.rng_for(9000 + seed)
+    B = int(rng.integers(1, 5))
+    hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 3, 4, 8]))
+    D = int(rng.choice([64, 128]))
+    page = int(rng.choice([0, 0, 16, 64, 128, 256]))
+    parents, prefix, qbegin = [], [], []
+    for _ in range(B):
+        n = int(rng.integers(1, 129))
+        parents.append(W.random_tree(rng, n, int(rng.integers(1, 14))))
+        prefix.append(int(rng.choice([0, 1, 15, 16, 17, 127, 128, 129, int(rng.integers(0, 3000))])))
+        qbegin.append(int(rng.integers(0, n)) if rng.random() < 0.3 else 0)
+    use_qbegin = any(qbegin)
+    case = W.make_attn_case(rng, parents=parents, prefix_lens=prefix, n_q_heads=hkv * G, n_kv_heads=hkv, head_dim=D,
+                            page_size=page, q_node_begin=qbegin if use_qbegin else None,
+                            q_std=float(rng.choice([1.0, 1.0, 4.0])), capacity_pad=int(rng.integers(0, 40)))
+    splits = int(rng.choice([0, 0, 1, 2, 3, 5, 8, 16]))
+    if rng.random() < 0.4:
+        monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
+    check_attention(case, f"random shape {seed}: B={B} Hkv={hkv} G={G} D={D} page={page} splits={splits}",
+                    num_splits=splits)
