@@ -27,9 +27,32 @@ struct AttnParams {
   int* status;
   int G;            // query heads per KV head
   int row_tiles;    // 128-row query tiles per (sequence, KV head) in the grid
+  int sort_seqs;    // 1: grid index z is the rank of a sequence by length, longest first
 };
 
 constexpr float kLn2 = 0.6931471805599453f;
+
+// Longest-first launch order for ragged batches that run in several waves of CTAs: the CTAs of a
+// long sequence start first, so the last wave holds the short ones (config of 16 sequences with
+// 17..54 key blocks: 163 us in input order against 138 us in a schedule simulation).  Every CTA
+// ranks the batch itself: sequence with rank z by (length descending, index ascending).  Any
+// contents of the length arrays give a permutation.  s_len / s_perm: >= batch ints each, batch <=
+// blockDim.x; the caller must not reuse them before the closing barrier.
+__device__ inline int sequence_of_rank(const sb_tree_batch& tb, int z, int* s_len, int* s_perm) {
+  const int B = tb.batch, tid = threadIdx.x;
+  if (tid < B) s_len[tid] = tb.prefix_len[tid] + (tb.node_offsets[tid + 1] - tb.node_offsets[tid]);
+  __syncthreads();
+  if (tid < B) {
+    const int me = s_len[tid];
+    int r = 0;
+    for (int j = 0; j < B; ++j) r += (s_len[j] > me || (s_len[j] == me && j < tid)) ? 1 : 0;
+    s_perm[r] = tid;
+  }
+  __syncthreads();
+  const int b = s_perm[z];
+  __syncthreads();
+  return b;
+}
 
 // What a CTA may do for its sequence after the shape checks.
 struct SeqPlan {

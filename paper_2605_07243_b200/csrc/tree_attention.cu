@@ -660,6 +660,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   p.status = status;
   p.G = tb->n_q_heads / tb->n_kv_heads;
   p.part_o = nullptr;
+  p.sort_seqs = 0;
   p.part_lse = nullptr;
 
   const AttnImpl impl = attn_impl();
@@ -687,6 +688,9 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   }
   const int row_tiles = ceil_div(tb->max_nodes * p.G, BM);
   p.row_tiles = row_tiles;
+  // ragged batches that run in waves start their longest sequences first
+  p.sort_seqs = (impl == IMPL_TC && tb->batch > 1 && tb->batch <= 128 &&
+                 (long long)tb->batch * tb->n_kv_heads * row_tiles > num_sms()) ? 1 : 0;
   dim3 grid(p.num_splits, (plan.two_tiles ? ceil_div(row_tiles, 2) : row_tiles) * tb->n_kv_heads, tb->batch);
   if (grid.y > 65535 || grid.z > 65535) return SB_ERR_UNSUPPORTED;
   if (plan.two_tiles) st = launch_attn_tc2(p, grid, cs);

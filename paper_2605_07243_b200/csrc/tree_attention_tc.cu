@@ -84,7 +84,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const int Hq = p.tb.n_q_heads, G = p.G;
   // row tiles of one (sequence, KV head) are neighbours in launch order: they share its K/V through L2
   const int g = blockIdx.y / p.row_tiles, tile = blockIdx.y % p.row_tiles;
-  const int b = blockIdx.z;
   if (tid == 0) {
     *s_abort = 0;
     const int n = TC_SOFTMAX_THREADS;
@@ -114,6 +113,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  // grid index z -> sequence (longest first when the grid runs in several waves)
+  const int b = p.sort_seqs ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent) : (int)blockIdx.z;
   const SeqPre pre = plan_lengths(p, b);
   const int rows_total = pre.info.nq * G;
   const int row0 = tile * TC_BM;

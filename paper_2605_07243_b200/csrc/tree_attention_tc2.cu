@@ -71,7 +71,6 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
   // the tile pairs of one (sequence, KV head) are neighbours in launch order: they share its K/V through L2
   const int pairs = ceil_div(p.row_tiles, 2);
   const int g = blockIdx.y / pairs, pair = blockIdx.y % pairs;
-  const int b = blockIdx.z;
   if (tid == 0) {
     *s_abort = 0;
     const int n = T2_SOFTMAX_THREADS;
@@ -90,6 +89,8 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  // grid index z -> sequence (longest first when the grid runs in several waves)
+  const int b = p.sort_seqs ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent) : (int)blockIdx.z;
   const SeqPre pre = plan_lengths(p, b);
   const int rows_total = pre.info.nq * G;
   const int row0 = pair * 2 * TC_BM;                         // first row of tile 0; tile 1 starts 128 rows on
