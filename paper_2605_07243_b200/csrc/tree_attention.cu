@@ -497,6 +497,15 @@ static SplitPlan plan_for(int s, bool oversubscribed) {
 
 enum AttnImpl { IMPL_TC = 0, IMPL_MMA = 1, IMPL_SIMPLE = 2 };
 
+// Upper bound of the 128-row query tiles any (sequence, KV head) needs: a sequence has at most
+// max_nodes query nodes and never more than there are query rows in the whole batch (a drafter
+// block that only queries its newest nodes stays at one tile although its tree is larger).
+static int max_row_tiles(const sb_tree_batch* tb, int total_q) {
+  const int G = tb->n_q_heads / tb->n_kv_heads;
+  const int nq = tb->max_nodes < total_q ? tb->max_nodes : total_q;
+  return ceil_div((nq > 0 ? nq : 1) * G, BM);
+}
+
 static AttnImpl attn_impl() {
   const char* impl = getenv("SB_ATTN_IMPL");
   if (impl && strcmp(impl, "simple") == 0) return IMPL_SIMPLE;
@@ -509,8 +518,7 @@ static AttnImpl attn_impl() {
 // chunks of a few KV blocks to even out ragged prefix lengths.  The chunks are grouped into
 // clusters of the largest divisor <= 8.  `granule` is the kernel's key-block size.
 static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_splits, AttnImpl impl) {
-  const int G = tb->n_q_heads / tb->n_kv_heads;
-  const int row_tiles = ceil_div(tb->max_nodes * G, BM);
+  const int row_tiles = max_row_tiles(tb, total_q);
   const int granule = impl == IMPL_TC ? 128 : BN;
   const int max_blocks = ceil_div(tb->max_kv_len, granule);
   const long long base = (long long)tb->batch * tb->n_kv_heads * row_tiles;
@@ -572,16 +580,27 @@ static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_spl
     }
     return plan_for(best, true);
   }
-  int s = (int)(sms / base);
-  if (s > max_blocks) s = max_blocks;
-  for (; s > 1; --s) {
+  // Few tiles: one wave.  Among the chunk counts whose clusters are all resident at once, take the
+  // cheapest under: blocks per chunk x 1.2 us, plus 6 us when the chunks of a tile do not fit one
+  // cluster (fp32 partials and the merge launch) -- 33 blocks over 8 KV heads: 8 chunks in one
+  // cluster of 8 (14.4 us) rather than 15 chunks in 3 clusters of 5 (22.7 us).
+  int s_max = (int)(sms / base);
+  if (s_max > max_blocks) s_max = max_blocks;
+  SplitPlan best = plan_for(1, false);
+  double best_cost = 1.2 * max_blocks;
+  for (int s = 2; s <= s_max; ++s) {
     const SplitPlan sp = plan_for(s, false);
     if (sp.outer > 1 && sp.cluster < 4) continue;  // partial traffic for little gain
     const int fit = impl == IMPL_TC ? attn_tc_max_active_clusters(tb->head_dim, sp.cluster)
                                     : max_active_clusters(tb->head_dim, sp.cluster);
-    if (fit <= 0 || base * sp.outer <= fit) return sp;
+    if (fit > 0 && base * sp.outer > fit) continue;
+    const double cost = 1.2 * ceil_div(max_blocks, s) + (sp.outer > 1 ? 6.0 : 0.0);
+    if (cost <= best_cost + 1e-9) {  // ties: more chunks (smaller merge slices per CTA)
+      best = sp;
+      best_cost = cost;
+    }
   }
-  return plan_for(1, false);
+  return best;
 }
 
 static size_t workspace_bytes_for(const sb_tree_batch* tb, int total_q, int outer) {
@@ -686,7 +705,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
     p.part_o = static_cast<float*>(workspace);
     p.part_lse = reinterpret_cast<float*>(static_cast<char*>(workspace) + o);
   }
-  const int row_tiles = ceil_div(tb->max_nodes * p.G, BM);
+  const int row_tiles = max_row_tiles(tb, total_q);
   p.row_tiles = row_tiles;
   // ragged batches that run in waves start their longest sequences first
   p.sort_seqs = (impl == IMPL_TC && tb->batch > 1 && tb->batch <= 128 &&
