@@ -14,6 +14,7 @@ from .oracle import (  # noqa: F401
     verify_accept,
     verifier_signal,
     verify_sample,
+    shift_project,
     accept_from_amax,
     kv_compact,
     tree_expand,

@@ -139,6 +139,18 @@ def rank_features(scores, vocab=None):
     return feats
 
 
+def shift_project(h, w, block_k):
+    """h uint16 (bf16 bits) [R, d], w uint16 [d_out, 2d] (block_k > 0) or [d_out, d] (block_k = 0) -> f64 [R, d_out]."""
+    h = np.ascontiguousarray(h, np.uint16)
+    w = np.ascontiguousarray(w, np.uint16)
+    n_rows, d = h.shape
+    d_out, kin = w.shape
+    assert kin == (2 * d if block_k > 0 else d)
+    out = np.zeros((n_rows, d_out), np.float64)
+    _load().sbo_shift_project(_p(h), _p(w), C.c_int(n_rows), C.c_int(d), C.c_int(d_out), C.c_int(block_k), _p(out))
+    return out
+
+
 def verifier_signal(scores, node_offsets, child_row, path_nodes, accept_len, bonus, max_depth, signal=None,
                     vocab=None):
     """-> dict(r_prob f64 [B], signal f64 [B] (= signal in + 1 - r), status int32 [B])."""

@@ -28,6 +28,8 @@
  *                         names the procedure only as "rejection sampling": the order in which siblings
  *                         are tried and the treatment of the draft distribution after a rejection are
  *                         readings -- for those PARITY IS UNPINNED by the paper.
+ *   sbo_shift_project   : numpy matmul on the explicitly concatenated input; W = [I, 0] returns the input,
+ *                         W = [0, I] the previous position's state (the first position its own).
  *   sbo_tree_expand     : hand-derived trees for the two printed branching maps; chain special
  *                         case; structural invariants.  The attach point of siblings, the cut
  *                         order at the node budget and the treatment of b = 0 are readings of
@@ -500,6 +502,34 @@ void sbo_rank_features(const float* scores, int64_t row_stride, int n_rows, int 
     f[13] = exp(e[0].val - log_z);
     f[14] = entropy;
     free(e);
+  }
+}
+
+/* ---- layer-wise shift between the drafter's decoder layers (Sec. 3.1, the equation for h-tilde) -- */
+
+/*
+ * Rows r = i * block_k + k are the K positions of block i.  Before the next layer, position k's
+ * state is concatenated with position k-1's state of the same block (the first position with its
+ * own) and projected back to d_out features:
+ *   out[r][f] = sum_j w[f][j] * h[r][j] + sum_j w[f][d + j] * h[prev(r)][j],
+ *   prev(r) = r - 1 if r % block_k != 0 else r.
+ * h bf16 [n_rows][d], w bf16 [d_out][2 d] (the projection acting on the concatenation), out f64.
+ * block_k = 0: plain projection out = h w^T with w [d_out][d].
+ */
+void sbo_shift_project(const uint16_t* h, const uint16_t* w, int n_rows, int d, int d_out, int block_k,
+                       double* out) {
+  const int kin = block_k > 0 ? 2 * d : d;
+#pragma omp parallel for schedule(static)
+  for (int r = 0; r < n_rows; ++r) {
+    const int prev = (block_k > 0 && r % block_k != 0) ? r - 1 : r;
+    for (int f = 0; f < d_out; ++f) {
+      double acc = 0.0;
+      for (int j = 0; j < d; ++j) acc += bf16_to_f64(w[(int64_t)f * kin + j]) * bf16_to_f64(h[(int64_t)r * d + j]);
+      if (block_k > 0)
+        for (int j = 0; j < d; ++j)
+          acc += bf16_to_f64(w[(int64_t)f * kin + d + j]) * bf16_to_f64(h[(int64_t)prev * d + j]);
+      out[(int64_t)r * d_out + f] = acc;
+    }
   }
 }
 

@@ -588,3 +588,28 @@ def test_verify_sample_low_temperature_is_greedy_and_walks_the_tree():
     no_row = oracle.verify_sample(ver.logits, scores, ver.node_offsets, ver.parent, ver.tok, np.full(n, -1, np.int32),
                                   1.0, np.zeros(n, np.float32), [0.5], 3)
     assert no_row["status"][0] == 5
+
+
+# ---- layer-wise shift projection between drafter layers (Sec. 3.1) ---------------------------------------------
+
+def test_shift_project_matches_numpy_on_the_concatenated_input():
+    rng = W.rng_for(38)
+    R, K, d, d_out = 12, 4, 96, 40
+    h = W.f32_to_bf16_bits(rng.standard_normal((R, d), dtype=np.float32))
+    w = W.f32_to_bf16_bits(rng.standard_normal((d_out, 2 * d), dtype=np.float32) * 0.1)
+    hf = W.bf16_bits_to_f32(h).astype(np.float64)
+    wf = W.bf16_bits_to_f32(w).astype(np.float64)
+    prev = np.asarray([r - 1 if r % K else r for r in range(R)])
+    want = np.concatenate([hf, hf[prev]], axis=1) @ wf.T          # library matmul on [h_k, h_{k-1}]
+    np.testing.assert_allclose(oracle.shift_project(h, w, K), want, rtol=1e-12, atol=1e-12)
+    # plain projection
+    w1 = W.f32_to_bf16_bits(rng.standard_normal((d_out, d), dtype=np.float32))
+    np.testing.assert_allclose(oracle.shift_project(h, w1, 0), hf @ W.bf16_bits_to_f32(w1).astype(np.float64).T,
+                               rtol=1e-12, atol=1e-12)
+    # W = [I, 0] returns the input; W = [0, I] returns the previous position's state, and the
+    # first position of a block gets its own (the convention h_0 = h_1)
+    eye = np.eye(d, dtype=np.float32)
+    zero = np.zeros((d, d), np.float32)
+    np.testing.assert_array_equal(oracle.shift_project(h, W.f32_to_bf16_bits(np.hstack([eye, zero])), K), hf)
+    np.testing.assert_array_equal(oracle.shift_project(h, W.f32_to_bf16_bits(np.hstack([zero, eye])), K), hf[prev])
+    assert (prev[::K] == np.arange(0, R, K)).all()
