@@ -13,6 +13,7 @@
  *   sb_rank_features   15-dim summary of each draft distribution        (Sec. 3.2, App. B)
  *   sb_verifier_signal verifier-derived update signal s = sum (1 - r)   (Sec. 3.4, Alg. 2)
  *   sb_verify_sample   stochastic (temperature > 0) tree verification   (Sec. 4.1, Sec. 4.2)
+ *   sb_shift_project   layer-wise shift projection between drafter layers (Sec. 3.1)
  *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
  *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
  *
@@ -186,6 +187,27 @@ size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab);
 sb_status sb_rank_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
                            float* features, void* workspace, size_t workspace_bytes, void* stream);
 size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
+
+/*
+ * sb_shift_project -- the layer-wise shift between consecutive decoder layers of the drafter
+ * (Sec. 3.1 "Within-block dependence", the equation for h-tilde): position k's state is
+ * concatenated with position k-1's state of the same block and projected back by W_shift.
+ *
+ *   h   bf16 [n_rows][d]: rows r = i * block_k + k are the block_k positions of block i.
+ *   w   bf16 [d_out][2 d] row-major: W_shift acting on the concatenation [h_k , h_{k-1}].
+ *   out bf16 [n_rows][d_out]: out[r] = w[:, :d] h[r] + w[:, d:] h[prev(r)], prev(r) = r - 1 inside a
+ *       block and r at its first position (the convention h_0 = h_1); fp32 accumulation.
+ *   block_k = 0: plain projection out = h w^T with w [d_out][d] (e.g. W_cond of the block forward).
+ *   Limits: n_rows <= 128, d a multiple of 64, d_out a multiple of 128, h and w 16-byte aligned.
+ *   workspace: sb_shift_project_workspace_bytes(...) bytes, 256-byte aligned (fp32 partials of the
+ *   K splits and one word that outlives the call: hand the same workspace to every call, or a zeroed
+ *   one).  status int32 [1]: SB_OK, or SB_ERR_CUDA if a bounded device wait gave up.
+ *   HBM-bound on the weights: 2 * d * d_out * 2 bytes are read once.
+ */
+sb_status sb_shift_project(const void* h, const void* w, int32_t n_rows, int32_t d, int32_t d_out,
+                           int32_t block_k, void* out, void* workspace, size_t workspace_bytes,
+                           int32_t* status, void* stream);
+size_t sb_shift_project_workspace_bytes(int32_t n_rows, int32_t d, int32_t d_out, int32_t block_k);
 
 /*
  * sb_verify_sample -- verification at temperature T > 0 by multi-candidate rejection sampling over

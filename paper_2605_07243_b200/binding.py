@@ -63,10 +63,11 @@ def load(build_if_missing: bool = True):
     lib.sb_kernel_launch_count.restype = C.c_int64
     for name in ("sb_tree_attention_workspace_bytes", "sb_tree_expand_workspace_bytes",
                  "sb_verify_accept_workspace_bytes", "sb_rank_features_workspace_bytes",
-                 "sb_verify_sample_workspace_bytes"):
+                 "sb_verify_sample_workspace_bytes", "sb_shift_project_workspace_bytes"):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
-                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal", "sb_verify_sample"):
+                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal", "sb_verify_sample",
+                 "sb_shift_project"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -76,7 +77,8 @@ EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspa
             "sb_tree_expand", "sb_tree_expand_workspace_bytes", "sb_verify_accept",
             "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
             "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_verifier_signal", "sb_verify_sample",
-            "sb_verify_sample_workspace_bytes", "sb_status_string",
+            "sb_verify_sample_workspace_bytes", "sb_shift_project", "sb_shift_project_workspace_bytes",
+            "sb_status_string",
             "sb_version",
             "sb_kernel_launch_count")
 
@@ -303,6 +305,30 @@ def sb_verify_sample(logits, scores, node_offsets, parent, tok, child_row, tempe
         C.c_size_t(workspace.numel()), _ptr(out["status"]), _stream())
     _check(rc, "sb_verify_sample")
     return out
+
+
+def sb_shift_project_workspace_bytes(n_rows: int, d: int, d_out: int, block_k: int) -> int:
+    return int(load().sb_shift_project_workspace_bytes(C.c_int32(n_rows), C.c_int32(d), C.c_int32(d_out),
+                                                       C.c_int32(block_k)))
+
+
+def sb_shift_project(h, w, block_k, *, out=None, workspace=None, status=None):
+    """h bf16 [R, d], w bf16 [d_out, 2d] (block_k > 0) or [d_out, d] (block_k = 0) -> out bf16 [R, d_out]."""
+    n_rows, d = h.shape
+    d_out = w.shape[0]
+    dev = h.device
+    out = torch.empty((n_rows, d_out), dtype=torch.bfloat16, device=dev) if out is None else out
+    status = torch.zeros(1, dtype=torch.int32, device=dev) if status is None else status
+    if w.shape[1] != (2 * d if block_k > 0 else d):
+        raise ValueError("w must be [d_out, 2d] with block_k > 0 and [d_out, d] with block_k = 0")
+    if workspace is None:
+        workspace = torch.zeros(max(sb_shift_project_workspace_bytes(n_rows, d, d_out, block_k), 256), dtype=torch.uint8,
+                                device=dev)
+    rc = load().sb_shift_project(_ptr(h, torch.bfloat16), _ptr(w, torch.bfloat16), C.c_int32(n_rows), C.c_int32(d),
+                                 C.c_int32(d_out), C.c_int32(block_k), _ptr(out, torch.bfloat16), _ptr(workspace),
+                                 C.c_size_t(workspace.numel()), _ptr(status, torch.int32), _stream())
+    _check(rc, "sb_shift_project")
+    return out, status
 
 
 SB_STATIC_SCRATCH_BYTES = 256 * 1024

@@ -169,6 +169,30 @@ class VerifyStep:
                                    e["child_row"], temperature, e["u_accept"], e["u_bonus"], self.max_depth,
                                    workspace=e["sample_ws"], out=e["sample_out"])
 
+    SHIFT_SETS = 4   # weight matrices rotated per run_shift_all(): 4 x 64 MB > L2
+
+    def run_shift_all(self, d=4096, block_k=4):
+        """The drafter's layer-wise shift projection on the expansion's rows (not part of run_device():
+        a 'next' row, timed on its own), once per weight matrix of a rotating set so that the weights
+        come from HBM every time."""
+        e = self.expand
+        if e is None:
+            return None
+        if "shift_w" not in e:
+            R = e["scores"].shape[0]
+            gen = torch.Generator(device="cpu").manual_seed(4321)
+            e["shift_h"] = torch.randn(R, d, generator=gen).to(torch.bfloat16).to(self.device)
+            e["shift_w"] = [(torch.randn(d, 2 * d, generator=gen) * 0.02).to(torch.bfloat16).to(self.device)
+                            for _ in range(self.SHIFT_SETS)]
+            e["shift_out"] = torch.empty(R, d, dtype=torch.bfloat16, device=self.device)
+            e["shift_ws"] = torch.zeros(sb.sb_shift_project_workspace_bytes(R, d, d, block_k), dtype=torch.uint8,
+                                        device=self.device)
+            e["shift_status"] = torch.zeros(1, dtype=torch.int32, device=self.device)
+        for w in e["shift_w"]:
+            sb.sb_shift_project(e["shift_h"], w, block_k, out=e["shift_out"], workspace=e["shift_ws"],
+                                status=e["shift_status"])
+        return e["shift_out"]
+
     def run_attention(self, layers=None):
         for l in range(self.n_layers) if layers is None else layers:
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,

@@ -565,3 +565,50 @@ def test_verify_sample_errors_and_degenerate_rows():
         sb.sb_verify_sample(t, s, dev.i32_tensor(node_offsets), dev.i32_tensor(parent), dev.i32_tensor(tok),
                             dev.i32_tensor(child_row), 1.0, u, ub, 6,
                             workspace=torch.empty(64, dtype=torch.uint8, device="cuda"))
+
+
+# ---- layer-wise shift projection (Sec. 3.1) -----------------------------------------------------------------
+
+def _check_shift(rng, R, d, d_out, K, w_std=0.02):
+    h = W.f32_to_bf16_bits(rng.standard_normal((R, d), dtype=np.float32))
+    w = W.f32_to_bf16_bits(rng.standard_normal((d_out, 2 * d if K > 0 else d), dtype=np.float32) * np.float32(w_std))
+    got, status = sb.sb_shift_project(dev.bf16_tensor(h), dev.bf16_tensor(w), K)
+    torch.cuda.synchronize()
+    assert int(status.cpu()[0]) == 0
+    got = got.float().cpu().numpy().astype(np.float64)
+    ref = oracle.shift_project(h, w, K)
+    err = np.abs(got - ref)
+    tol = 1e-2 + 1e-2 * np.abs(ref)          # bf16 output of an fp32 accumulation
+    assert (err <= tol).all(), f"max err {err.max():.3e} at |ref| {np.abs(ref).flat[err.argmax()]:.3e}"
+    return got, ref
+
+
+@pytest.mark.parametrize("R,K", [(32, 4), (4, 4), (60, 4), (128, 8), (17, 1)])
+def test_shift_project_8b_shape(R, K):
+    """d = d_out = 4096 (the 8B drafter's width): 64 MB of weights streamed once."""
+    _check_shift(W.rng_for(120 + R), R, 4096, 4096, K)
+
+
+@pytest.mark.parametrize("d,d_out", [(64, 128), (192, 384), (1024, 256), (5120, 128)])
+def test_shift_project_other_shapes_and_plain_projection(d, d_out):
+    rng = W.rng_for(130 + d)
+    _check_shift(rng, 24, d, d_out, 4, w_std=0.05)
+    _check_shift(rng, 9, d, d_out, 0, w_std=0.05)       # plain projection, n_rows not a multiple of 16
+
+
+def test_shift_project_pure_shift_and_host_errors():
+    rng = W.rng_for(140)
+    d = 256
+    h = W.f32_to_bf16_bits(rng.standard_normal((12, d), dtype=np.float32))
+    eye, zero = np.eye(d, dtype=np.float32), np.zeros((d, d), np.float32)
+    got, _ = sb.sb_shift_project(dev.bf16_tensor(h), dev.bf16_tensor(W.f32_to_bf16_bits(np.hstack([zero, eye]))), 4)
+    torch.cuda.synchronize()
+    prev = np.asarray([r - 1 if r % 4 else r for r in range(12)])
+    np.testing.assert_array_equal(got.view(torch.int16).cpu().numpy().view(np.uint16), h[prev])   # bit-exact copy
+    ht, wt = dev.bf16_tensor(h), dev.bf16_tensor(W.f32_to_bf16_bits(np.hstack([zero, eye])))
+    with pytest.raises(sb.SbError):
+        sb.sb_shift_project(ht[:, :100].contiguous(), wt[:, :200].contiguous(), 4)      # d not a multiple of 64
+    with pytest.raises(sb.SbError):
+        sb.sb_shift_project(torch.cat([ht] * 11), wt, 4)                                 # more than 128 rows
+    with pytest.raises(sb.SbError):
+        sb.sb_shift_project(ht, wt, 4, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
