@@ -251,28 +251,64 @@ class VerifyStep:
 
     def run_from_host(self):
         """Inputs in pinned host memory -> device, the whole iteration, results -> pinned host
-        memory.  Enqueue only; synchronise the stream before reading the host results."""
+        memory.  Enqueue only; synchronise the current stream before reading the host results.
+
+        The copies are pipelined with the kernels: a copy stream brings layer l's K, V and Q while
+        layer l-1 is being attended to, a second one returns each layer's output while later layers
+        are still arriving (the link is full duplex).  Both streams fork from the current stream
+        at entry and join it at the end, so to the caller the call is ordered like any other work
+        of that stream."""
         h = self.host
-        self.k_all.copy_(h["k"], non_blocking=True)
-        self.v_all.copy_(h["v"], non_blocking=True)
-        self.q_all.copy_(h["q"], non_blocking=True)
-        self.tb.parent.copy_(h["parent"], non_blocking=True)
-        self.tb.node_offsets.copy_(h["node_offsets"], non_blocking=True)
-        self.tb.prefix_len.copy_(h["prefix_len"], non_blocking=True)
-        self.logits.copy_(h["logits"], non_blocking=True)
-        self.tok.copy_(h["tok"], non_blocking=True)
-        if "page_table" in h:
-            self.tb.page_table.copy_(h["page_table"], non_blocking=True)
-        if self.expand is not None:
-            self.expand["scores"].copy_(h["scores"], non_blocking=True)
-            self.expand["bucket"].copy_(h["bucket"], non_blocking=True)
-            self.expand["start_parent"].copy_(h["start_parent"], non_blocking=True)
-        self.run_device()
-        h["out"].copy_(self.out_all, non_blocking=True)
-        h["lse"].copy_(self.lse_all, non_blocking=True)
+        main = torch.cuda.current_stream()
+        L = self.n_layers
+        if not hasattr(self, "_h2d"):
+            self._h2d, self._d2h = torch.cuda.Stream(), torch.cuda.Stream()
+            self._ev = {k: torch.cuda.Event() for k in ("fork", "small", "logits", "d2h_end")}
+            self._ev_in = [torch.cuda.Event() for _ in range(L)]
+            self._ev_done = [torch.cuda.Event() for _ in range(L)]
+        ev = self._ev
+        ev["fork"].record(main)
+        self._h2d.wait_event(ev["fork"])
+        self._d2h.wait_event(ev["fork"])
+        with torch.cuda.stream(self._h2d):
+            self.tb.parent.copy_(h["parent"], non_blocking=True)
+            self.tb.node_offsets.copy_(h["node_offsets"], non_blocking=True)
+            self.tb.prefix_len.copy_(h["prefix_len"], non_blocking=True)
+            self.tok.copy_(h["tok"], non_blocking=True)
+            if "page_table" in h:
+                self.tb.page_table.copy_(h["page_table"], non_blocking=True)
+            if self.expand is not None:
+                self.expand["scores"].copy_(h["scores"], non_blocking=True)
+                self.expand["bucket"].copy_(h["bucket"], non_blocking=True)
+                self.expand["start_parent"].copy_(h["start_parent"], non_blocking=True)
+            ev["small"].record()
+            for l in range(L):
+                self.q_all[l].copy_(h["q"][l], non_blocking=True)
+                self.k_all[l].copy_(h["k"][l], non_blocking=True)
+                self.v_all[l].copy_(h["v"][l], non_blocking=True)
+                self._ev_in[l].record()
+            self.logits.copy_(h["logits"], non_blocking=True)
+            ev["logits"].record()
+        main.wait_event(ev["small"])
+        self.run_ancestors()
+        self.run_expand()
+        for l in range(L):
+            main.wait_event(self._ev_in[l])
+            self.run_attention(layers=[l])
+            self._ev_done[l].record(main)
+            with torch.cuda.stream(self._d2h):
+                self._d2h.wait_event(self._ev_done[l])
+                h["out"][l].copy_(self.out_all[l], non_blocking=True)
+                h["lse"][l].copy_(self.lse_all[l], non_blocking=True)
+        with torch.cuda.stream(self._d2h):
+            ev["d2h_end"].record()
+        main.wait_event(ev["logits"])
+        self.run_accept()
+        self.run_compact()
         for k, t in self.accept.items():
             h["res"][k].copy_(t, non_blocking=True)
         h["new_len"].copy_(self.new_len, non_blocking=True)
+        main.wait_event(ev["d2h_end"])
 
     # ---- accounting -------------------------------------------------------------------------
 
