@@ -612,3 +612,23 @@ def test_shift_project_pure_shift_and_host_errors():
         sb.sb_shift_project(torch.cat([ht] * 11), wt, 4)                                 # more than 128 rows
     with pytest.raises(sb.SbError):
         sb.sb_shift_project(ht, wt, 4, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+
+
+@pytest.mark.parametrize("vocab", [2, 3, 40, 300])
+def test_verify_sample_tiny_vocabularies(vocab):
+    """Vocabularies smaller than the cluster's 256 segments (most warps own nothing)."""
+    rng = W.rng_for(150 + vocab)
+    parents = [W.random_tree(rng, 10, 4), W.chain_tree(3)]
+    n_children = max(np.bincount(np.concatenate([p[p >= 0] for p in parents])).max(), 1)
+    if n_children > vocab:                       # siblings carry distinct tokens
+        parents = [W.chain_tree(6), W.chain_tree(3)]
+    case = _sample_case(rng, parents, vocab, "f32", std=1.0)
+    for rep in range(3):
+        _check_sample(rng, *case, temperature=1.0, max_depth=6)
+
+
+def test_shift_project_single_row_and_smallest_shapes():
+    rng = W.rng_for(160)
+    _check_shift(rng, 1, 64, 128, 1, w_std=0.1)
+    _check_shift(rng, 1, 4096, 128, 0)
+    _check_shift(rng, 128, 64, 128, 128, w_std=0.1)
