@@ -7,12 +7,15 @@
 //   loader warps   one thread per operand issues TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle,
 //                  no multicast) of the K and V blocks straight into the shared-memory layouts the
 //                  tensor core reads (K, Q, P: K-major; V: MN-major), 2 stages each, completion by
-//                  mbarrier transaction count; paged caches load one box per page piece.  V rows past
-//                  the end of the sequence are zeroed (P is 0 there, but 0 * garbage must stay 0).
+//                  mbarrier transaction count; paged caches load one box per page piece, the page ids
+//                  of the next block being fetched while its stage is still busy.  A V block lands
+//                  on the barrier the MMA warp waits on, except the one whose rows pass the end of
+//                  the sequence: those rows are zeroed first (P is 0 there, but 0 * garbage must stay 0).
 //                  The Q tile is one TMA box {64 columns, G heads, 128/G nodes} per column half when
 //                  G divides 128, else a 16-byte cp.async gather by the softmax warps;
 //   MMA warp       one thread issues  S_j = Q K_j^T  (tcgen05.mma, fp32 accumulator in TMEM, two S
 //                  buffers) and  O += P_j V_j  with P_j read from TMEM and O accumulated in TMEM;
+//                  operand descriptors are constant halves plus an offset (two adds per MMA);
 //   softmax warps  8 warps, two threads per row (TMEM lane), each owning 64 of a block's 128 columns:
 //                  read S once from TMEM into registers (tcgen05.ld; the S buffer is released at
 //                  once), apply the softmax scale and the tree mask (one 128-bit ancestor set per
@@ -25,7 +28,9 @@
 //
 // All hand-offs are mbarriers (tcgen05.commit on the MMA side); every wait is bounded and reports
 // SB_ERR_CUDA instead of spinning forever.  The chunk results of the CTAs of a cluster are merged
-// through distributed shared memory exactly as in the mma.sync kernel.
+// through distributed shared memory: every CTA stages its rows normalised in bf16 with (m, l), sends
+// each owner CTA its slice with one bulk shared-to-shared copy, and the owner reduces and stores.
+// Grids that run in several waves take their sequences longest first (attention_common.cuh).
 #include <cstdio>
 #include <cstdlib>
 
