@@ -168,7 +168,8 @@ __global__ void __launch_bounds__(VS_THREADS) verify_sample_kernel(
       const bool in_vocab = x >= 0 && x < vocab;
       cluster.sync();  // pw / qw as the previous round left them, whichever CTA wrote them
       if (tid == 0) {
-        const float pxu = in_vocab ? pw[x] : 0.f, qxu = in_vocab ? qw[x] : 0.f;
+        // these two words may have been written by another CTA of the cluster: read them from L2
+        const float pxu = in_vocab ? __ldcg(pw + x) : 0.f, qxu = in_vocab ? __ldcg(qw + x) : 0.f;
         const float px = pxu / zp;
         const float qx = zq > 0.f ? qxu / zq : 0.f;
         s_take = qx > 0.f ? (u_accept[o + c] < px / qx) : (px > 0.f);
