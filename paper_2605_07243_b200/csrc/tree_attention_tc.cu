@@ -58,7 +58,9 @@ constexpr size_t attn_tc_smem_bytes() {
 }
 
 
-template <int D>
+// SORTED: grid index z is the rank of a sequence by length (a compile-time switch: even an untaken
+// branch to the ranking code cost the one-wave configurations 0.1 us per launch).
+template <int D, bool SORTED>
 __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams p,
                                                                 const __grid_constant__ CUtensorMap kmap,
                                                                 const __grid_constant__ CUtensorMap vmap,
@@ -119,7 +121,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // grid index z -> sequence (longest first when the grid runs in several waves)
-  const int b = p.sort_seqs ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent) : (int)blockIdx.z;
+  const int b = SORTED ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent) : (int)blockIdx.z;
   const SeqPre pre = plan_lengths(p, b);
   const int rows_total = pre.info.nq * G;
   const int row0 = tile * TC_BM;
@@ -614,7 +616,9 @@ template <int D>
 static bool tc_prepare() {
   static bool done = false;
   if (!done) {
-    if (cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(attn_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_tc_smem_bytes<D>()) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)attn_tc_smem_bytes<D>()) != cudaSuccess) {
       cudaGetLastError();
       return false;
@@ -635,10 +639,10 @@ int attn_tc_max_active_clusters(int D, int cluster) {
     cudaError_t e = cudaErrorUnknown;
     if (D == 64 && tc_prepare<64>()) {
       cudaLaunchConfig_t cfg = tc_config<64>(dim3(cluster * 64, 1, 1), cluster, nullptr, attr);
-      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<64>, &cfg);
+      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<64, false>, &cfg);
     } else if (D == 128 && tc_prepare<128>()) {
       cudaLaunchConfig_t cfg = tc_config<128>(dim3(cluster * 64, 1, 1), cluster, nullptr, attr);
-      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<128>, &cfg);
+      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<128, false>, &cfg);
     }
     if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
     cache[di][cluster] = n;
@@ -665,7 +669,9 @@ static sb_status launch_tc(const AttnParams& p, dim3 grid, int cluster, cudaStre
   } else {
     qmap = kmap;  // unused by the kernel in this mode
   }
-  if (cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, p, kmap, vmap, qmap, box_rows, q_tma) != cudaSuccess) {
+  const cudaError_t le = p.sort_seqs ? cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, true>, p, kmap, vmap, qmap, box_rows, q_tma)
+                                     : cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, false>, p, kmap, vmap, qmap, box_rows, q_tma);
+  if (le != cudaSuccess) {
     cudaGetLastError();
     return SB_ERR_CUDA;
   }
