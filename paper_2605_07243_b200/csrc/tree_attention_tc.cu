@@ -58,14 +58,21 @@ constexpr size_t attn_tc_smem_bytes() {
 }
 
 
-// SORTED: grid index z is the rank of a sequence by length (a compile-time switch: even an untaken
-// branch to the ranking code cost the one-wave configurations 0.1 us per launch).
-template <int D, bool SORTED>
+// FAST: the common single-wave case fixed at compile time -- contiguous cache (one 128-row TMA box per
+// block, no page table), Q tile by TMA, all chunks of a tile in one cluster (no fp32 partials), grid
+// index z = sequence.  The general instantiation decides all of that at run time (paged caches, a
+// gathered Q tile, partials for attn_merge_kernel, sequences taken longest first).  Code that is
+// never executed still costs a kernel this short: an untaken branch to the sequence ranking alone
+// was 0.1 us per launch.
+template <int D, bool FAST>
 __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams p,
                                                                 const __grid_constant__ CUtensorMap kmap,
                                                                 const __grid_constant__ CUtensorMap vmap,
                                                                 const __grid_constant__ CUtensorMap qmap,
-                                                                const int box_rows, const int q_tma) {
+                                                                const int box_rows_arg, const int q_tma_arg) {
+  const int box_rows = FAST ? TC_BN : box_rows_arg;
+  const int q_tma = FAST ? 1 : q_tma_arg;
+  const int page_size = FAST ? 0 : p.tb.page_size;
   constexpr int CH = D / 8;                   // 16-byte chunks per row
   constexpr int TILE_BYTES = TC_BN * D * 2;   // one K or V stage
   constexpr int DH = D / 2;                   // output columns per softmax thread
@@ -121,7 +128,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // grid index z -> sequence (longest first when the grid runs in several waves)
-  const int b = SORTED ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent) : (int)blockIdx.z;
+  const int b = (!FAST && p.sort_seqs) ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent)
+                                       : (int)blockIdx.z;
   const SeqPre pre = plan_lengths(p, b);
   const int rows_total = pre.info.nq * G;
   const int row0 = tile * TC_BM;
@@ -154,13 +162,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   // pieces), so that a loader can have them in registers before the stage it waits for is free.
   constexpr int MAX_PIECES = TC_BN / 16;
   auto lookup_pages = [&](int j, int (&pg)[MAX_PIECES]) {
-    if (p.tb.page_size == 0) return;
+    if (FAST || page_size == 0) return;
     const int nj = min(TC_BN, chunk_keys - j * TC_BN);
     const int k0 = key_begin + j * TC_BN;
     const int pieces = ceil_div(nj, box_rows);
 #pragma unroll 1
     for (int i = 0; i < MAX_PIECES; ++i)
-      if (i < pieces) pg[i] = p.tb.page_table[(long long)b * p.tb.max_pages + (k0 + i * box_rows) / p.tb.page_size];
+      if (i < pieces) pg[i] = p.tb.page_table[(long long)b * p.tb.max_pages + (k0 + i * box_rows) / (FAST ? 1 : page_size)];
   };
   auto issue_pieces = [&](int j, const int (&pg)[MAX_PIECES], const CUtensorMap* map, uint32_t stage_addr,
                           uint64_t* bar) {
@@ -173,10 +181,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       if (i >= pieces) break;
       const int key = k0 + i * box_rows;
       int c2 = key, c3 = b;
-      if (p.tb.page_size != 0) {
+      if (page_size != 0) {
         int page = pg[i];
         if (page < 0 || page >= p.tb.num_pages) page = 0;  // reported by the designated CTA
-        c2 = key & (p.tb.page_size - 1);
+        c2 = key & (page_size - 1);
         c3 = page;
       }
 #pragma unroll
@@ -563,7 +571,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
       const float lse2 = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
       if (has_cols) {
-        if (p.outer == 1) {
+        if (FAST || p.outer == 1) {
           uint4 packed;
           packed.x = pack_bf16(acc[0] * inv, acc[1] * inv);
           packed.y = pack_bf16(acc[2] * inv, acc[3] * inv);
@@ -669,8 +677,9 @@ static sb_status launch_tc(const AttnParams& p, dim3 grid, int cluster, cudaStre
   } else {
     qmap = kmap;  // unused by the kernel in this mode
   }
-  const cudaError_t le = p.sort_seqs ? cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, true>, p, kmap, vmap, qmap, box_rows, q_tma)
-                                     : cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, false>, p, kmap, vmap, qmap, box_rows, q_tma);
+  const bool fast = p.tb.page_size == 0 && q_tma && p.outer == 1 && !p.sort_seqs;
+  const cudaError_t le = fast ? cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, true>, p, kmap, vmap, qmap, box_rows, q_tma)
+                              : cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, false>, p, kmap, vmap, qmap, box_rows, q_tma);
   if (le != cudaSuccess) {
     cudaGetLastError();
     return SB_ERR_CUDA;
