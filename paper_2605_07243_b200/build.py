@@ -19,6 +19,7 @@ INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xcompiler", "-fPIC", "--shared", "-Xcompiler", "-Wall",
+    "--threads", "0",   # source files compiled in parallel
 ]
 
 

@@ -63,13 +63,15 @@ constexpr size_t attn_tc_smem_bytes() {
 // index z = sequence.  The general instantiation decides all of that at run time (paged caches, a
 // gathered Q tile, partials for attn_merge_kernel, sequences taken longest first).  Code that is
 // never executed still costs a kernel this short: an untaken branch to the sequence ranking alone
-// was 0.1 us per launch.
-template <int D, bool FAST>
+// was 0.1 us per launch, and knowing the cluster size (CS = 1..8, the chunks of a tile) at compile
+// time another 0.4 us.  CS = 0 is the general instantiation.
+template <int D, int CS>
 __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams p,
                                                                 const __grid_constant__ CUtensorMap kmap,
                                                                 const __grid_constant__ CUtensorMap vmap,
                                                                 const __grid_constant__ CUtensorMap qmap,
                                                                 const int box_rows_arg, const int q_tma_arg) {
+  constexpr bool FAST = CS > 0;
   const int box_rows = FAST ? TC_BN : box_rows_arg;
   const int q_tma = FAST ? 1 : q_tma_arg;
   const int page_size = FAST ? 0 : p.tb.page_size;
@@ -92,7 +94,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   cg::cluster_group cluster = cg::this_cluster();
-  const int S = (int)cluster.num_blocks();
+  const int S = FAST ? CS : (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
   const int split = blockIdx.x;
   const int Hq = p.tb.n_q_heads, G = p.G;
@@ -630,10 +632,14 @@ template <int D>
 static bool tc_prepare() {
   static bool done = false;
   if (!done) {
-    if (cudaFuncSetAttribute(attn_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_tc_smem_bytes<D>()) != cudaSuccess ||
-        cudaFuncSetAttribute(attn_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_tc_smem_bytes<D>()) != cudaSuccess) {
+    bool all = true;
+#define SB_TC_PREPARE(cs_)                                                                                       \
+  all = all && cudaFuncSetAttribute(attn_tc_kernel<D, cs_>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
+                                    (int)attn_tc_smem_bytes<D>()) == cudaSuccess;
+    SB_TC_PREPARE(0) SB_TC_PREPARE(1) SB_TC_PREPARE(2) SB_TC_PREPARE(3) SB_TC_PREPARE(4)
+    SB_TC_PREPARE(5) SB_TC_PREPARE(6) SB_TC_PREPARE(7) SB_TC_PREPARE(8)
+#undef SB_TC_PREPARE
+    if (!all) {
       cudaGetLastError();
       return false;
     }
@@ -653,10 +659,10 @@ int attn_tc_max_active_clusters(int D, int cluster) {
     cudaError_t e = cudaErrorUnknown;
     if (D == 64 && tc_prepare<64>()) {
       cudaLaunchConfig_t cfg = tc_config<64>(dim3(cluster * 64, 1, 1), cluster, nullptr, attr);
-      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<64, false>, &cfg);
+      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<64, 0>, &cfg);
     } else if (D == 128 && tc_prepare<128>()) {
       cudaLaunchConfig_t cfg = tc_config<128>(dim3(cluster * 64, 1, 1), cluster, nullptr, attr);
-      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<128, false>, &cfg);
+      e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<128, 0>, &cfg);
     }
     if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
     cache[di][cluster] = n;
@@ -684,8 +690,15 @@ static sb_status launch_tc(const AttnParams& p, dim3 grid, int cluster, cudaStre
     qmap = kmap;  // unused by the kernel in this mode
   }
   const bool fast = p.tb.page_size == 0 && q_tma && p.outer == 1 && !p.sort_seqs;
-  const cudaError_t le = fast ? cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, true>, p, kmap, vmap, qmap, box_rows, q_tma)
-                              : cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, false>, p, kmap, vmap, qmap, box_rows, q_tma);
+  cudaError_t le = cudaErrorInvalidValue;
+  switch (fast ? cluster : 0) {
+#define SB_TC_LAUNCH(cs_) \
+  case cs_: le = cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, cs_>, p, kmap, vmap, qmap, box_rows, q_tma); break;
+    SB_TC_LAUNCH(0) SB_TC_LAUNCH(1) SB_TC_LAUNCH(2) SB_TC_LAUNCH(3) SB_TC_LAUNCH(4)
+    SB_TC_LAUNCH(5) SB_TC_LAUNCH(6) SB_TC_LAUNCH(7) SB_TC_LAUNCH(8)
+#undef SB_TC_LAUNCH
+    default: break;
+  }
   if (le != cudaSuccess) {
     cudaGetLastError();
     return SB_ERR_CUDA;
