@@ -34,7 +34,7 @@ N_LAYERS = 32
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on this workload, from the
 # ncu capture summarised in profiles/attn_tc_kernel_c2_verify_layer.md
-ATTN_DRAM_TRAFFIC_BYTES = 9209856
+ATTN_DRAM_TRAFFIC_BYTES = 9189120
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -323,7 +323,7 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e},
         "gpu_launches": gpu_launches,
-        "roofline": {"bound": "hbm", "kernel": "sb::attn_tc_kernel<128> (tcgen05), one launch per layer",
+        "roofline": {"bound": "hbm", "kernel": "sb::attn_tc_kernel<128, 6> (tcgen05), one launch per layer",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"{peak_kind} HBM copy bandwidth", "traffic": ATTN_DRAM_TRAFFIC_BYTES,
                      "algorithmic_bytes_per_launch": attn_bytes,
