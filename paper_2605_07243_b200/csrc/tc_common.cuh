@@ -122,6 +122,11 @@ __device__ inline void dsmem_bulk_copy(uint32_t dst_cluster_addr, uint32_t src_c
 __device__ inline void mbar_arrive_remote(uint32_t bar_cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
+// The same without release ordering: for an arrive that publishes no memory of this thread (a pure
+// "I have seen my barrier complete" signal), which then does not wait for the thread's earlier writes.
+__device__ inline void mbar_arrive_remote_relaxed(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
 __device__ inline void softmax_group_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 // 32 consecutive 32-bit columns of this thread's TMEM lane <- registers.
 __device__ inline void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {

@@ -528,8 +528,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
                         (uint32_t)(n * ROWB), mapa_u32(smem_u32(&s_bar[MERGE_BAR]), c));
     }
     merge_ok = mbar_wait(&s_bar[MERGE_BAR], 0, s_abort);
-    // every source's slice has landed here: tell each source that its staging rows are free
-    if (tid < S) mbar_arrive_remote(mapa_u32(smem_u32(&s_bar[ACK_BAR]), tid));
+    // Every source's slice has landed here: tell each source that its staging rows are free.  The
+    // last warp does it (it owns the fewest rows of the reduction below, often none), and the arrive
+    // carries no data, so it needs no release ordering.
+    if (warp == TC_THREADS / 32 - 1 && lane < S) mbar_arrive_remote_relaxed(mapa_u32(smem_u32(&s_bar[ACK_BAR]), lane));
   } else {
     __syncthreads();
   }
