@@ -15,6 +15,7 @@ from .oracle import (  # noqa: F401
     verifier_signal,
     verify_sample,
     shift_project,
+    fuse_project,
     accept_from_amax,
     kv_compact,
     tree_expand,

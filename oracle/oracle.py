@@ -151,6 +151,20 @@ def shift_project(h, w, block_k):
     return out
 
 
+def fuse_project(c, e, q, w, gain_c=None, gain_e=None, gain_q=None, eps=1e-6):
+    """c, e uint16 (bf16 bits) [S, d], q uint16 [K, d], w uint16 [d_out, 3d], gains f32 [d] or None -> f64 [S*K, d_out]."""
+    c, e, q, w = (np.ascontiguousarray(a, np.uint16) for a in (c, e, q, w))
+    n_starts, d = c.shape
+    block_k = q.shape[0]
+    d_out = w.shape[0]
+    assert e.shape == c.shape and q.shape[1] == d and w.shape[1] == 3 * d
+    gains = [None if g is None else np.ascontiguousarray(g, np.float32) for g in (gain_c, gain_e, gain_q)]
+    out = np.zeros((n_starts * block_k, d_out), np.float64)
+    _load().sbo_fuse_project(_p(c), _p(e), _p(q), *[_p(g) for g in gains], C.c_double(eps),
+                             _p(w), C.c_int(n_starts), C.c_int(block_k), C.c_int(d), C.c_int(d_out), _p(out))
+    return out
+
+
 def verifier_signal(scores, node_offsets, child_row, path_nodes, accept_len, bonus, max_depth, signal=None,
                     vocab=None):
     """-> dict(r_prob f64 [B], signal f64 [B] (= signal in + 1 - r), status int32 [B])."""

@@ -30,6 +30,11 @@
  *                         readings -- for those PARITY IS UNPINNED by the paper.
  *   sbo_shift_project   : numpy matmul on the explicitly concatenated input; W = [I, 0] returns the input,
  *                         W = [0, I] the previous position's state (the first position its own).
+ *   sbo_fuse_project    : numpy (mean-square, concatenate, matmul) on a non-square W; closed forms for
+ *                         W = [I, 0, 0] with constant and two-valued inputs; invariance under
+ *                         rescaling an input when eps = 0; the difference between two positions of a
+ *                         block does not depend on the start.  "norm" is not specified by the paper:
+ *                         the RMS norm is a reading -- for the choice of norm PARITY IS UNPINNED.
  *   sbo_tree_expand     : hand-derived trees for the two printed branching maps; chain special
  *                         case; structural invariants.  The attach point of siblings, the cut
  *                         order at the node budget and the treatment of b = 0 are readings of
@@ -530,6 +535,43 @@ void sbo_shift_project(const uint16_t* h, const uint16_t* w, int n_rows, int d, 
           acc += bf16_to_f64(w[(int64_t)f * kin + d + j]) * bf16_to_f64(h[(int64_t)prev * d + j]);
       out[(int64_t)r * d_out + f] = acc;
     }
+  }
+}
+
+/* ---- the drafter's per-position input (Sec. 3.1, the equation for h^(0)) -------------------------- */
+
+/*
+ * h0[s * K + k] = W_fuse [ norm(c_s), norm(e_s), norm(q_k) ]:  c_s the context feature of start s,
+ * e_s the embedding of its last committed token (both shared by the K positions of the block: the
+ * prefix broadcast), q_k the learnable query of draft depth k.  The paper says only "normalized";
+ * read as the root-mean-square norm of the target's architecture with a learnable gain,
+ *   norm(x)[j] = g[j] * x[j] / sqrt(mean_j x[j]^2 + eps)        (g = NULL: all ones).
+ * c, e bf16 [n_starts][d], q bf16 [block_k][d], gains f32 [d], w bf16 [d_out][3 d], out f64
+ * [n_starts * block_k][d_out].
+ */
+static void rms_norm_f64(const uint16_t* x, const float* g, int d, double eps, double* y) {
+  double ss = 0.0;
+  for (int j = 0; j < d; ++j) { const double v = bf16_to_f64(x[j]); ss += v * v; }
+  const double inv = 1.0 / sqrt(ss / d + eps);
+  for (int j = 0; j < d; ++j) y[j] = (g ? (double)g[j] : 1.0) * bf16_to_f64(x[j]) * inv;
+}
+
+void sbo_fuse_project(const uint16_t* c, const uint16_t* e, const uint16_t* q, const float* gain_c,
+                      const float* gain_e, const float* gain_q, double eps, const uint16_t* w, int n_starts,
+                      int block_k, int d, int d_out, double* out) {
+#pragma omp parallel for schedule(static)
+  for (int r = 0; r < n_starts * block_k; ++r) {
+    const int s = r / block_k, k = r % block_k;
+    double* x = (double*)malloc(sizeof(double) * 3 * d);  /* the concatenation of the equation */
+    rms_norm_f64(c + (int64_t)s * d, gain_c, d, eps, x);
+    rms_norm_f64(e + (int64_t)s * d, gain_e, d, eps, x + d);
+    rms_norm_f64(q + (int64_t)k * d, gain_q, d, eps, x + 2 * d);
+    for (int f = 0; f < d_out; ++f) {
+      double acc = 0.0;
+      for (int j = 0; j < 3 * d; ++j) acc += bf16_to_f64(w[(int64_t)f * 3 * d + j]) * x[j];
+      out[(int64_t)r * d_out + f] = acc;
+    }
+    free(x);
   }
 }
 

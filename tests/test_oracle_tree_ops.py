@@ -613,3 +613,84 @@ def test_shift_project_matches_numpy_on_the_concatenated_input():
     np.testing.assert_array_equal(oracle.shift_project(h, W.f32_to_bf16_bits(np.hstack([eye, zero])), K), hf)
     np.testing.assert_array_equal(oracle.shift_project(h, W.f32_to_bf16_bits(np.hstack([zero, eye])), K), hf[prev])
     assert (prev[::K] == np.arange(0, R, K)).all()
+
+
+# ---- the drafter's fused per-position input (Sec. 3.1, the equation for h^(0)) ------------------------------------
+
+def _fuse_inputs(rng, S, K, d, d_out, scale=1.0):
+    c = W.f32_to_bf16_bits(rng.standard_normal((S, d), dtype=np.float32) * 3.0 * scale)
+    e = W.f32_to_bf16_bits(rng.standard_normal((S, d), dtype=np.float32) * 0.05)
+    q = W.f32_to_bf16_bits(rng.standard_normal((K, d), dtype=np.float32))
+    w = W.f32_to_bf16_bits(rng.standard_normal((d_out, 3 * d), dtype=np.float32) * 0.1)
+    return c, e, q, w
+
+
+def test_fuse_project_matches_numpy_on_the_concatenated_normalised_input():
+    rng = W.rng_for(51)
+    S, K, d, d_out = 5, 4, 96, 40                                 # W is not square: a transposed operand cannot pass
+    c, e, q, w = _fuse_inputs(rng, S, K, d, d_out)
+    gains = [rng.uniform(0.5, 1.5, d).astype(np.float32) for _ in range(3)]
+    eps = 1e-5
+    f64 = lambda bits: W.bf16_bits_to_f32(bits).astype(np.float64)
+
+    def norm(x, g):
+        return g.astype(np.float64) * x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
+
+    cn, en, qn = norm(f64(c), gains[0]), norm(f64(e), gains[1]), norm(f64(q), gains[2])
+    x = np.concatenate([np.repeat(cn, K, axis=0), np.repeat(en, K, axis=0), np.tile(qn, (S, 1))], axis=1)
+    want = x @ f64(w).T
+    got = oracle.fuse_project(c, e, q, w, *gains, eps=eps)
+    assert got.shape == (S * K, d_out)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    # gains left out are ones
+    ones = np.ones(d, np.float32)
+    np.testing.assert_allclose(oracle.fuse_project(c, e, q, w, eps=eps), oracle.fuse_project(c, e, q, w, ones, ones, ones, eps=eps),
+                               rtol=0, atol=0)
+
+
+def test_fuse_project_closed_forms_with_selector_weights():
+    S, K, d = 2, 3, 8
+    eye, zero = np.eye(d, dtype=np.float32), np.zeros((d, d), np.float32)
+    # c_0 = (3, 4, 3, 4, ...): mean square 12.5; c_1 constant -2: norm = -1 everywhere (eps = 0)
+    c = np.stack([np.tile([3.0, 4.0], d // 2), np.full(d, -2.0)]).astype(np.float32)
+    e = np.stack([np.full(d, 0.5), np.tile([1.0, -1.0], d // 2)]).astype(np.float32)
+    q = np.stack([np.full(d, 7.0), np.tile([0.0, 2.0], d // 2), np.tile([1.0, 0.0], d // 2)]).astype(np.float32)
+    bits = W.f32_to_bf16_bits
+    sel = lambda i: bits(np.hstack([eye if j == i else zero for j in range(3)]))
+    out_c = oracle.fuse_project(bits(c), bits(e), bits(q), sel(0), eps=0.0)
+    for k in range(K):                                            # the prefix broadcast: the same c for every position
+        np.testing.assert_allclose(out_c[0 * K + k], np.tile([3.0, 4.0], d // 2) / np.sqrt(12.5), rtol=1e-15)
+        np.testing.assert_allclose(out_c[1 * K + k], np.full(d, -1.0), rtol=1e-15)
+    out_e = oracle.fuse_project(bits(c), bits(e), bits(q), sel(1), eps=0.0)
+    np.testing.assert_allclose(out_e[0], np.full(d, 1.0), rtol=1e-15)
+    np.testing.assert_allclose(out_e[K + 2], np.tile([1.0, -1.0], d // 2), rtol=1e-15)
+    out_q = oracle.fuse_project(bits(c), bits(e), bits(q), sel(2), eps=0.0)
+    for s in range(S):                                            # only q varies across the positions of a block
+        np.testing.assert_allclose(out_q[s * K + 0], np.full(d, 1.0), rtol=1e-15)
+        np.testing.assert_allclose(out_q[s * K + 1], np.tile([0.0, np.sqrt(2.0)], d // 2), rtol=1e-15)
+        np.testing.assert_allclose(out_q[s * K + 2], np.tile([np.sqrt(2.0), 0.0], d // 2), rtol=1e-15)
+    # eps enters under the root: constant input a gives a / sqrt(a^2 + eps)
+    out_eps = oracle.fuse_project(bits(c), bits(e), bits(q), sel(0), eps=5.0)
+    np.testing.assert_allclose(out_eps[K], np.full(d, -2.0 / 3.0), rtol=1e-15)
+    # a gain multiplies after the normalisation
+    g = np.arange(1, d + 1, dtype=np.float32)
+    out_g = oracle.fuse_project(bits(c), bits(e), bits(q), sel(0), gain_c=g, eps=0.0)
+    np.testing.assert_allclose(out_g[K], -g.astype(np.float64), rtol=1e-15)
+
+
+def test_fuse_project_invariants():
+    rng = W.rng_for(52)
+    S, K, d, d_out = 4, 4, 64, 24
+    c, e, q, w = _fuse_inputs(rng, S, K, d, d_out)
+    base = oracle.fuse_project(c, e, q, w, eps=0.0)
+    # with eps = 0 each input is normalised on its own: rescaling one by a power of two changes nothing
+    c4 = W.f32_to_bf16_bits(W.bf16_bits_to_f32(c) * 4.0)
+    e8 = W.f32_to_bf16_bits(W.bf16_bits_to_f32(e) * 0.125)
+    np.testing.assert_allclose(oracle.fuse_project(c4, e8, q, w, eps=0.0), base, rtol=1e-12, atol=1e-12)
+    # the difference between two positions of a block comes from the queries alone: the same for every start
+    diffs = base.reshape(S, K, d_out) - base.reshape(S, K, d_out)[:, :1]
+    np.testing.assert_allclose(diffs, np.broadcast_to(diffs[0], diffs.shape), rtol=1e-10, atol=1e-10)
+    assert np.abs(diffs[0, 1:]).max() > 0.1
+    # linear in W
+    w2 = W.f32_to_bf16_bits(W.bf16_bits_to_f32(w) * 2.0)
+    np.testing.assert_allclose(oracle.fuse_project(c, e, q, w2, eps=0.0), 2.0 * base, rtol=1e-12, atol=1e-12)
