@@ -240,6 +240,8 @@ def run_ours(args):
         g_sample = capture(torch, step.run_sample)
         step.run_shift_all()
         g_shift = capture(torch, step.run_shift_all)
+        step.run_fuse_all()
+        g_fuse = capture(torch, step.run_fuse_all)
 
         for _ in range(max(args.warmup, 3)):
             g_step.replay()
@@ -270,11 +272,13 @@ def run_ours(args):
         for name, g in (("expand", g_expand), ("accept", g_accept), ("compact", g_compact),
                         ("rank_features_not_in_step", g_features), ("verifier_signal_not_in_step", g_signal),
                         ("verify_sample_T1_not_in_step", g_sample),
-                        ("shift_project_32x4096_not_in_step", g_shift)):
+                        ("shift_project_32x4096_not_in_step", g_shift),
+                        ("fuse_project_8x4x4096_not_in_step", g_fuse)):
             for _ in range(3):
                 g.replay()
             parts_ms[name] = time_graph(torch, g, 20, False) / 20
         parts_ms["shift_project_32x4096_not_in_step"] /= step.SHIFT_SETS   # one graph = one call per weight set
+        parts_ms["fuse_project_8x4x4096_not_in_step"] /= step.FUSE_SETS
 
         # end to end: inputs in pinned host memory, results back to pinned host memory
         e2e_steps = 1 if args.quick else max(3, min(args.steps, 5))

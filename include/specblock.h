@@ -14,6 +14,7 @@
  *   sb_verifier_signal verifier-derived update signal s = sum (1 - r)   (Sec. 3.4, Alg. 2)
  *   sb_verify_sample   stochastic (temperature > 0) tree verification   (Sec. 4.1, Sec. 4.2)
  *   sb_shift_project   layer-wise shift projection between drafter layers (Sec. 3.1)
+ *   sb_fuse_project    the drafter's fused per-position input h^(0)      (Sec. 3.1 "Block forward")
  *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
  *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
  *
@@ -203,11 +204,46 @@ size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
  *   K splits and one word that outlives the call: hand the same workspace to every call, or a zeroed
  *   one).  status int32 [1]: SB_OK, or SB_ERR_CUDA if a bounded device wait gave up.
  *   HBM-bound on the weights: 2 * d * d_out * 2 bytes are read once.
+ *   Ordering: the kernels are programmatic dependents of whatever precedes the call in the stream.
+ *   h (and every output) is touched only after that work has completed, but the first tiles of w
+ *   are requested earlier: w must not be written by the ONE kernel enqueued immediately before the
+ *   call (weights updated earlier in the stream are seen as usual).
  */
 sb_status sb_shift_project(const void* h, const void* w, int32_t n_rows, int32_t d, int32_t d_out,
                            int32_t block_k, void* out, void* workspace, size_t workspace_bytes,
                            int32_t* status, void* stream);
 size_t sb_shift_project_workspace_bytes(int32_t n_rows, int32_t d, int32_t d_out, int32_t block_k);
+
+/*
+ * sb_fuse_project -- the per-position input of a drafter block (Sec. 3.1 "Block forward", the
+ * equation for h^(0)): the context feature c_s of start s, the embedding e_s of its last committed
+ * token and the learnable query q_k of draft depth k are normalised, concatenated and projected by
+ * W_fuse.  c_s and e_s are shared by the block_k positions of a block (the prefix broadcast).
+ *
+ *   c, e bf16 [n_starts][d];  q bf16 [block_k][d];  w bf16 [d_out][3 d] row-major, acting on
+ *   [norm(c) , norm(e) , norm(q)].  "norm" is not specified further by the paper; here it is
+ *   norm(x)[j] = gain[j] * x[j] / sqrt(mean_j x[j]^2 + eps), gains fp32 [d] or NULL for ones (the
+ *   normalised rows are rounded to bf16, the type of the tensor-core operand).
+ *   out bf16 [n_starts * block_k][d_out], row s * block_k + k; fp32 accumulation.
+ *   Since out[s, k] = w_c norm(c_s) + w_e norm(e_s) + w_q norm(q_k), the GEMM has
+ *   max(n_starts, block_k) columns and every third of w is read once.  The last term does not
+ *   depend on the start or on the call: with q_term_valid = 0 it is computed and, if q_term is not
+ *   NULL, stored there (fp32 [block_k][d_out]); with q_term_valid = 1 it is read from q_term and only
+ *   the first 2 d columns of w are streamed.  Both ways give bit-identical outputs.
+ *   Limits: n_starts, block_k <= 128, d a multiple of 64, d_out a multiple of 128, pointers 16-byte
+ *   aligned (out 8).  workspace: sb_fuse_project_workspace_bytes(...) bytes, 256-byte aligned (the
+ *   normalised rows, fp32 partials and one word that outlives the call, as for sb_shift_project).
+ *   status int32 [1]: SB_OK, or SB_ERR_CUDA if a bounded device wait gave up.
+ *   HBM-bound on the weights: (3 or 2) * d * d_out * 2 bytes.  Ordering as for sb_shift_project: c, e, q,
+ *   the gains and q_term are read after the preceding work has completed, the first tiles of w before.
+ */
+sb_status sb_fuse_project(const void* c, const void* e, const void* q, const float* gain_c,
+                          const float* gain_e, const float* gain_q, float eps, const void* w,
+                          int32_t n_starts, int32_t block_k, int32_t d, int32_t d_out, float* q_term,
+                          int32_t q_term_valid, void* out, void* workspace, size_t workspace_bytes,
+                          int32_t* status, void* stream);
+size_t sb_fuse_project_workspace_bytes(int32_t n_starts, int32_t block_k, int32_t d, int32_t d_out,
+                                       int32_t q_term_valid);
 
 /*
  * sb_verify_sample -- verification at temperature T > 0 by multi-candidate rejection sampling over

@@ -63,11 +63,12 @@ def load(build_if_missing: bool = True):
     lib.sb_kernel_launch_count.restype = C.c_int64
     for name in ("sb_tree_attention_workspace_bytes", "sb_tree_expand_workspace_bytes",
                  "sb_verify_accept_workspace_bytes", "sb_rank_features_workspace_bytes",
-                 "sb_verify_sample_workspace_bytes", "sb_shift_project_workspace_bytes"):
+                 "sb_verify_sample_workspace_bytes", "sb_shift_project_workspace_bytes",
+                 "sb_fuse_project_workspace_bytes"):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
                  "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal", "sb_verify_sample",
-                 "sb_shift_project"):
+                 "sb_shift_project", "sb_fuse_project"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -78,7 +79,7 @@ EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspa
             "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
             "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_verifier_signal", "sb_verify_sample",
             "sb_verify_sample_workspace_bytes", "sb_shift_project", "sb_shift_project_workspace_bytes",
-            "sb_status_string",
+            "sb_fuse_project", "sb_fuse_project_workspace_bytes", "sb_status_string",
             "sb_version",
             "sb_kernel_launch_count")
 
@@ -328,6 +329,38 @@ def sb_shift_project(h, w, block_k, *, out=None, workspace=None, status=None):
                                  C.c_int32(d_out), C.c_int32(block_k), _ptr(out, torch.bfloat16), _ptr(workspace),
                                  C.c_size_t(workspace.numel()), _ptr(status, torch.int32), _stream())
     _check(rc, "sb_shift_project")
+    return out, status
+
+
+def sb_fuse_project_workspace_bytes(n_starts: int, block_k: int, d: int, d_out: int, q_term_valid: bool) -> int:
+    return int(load().sb_fuse_project_workspace_bytes(C.c_int32(n_starts), C.c_int32(block_k), C.c_int32(d),
+                                                      C.c_int32(d_out), C.c_int32(1 if q_term_valid else 0)))
+
+
+def sb_fuse_project(c, e, q, w, *, gain_c=None, gain_e=None, gain_q=None, eps=1e-6, q_term=None, q_term_valid=False,
+                    out=None, workspace=None, status=None):
+    """c, e bf16 [S, d], q bf16 [K, d], w bf16 [d_out, 3d] -> out bf16 [S*K, d_out] (row s*K + k).
+    q_term fp32 [K, d_out]: written when q_term_valid is false, read (and a third of w skipped) when true."""
+    n_starts, d = c.shape
+    block_k = q.shape[0]
+    d_out = w.shape[0]
+    dev = c.device
+    if e.shape != c.shape or q.shape[1] != d or w.shape[1] != 3 * d:
+        raise ValueError("expected c, e [S, d], q [K, d], w [d_out, 3d]")
+    if q_term is not None and tuple(q_term.shape) != (block_k, d_out):
+        raise ValueError("q_term must be [K, d_out]")
+    out = torch.empty((n_starts * block_k, d_out), dtype=torch.bfloat16, device=dev) if out is None else out
+    status = torch.zeros(1, dtype=torch.int32, device=dev) if status is None else status
+    if workspace is None:
+        workspace = torch.zeros(max(sb_fuse_project_workspace_bytes(n_starts, block_k, d, d_out, q_term_valid), 256),
+                                dtype=torch.uint8, device=dev)
+    rc = load().sb_fuse_project(_ptr(c, torch.bfloat16), _ptr(e, torch.bfloat16), _ptr(q, torch.bfloat16),
+                                _ptr(gain_c, torch.float32), _ptr(gain_e, torch.float32), _ptr(gain_q, torch.float32),
+                                C.c_float(eps), _ptr(w, torch.bfloat16), C.c_int32(n_starts), C.c_int32(block_k),
+                                C.c_int32(d), C.c_int32(d_out), _ptr(q_term, torch.float32),
+                                C.c_int32(1 if q_term_valid else 0), _ptr(out, torch.bfloat16), _ptr(workspace),
+                                C.c_size_t(workspace.numel()), _ptr(status, torch.int32), _stream())
+    _check(rc, "sb_fuse_project")
     return out, status
 
 

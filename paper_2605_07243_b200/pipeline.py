@@ -193,6 +193,41 @@ class VerifyStep:
                                 status=e["shift_status"])
         return e["shift_out"]
 
+    FUSE_SETS = 3    # W_fuse matrices rotated per run_fuse_all(): 3 x 96 MB (64 MB of each streamed) > L2
+
+    def run_fuse_all(self, d=4096, n_starts=8, block_k=4):
+        """The drafter's fused per-position input (W_fuse over the normalised context, embedding and
+        position query) for a block forward of n_starts starts, with the query term cached as in steady
+        state; timed on its own like run_shift_all(), once per weight matrix of a rotating set."""
+        e = self.expand
+        if e is None:
+            return None
+        if "fuse_w" not in e:
+            gen = torch.Generator(device="cpu").manual_seed(8765)
+            bf = lambda *shape, std=1.0: (torch.randn(*shape, generator=gen) * std).to(torch.bfloat16).to(self.device)
+            e["fuse_c"], e["fuse_e"], e["fuse_q"] = bf(n_starts, d, std=3.0), bf(n_starts, d, std=0.05), bf(block_k, d)
+            e["fuse_w"] = [bf(d, 3 * d, std=0.02) for _ in range(self.FUSE_SETS)]
+            e["fuse_gain"] = [(torch.rand(d, generator=gen) + 0.5).to(self.device) for _ in range(3)]
+            e["fuse_out"] = torch.empty(n_starts * block_k, d, dtype=torch.bfloat16, device=self.device)
+            e["fuse_ws"] = torch.zeros(sb.sb_fuse_project_workspace_bytes(n_starts, block_k, d, d, False),
+                                       dtype=torch.uint8, device=self.device)
+            e["fuse_status"] = torch.zeros(1, dtype=torch.int32, device=self.device)
+            e["fuse_q_term"] = []
+            for w in e["fuse_w"]:        # the first call with a weight matrix leaves its query term behind
+                qt = torch.empty(block_k, d, dtype=torch.float32, device=self.device)
+                self._fuse_call(w, qt, False)
+                e["fuse_q_term"].append(qt)
+        for w, qt in zip(e["fuse_w"], e["fuse_q_term"]):
+            self._fuse_call(w, qt, True)
+        return e["fuse_out"]
+
+    def _fuse_call(self, w, q_term, valid):
+        e = self.expand
+        g = e["fuse_gain"]
+        sb.sb_fuse_project(e["fuse_c"], e["fuse_e"], e["fuse_q"], w, gain_c=g[0], gain_e=g[1], gain_q=g[2], eps=1e-5,
+                           q_term=q_term, q_term_valid=valid, out=e["fuse_out"], workspace=e["fuse_ws"],
+                           status=e["fuse_status"])
+
     def run_attention(self, layers=None):
         for l in range(self.n_layers) if layers is None else layers:
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,

@@ -632,3 +632,79 @@ def test_shift_project_single_row_and_smallest_shapes():
     _check_shift(rng, 1, 64, 128, 1, w_std=0.1)
     _check_shift(rng, 1, 4096, 128, 0)
     _check_shift(rng, 128, 64, 128, 128, w_std=0.1)
+
+
+# ---- the drafter's fused per-position input (Sec. 3.1, the equation for h^(0)) ------------------------------------
+
+def _check_fuse(rng, S, K, d, d_out, *, gains=True, eps=1e-5, w_std=0.02):
+    c = W.f32_to_bf16_bits(rng.standard_normal((S, d), dtype=np.float32) * np.float32(3.0))
+    e = W.f32_to_bf16_bits(rng.standard_normal((S, d), dtype=np.float32) * np.float32(0.05))
+    q = W.f32_to_bf16_bits(rng.standard_normal((K, d), dtype=np.float32))
+    w = W.f32_to_bf16_bits(rng.standard_normal((d_out, 3 * d), dtype=np.float32) * np.float32(w_std))
+    g = [rng.uniform(0.5, 1.5, d).astype(np.float32) if gains else None for _ in range(3)]
+    gt = [None if x is None else torch.from_numpy(x).cuda() for x in g]
+    ct, et, qt, wt = (dev.bf16_tensor(a) for a in (c, e, q, w))
+    q_term = torch.full((K, d_out), float("nan"), dtype=torch.float32, device="cuda")
+    full, status = sb.sb_fuse_project(ct, et, qt, wt, gain_c=gt[0], gain_e=gt[1], gain_q=gt[2], eps=eps, q_term=q_term)
+    torch.cuda.synchronize()
+    assert int(status.cpu()[0]) == 0
+    ref = oracle.fuse_project(c, e, q, w, *g, eps=eps)
+    got = full.float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref)
+    # The normalised rows are rounded to bf16 before the tensor-core product (relative 2^-9 per element,
+    # independent): an absolute error of about 1e-3 of the outputs' root mean square, whatever |ref| is.
+    # The absolute term of the bound therefore scales with that root mean square (about 9 sigma).
+    scale = max(1.0, float(np.sqrt(np.mean(ref * ref))))
+    tol = 1e-2 * scale + 1e-2 * np.abs(ref)
+    assert (err <= tol).all(), f"max err/tol {(err / tol).max():.3f}"
+    # the cached query term: two thirds of the weights streamed, the same bits out
+    assert bool(torch.isfinite(q_term).all())
+    again, status2 = sb.sb_fuse_project(ct, et, qt, wt, gain_c=gt[0], gain_e=gt[1], gain_q=gt[2], eps=eps, q_term=q_term,
+                                        q_term_valid=True)
+    torch.cuda.synchronize()
+    assert int(status2.cpu()[0]) == 0
+    assert torch.equal(again.view(torch.int16), full.view(torch.int16))
+    # the query term itself: W_q norm(q_k), i.e. the oracle with the other two thirds of W zeroed
+    wq = W.bf16_bits_to_f32(w).copy()
+    wq[:, :2 * d] = 0
+    ref_q = oracle.fuse_project(c[:1], e[:1], q, W.f32_to_bf16_bits(wq), *g, eps=eps)
+    errq = np.abs(q_term.cpu().numpy().astype(np.float64) - ref_q)
+    assert (errq <= 1e-2 * scale + 1e-2 * np.abs(ref_q)).all()
+    return got, ref
+
+
+@pytest.mark.parametrize("S,K", [(8, 4), (1, 4), (16, 4), (3, 8), (128, 1)])
+def test_fuse_project_8b_shape(S, K):
+    """d = d_out = 4096 (the 8B drafter's width): 96 MB of weights, 64 MB with the query term cached."""
+    _check_fuse(W.rng_for(170 + S), S, K, 4096, 4096)
+
+
+@pytest.mark.parametrize("d,d_out", [(64, 128), (192, 384), (1024, 256)])
+def test_fuse_project_other_shapes(d, d_out):
+    rng = W.rng_for(180 + d)
+    _check_fuse(rng, 5, 4, d, d_out, w_std=0.05)
+    _check_fuse(rng, 2, 7, d, d_out, gains=False, eps=0.0, w_std=0.05)   # more positions than starts, no gains
+
+
+def test_fuse_project_selector_weights_and_host_errors():
+    rng = W.rng_for(190)
+    S, K, d = 3, 4, 128
+    eye, zero = np.eye(d, dtype=np.float32), np.zeros((d, d), np.float32)
+    c = W.f32_to_bf16_bits(np.stack([np.tile([3.0, 4.0], d // 2), np.full(d, -2.0), np.full(d, 0.25)]).astype(np.float32))
+    e = W.f32_to_bf16_bits(rng.standard_normal((S, d), dtype=np.float32))
+    q = W.f32_to_bf16_bits(rng.standard_normal((K, d), dtype=np.float32))
+    ct, et, qt = dev.bf16_tensor(c), dev.bf16_tensor(e), dev.bf16_tensor(q)
+    wt = dev.bf16_tensor(W.f32_to_bf16_bits(np.hstack([eye, zero, zero])))
+    got, _ = sb.sb_fuse_project(ct, et, qt, wt, eps=0.0)
+    torch.cuda.synchronize()
+    got = got.float().cpu().numpy().reshape(S, K, d)
+    want = np.stack([np.tile([3.0, 4.0], d // 2) / np.sqrt(12.5), np.full(d, -1.0), np.full(d, 1.0)])
+    for k in range(K):                                   # the prefix broadcast: every position sees the same c
+        np.testing.assert_allclose(got[:, k], want, rtol=2.0 ** -8)
+    with pytest.raises(sb.SbError):
+        sb.sb_fuse_project(ct[:, :100].contiguous(), et[:, :100].contiguous(), qt[:, :100].contiguous(),
+                           wt[:, :300].contiguous())                                  # d not a multiple of 64
+    with pytest.raises(sb.SbError):
+        sb.sb_fuse_project(ct, et, qt, wt, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(sb.SbError):
+        sb.sb_fuse_project(ct, et, qt, wt, q_term_valid=True)                         # no q_term to read
