@@ -242,6 +242,14 @@ def run_ours(args):
         g_shift = capture(torch, step.run_shift_all)
         step.run_fuse_all()
         g_fuse = capture(torch, step.run_fuse_all)
+        # one whole iteration (two drafter blocks growing the tree on the device, then the verify forward on it)
+        from paper_2605_07243_b200.iteration import build_8b_iteration
+        iteration = build_8b_iteration(layers, ver.logits, ver.max_depth, num_splits=args.num_splits)
+        iteration.run()
+        side.synchronize()
+        assert int(iteration.attn_status.max()) == 0 and int(iteration.accept["status"].max()) == 0
+        assert all(int(e["status"][0]) == 0 for e in iteration.blocks)
+        g_iter = capture(torch, iteration.run)
 
         for _ in range(max(args.warmup, 3)):
             g_step.replay()
@@ -273,7 +281,8 @@ def run_ours(args):
                         ("rank_features_not_in_step", g_features), ("verifier_signal_not_in_step", g_signal),
                         ("verify_sample_T1_not_in_step", g_sample),
                         ("shift_project_32x4096_not_in_step", g_shift),
-                        ("fuse_project_8x4x4096_not_in_step", g_fuse)):
+                        ("fuse_project_8x4x4096_not_in_step", g_fuse),
+                        ("whole_iteration_2_blocks_32_layers_not_in_step", g_iter)):
             for _ in range(3):
                 g.replay()
             parts_ms[name] = time_graph(torch, g, 20, False) / 20
