@@ -10,11 +10,15 @@
 //                         ascending) is kept by strict compares.  The CTA then pops its 16 best in order.
 //   topk_partial_reg_kernel: the same result with the chunk held in registers (one HBM pass, no re-read),
 //                         used whenever rows are 16-byte aligned and a chunk has at most 16384 elements.
-//   expand_finish_kernel: one CTA.  A warp per row merges the chunk lists held in registers; then the
-//                         append is done in parallel: a row is alive iff every earlier position of its
-//                         block has width >= 1, its first node id is an exclusive prefix sum of the
-//                         alive rows' widths, and the node budget clips the tail (a clipped rank-0 node
-//                         can only silence rows that the full budget silences anyway).
+//   expand_rows_kernel  : the finishing kernel for up to 1024 rows, a CTA per row and no CTA waiting for another:
+//                         the branching structure (widths, prefix sums, parents) depends on the inputs alone
+//                         and is derived by every CTA before the dependency wait; after it the CTA ranks its
+//                         row's candidates by counting larger 64-bit keys and writes the row's own nodes.
+//   expand_finish_kernel: the same for any number of rows in ONE CTA.  A warp per row merges the chunk lists
+//                         held in registers; then the append is done in parallel: a row is alive iff every
+//                         earlier position of its block has width >= 1, its first node id is an exclusive
+//                         prefix sum of the alive rows' widths, and the node budget clips the tail (a clipped
+//                         rank-0 node can only silence rows that the full budget silences anyway).
 #include "tc_common.cuh"
 
 namespace sb {
@@ -59,7 +63,8 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
                                                                     int n_chunks, bool vec_ok,
                                                                     float* __restrict__ part_val,
                                                                     int* __restrict__ part_idx,
-                                                                    float* __restrict__ part_stats) {
+                                                                    float* __restrict__ part_stats, const int* __restrict__ n_nodes_in,
+    int* __restrict__ n0_snapshot) {
   __shared__ float s_val[SB_KMAX][TOPK_THREADS];  // [rank][thread]: conflict-free per-thread lists
   __shared__ int s_idx[SB_KMAX][TOPK_THREADS];
   __shared__ float s_wv[TOPK_THREADS / 32];
@@ -70,6 +75,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_kernel(const float*
   const int begin = c * chunk;
   const int end = min(vocab, begin + chunk);
   pdl_release();  // the finishing kernel may start its prologue
+  if (n0_snapshot && row == 0 && c == 0 && tid == 0) *n0_snapshot = *n_nodes_in;  // the finishing kernel overwrites the counter
 
   // pass 1: thread maxima -> threshold tau = 16th largest of them
   const int n_vec = vec_ok ? max(0, (end - begin) / 4) : 0;
@@ -207,7 +213,8 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
                                                                         long long row_stride, int vocab, int chunk,
                                                                         int n_chunks, float* __restrict__ part_val,
                                                                         int* __restrict__ part_idx,
-                                                                        float* __restrict__ part_stats) {
+                                                                        float* __restrict__ part_stats, const int* __restrict__ n_nodes_in,
+    int* __restrict__ n0_snapshot) {
   __shared__ float s_val[SB_KMAX][TOPK_THREADS];  // fallback lists; the candidate arrays alias them
   __shared__ int s_idx[SB_KMAX][TOPK_THREADS];
   __shared__ float s_group[16];
@@ -224,6 +231,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
   const int begin = c * chunk;
   const int end = min(vocab, begin + chunk);
   pdl_release();  // the finishing kernel may start its prologue
+  if (n0_snapshot && row == 0 && c == 0 && tid == 0) *n0_snapshot = *n_nodes_in;  // the finishing kernel overwrites the counter
   const int n_elems = max(0, end - begin);
   const int n_vec = n_elems / 4;  // whole float4s; up to 3 tail elements are handled apart
   const float4* vb = reinterpret_cast<const float4*>(base + begin);
@@ -567,6 +575,157 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
   }
 }
 
+// The finishing kernel for up to ROWS_MAX rows: grid = rows, one CTA per row, no CTA waits for another.
+//  - Before the dependency wait (so under the scan kernel): every CTA derives, from the call's inputs
+//    alone, the width of every row (a row is alive iff every earlier position of its block has width
+//    >= 1) and their exclusive prefix sum; it keeps what its own row needs (first node id relative to the
+//    old node count, width, the previous row's first id = the parent of positions k > 0).
+//  - After the wait: the old node count (a snapshot the scan kernel took of the in/out counter, which
+//    CTA 0 overwrites at the end), the argument checks that need it, then the merge of the row's chunk
+//    lists -- one sortable 64-bit key per candidate (the value mapped to an unsigned integer that grows
+//    with it, -0 as +0 so that equal values tie, then the complement of the id; fillers below every real
+//    entry and distinct by position), every candidate's rank = the number of larger keys, counted by
+//    several threads per candidate -- and the row's own nodes: rank j < width becomes node first + j.
+constexpr int ROWS_THREADS = 256;
+constexpr int ROWS_MAX = 4 * ROWS_THREADS;
+constexpr int MERGE_MAX = 32 * SB_KMAX;  // at most 32 chunk lists per row
+
+__global__ void __launch_bounds__(ROWS_THREADS) expand_rows_kernel(
+    int n_rows, int n_chunks, const float* __restrict__ part_val, const int* __restrict__ part_idx, int block_k,
+    const uint8_t* __restrict__ bucket, int4 bmap, const int* __restrict__ start_parent, int node_budget,
+    int vocab, const int* __restrict__ n0_snapshot, int* __restrict__ n_nodes, int* __restrict__ tok,
+    int* __restrict__ parent, int* __restrict__ depth, int* __restrict__ node_row, int* __restrict__ node_rank,
+    int* __restrict__ topk_tok, float* __restrict__ topk_val, int* __restrict__ status) {
+  __shared__ __align__(16) unsigned long long s_key[MERGE_MAX];
+  __shared__ float s_val[MERGE_MAX];
+  __shared__ int s_rank[MERGE_MAX];
+  __shared__ int s_warp_sum[ROWS_THREADS / 32];
+  __shared__ int s_my[3];  // this CTA's row: first id (relative), width, the previous row's first id (relative)
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rr = blockIdx.x;
+  const int n_cand = n_chunks * SB_KMAX;
+  auto width_of_bucket = [&](int bk) {
+    const int w = bk == 0 ? bmap.x : bk == 1 ? bmap.y : bk == 2 ? bmap.z : bmap.w;
+    return w < vocab ? w : vocab;
+  };
+  // ---- inputs only: widths of all rows, their prefix sums, this row's share -------------------------
+  const int rpt = ceil_div(n_rows, ROWS_THREADS);  // consecutive rows per thread (<= 4)
+  int w_loc[4] = {0, 0, 0, 0};
+  int wsum = 0;
+  bool bad = false;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = tid * rpt + i;
+    if (i < rpt && r < n_rows) {
+      const int kpos = r % block_k;
+      const int bk = bucket[r];
+      bad = bad || bk > 3;
+      bool alive = true;
+      for (int k = 1; k <= kpos; ++k) alive = alive && width_of_bucket(bucket[r - k]) >= 1;
+      w_loc[i] = alive ? width_of_bucket(bk) : 0;
+      wsum += w_loc[i];
+    }
+  }
+  int sp_loc[4] = {-1, -1, -1, -1};  // this thread's share of the starts, checked once the node count is known
+  const int n_starts = n_rows / block_k;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (tid + i * ROWS_THREADS < n_starts) sp_loc[i] = start_parent[tid + i * ROWS_THREADS];
+  const int start = start_parent[rr / block_k];
+  const int start_depth = (start >= 0 && start < node_budget) ? depth[start] : 0;  // an existing node: never rewritten
+  int incl = wsum;
+#pragma unroll
+  for (int sft = 1; sft < 32; sft <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, incl, sft);
+    if (lane >= sft) incl += o;
+  }
+  if (lane == 31) s_warp_sum[warp] = incl;
+  for (int c = tid; c < n_cand; c += ROWS_THREADS) s_rank[c] = 0;
+  __syncthreads();
+  int run = incl - wsum;
+  for (int w = 0; w < warp; ++w) run += s_warp_sum[w];
+  int total = 0;
+  for (int w = 0; w < ROWS_THREADS / 32; ++w) total += s_warp_sum[w];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = tid * rpt + i;
+    if (i < rpt) {
+      if (r == rr) { s_my[0] = run; s_my[1] = w_loc[i]; }
+      if (r == rr - 1) s_my[2] = run;
+      run += w_loc[i];
+    }
+  }
+  pdl_wait();  // the chunk lists and the snapshot of the node count are complete from here on
+  const int n0 = *n0_snapshot;
+  bad = bad || n0 < 0 || n0 > node_budget;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (tid + i * ROWS_THREADS < n_starts) bad = bad || sp_loc[i] < -1 || sp_loc[i] >= n0;
+  // ---- merge this row's chunk lists ----------------------------------------------------------------------
+  const float* pv = part_val + (long long)rr * n_cand;
+  const int* pi = part_idx + (long long)rr * n_cand;
+  for (int c = tid; c < n_cand; c += ROWS_THREADS) {
+    float v = pv[c];
+    const int id = pi[c];
+    s_val[c] = v;
+    if (!(v == v)) v = -INFINITY;
+    uint32_t u = __float_as_uint(v == 0.f ? 0.f : v);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    const uint32_t low = id == kNoId ? 0x7fffffffu - (uint32_t)c : 0xffffffffu - (uint32_t)id;
+    s_key[c] = ((unsigned long long)u << 32) | low;
+  }
+  const int any_bad = __syncthreads_or(bad ? 1 : 0);  // also publishes the keys, s_my and the zeroed counts
+  {
+    // candidate c, part p of the list: `parts` threads share one candidate
+    const int parts = n_cand <= ROWS_THREADS ? ROWS_THREADS / n_cand : 1;
+    const int n_pairs = n_cand / 2;
+    const int per = ceil_div(n_pairs, parts);
+    const ulonglong2* kp = reinterpret_cast<const ulonglong2*>(s_key);
+    for (int w = tid; w < n_cand * parts; w += ROWS_THREADS) {
+      const int c = w % n_cand, part = w / n_cand;
+      const unsigned long long key = s_key[c];
+      const int hi = min(n_pairs, (part + 1) * per);
+      int cnt = 0;
+#pragma unroll 2
+      for (int o = part * per; o < hi; ++o) {
+        const ulonglong2 k2 = kp[o];
+        cnt += (k2.x > key ? 1 : 0) + (k2.y > key ? 1 : 0);
+      }
+      if (cnt) atomicAdd(&s_rank[c], cnt);
+    }
+  }
+  __syncthreads();
+  const int first = n0 + s_my[0], width = s_my[1];
+  const int kpos = rr % block_k;
+  const int par = kpos == 0 ? start : n0 + s_my[2];  // the rank-0 node of the previous position
+  const int node_depth = (start == -1 ? 0 : start_depth + 1) + kpos;
+  for (int c = tid; c < n_cand; c += ROWS_THREADS) {
+    const int rank = s_rank[c];
+    if (rank >= SB_KMAX) continue;
+    const uint32_t low = (uint32_t)s_key[c];
+    const int id = low < 0x80000000u ? -1 : (int)(0xffffffffu - low);
+    topk_tok[rr * SB_KMAX + rank] = id;
+    topk_val[rr * SB_KMAX + rank] = s_val[c];
+    if (!any_bad && rank < width && first + rank < node_budget) {
+      const int n = first + rank;
+      tok[n] = id;
+      parent[n] = par;
+      depth[n] = node_depth;
+      node_row[n] = rr;
+      node_rank[n] = rank;
+    }
+  }
+  if (rr == 0 && tid == 0) {
+    if (any_bad) {
+      *status = SB_ERR_INVALID_ARG;
+    } else {
+      const int n_new = n0 + total;
+      *n_nodes = n_new < node_budget ? n_new : node_budget;
+      *status = SB_OK;
+    }
+  }
+}
+
 // psi(p) of every row from the chunk partials: a warp per row merges the chunk lists (value
 // descending, id ascending) and the chunk statistics (m, s, t):  M = max m_c,
 // S = sum s_c e^(m_c - M), T = sum t_c e^(m_c - M); ln Z = M + ln S; entropy = ln Z - T / S.
@@ -659,6 +818,11 @@ static int topk_chunks(int n_rows, int vocab) {
   return nc;
 }
 
+// Bytes of one kind of chunk lists (values, or ids) of all rows, rounded to 256.
+static size_t topk_list_bytes(int n_rows, int vocab) {
+  return ((size_t)n_rows * topk_chunks(n_rows, vocab) * SB_KMAX * 4 + 255) & ~(size_t)255;
+}
+
 // Dynamic shared memory of topk_partial_reg_kernel: the staged chunk.  Both instantiations are told
 // once that they may exceed the default 48 KB together with their static arrays.
 static size_t topk_stage_bytes(int chunk) {
@@ -676,8 +840,7 @@ static size_t topk_stage_bytes(int chunk) {
 
 extern "C" size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab) {
   if (n_rows < 1 || vocab < 1) return 0;
-  const size_t nc = (size_t)sb::topk_chunks(n_rows, vocab);
-  return 2 * (((size_t)n_rows * nc * SB_KMAX * 4 + 255) & ~(size_t)255);
+  return 2 * sb::topk_list_bytes(n_rows, vocab) + 256;  // value lists, id lists, the snapshot of the node count
 }
 
 extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
@@ -702,17 +865,26 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
   int chunk = ceil_div(vocab, nc);
   chunk = ceil_div(chunk, 4) * 4;
   const bool vec_ok = (reinterpret_cast<uintptr_t>(scores) & 15) == 0 && row_stride % 4 == 0;
+  const size_t list_bytes = topk_list_bytes(n_rows, vocab);
   float* part_val = static_cast<float*>(workspace);
-  int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + need / 2);
+  int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + list_bytes);
+  int* n0_snapshot = reinterpret_cast<int*>(static_cast<char*>(workspace) + 2 * list_bytes);
+  const bool by_rows = n_rows <= ROWS_MAX;  // else the single-CTA finishing kernel, which reads the counter itself
   dim3 grid(nc, n_rows);
   if (vec_ok && chunk <= TOPK_REG_ELEMS)
-    topk_partial_reg_kernel<false><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(scores, row_stride, vocab, chunk, nc, part_val,
-                                                                  part_idx, nullptr);
+    topk_partial_reg_kernel<false><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(
+        scores, row_stride, vocab, chunk, nc, part_val, part_idx, nullptr, n_nodes, by_rows ? n0_snapshot : nullptr);
   else
     topk_partial_kernel<false><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
-                                                              part_idx, nullptr);
+                                                              part_idx, nullptr, n_nodes,
+                                                              by_rows ? n0_snapshot : nullptr);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
+  if (by_rows)
+    return launch_dependent(expand_rows_kernel, dim3(n_rows), dim3(ROWS_THREADS), cs, n_rows, nc, part_val, part_idx,
+                            block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
+                            vocab, n0_snapshot, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val,
+                            status);
   return launch_dependent(expand_finish_kernel, dim3(1), dim3(FINISH_THREADS), cs, n_rows, nc, part_val, part_idx,
                           block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
                           vocab, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val, status);
@@ -736,17 +908,17 @@ extern "C" sb_status sb_rank_features(const float* scores, int64_t row_stride, i
   int chunk = ceil_div(vocab, nc);
   chunk = ceil_div(chunk, 4) * 4;
   const bool vec_ok = (reinterpret_cast<uintptr_t>(scores) & 15) == 0 && row_stride % 4 == 0;
-  const size_t lists = sb_tree_expand_workspace_bytes(n_rows, vocab);
+  const size_t list_bytes = topk_list_bytes(n_rows, vocab);
   float* part_val = static_cast<float*>(workspace);
-  int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + lists / 2);
-  float* part_stats = reinterpret_cast<float*>(static_cast<char*>(workspace) + lists);
+  int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + list_bytes);
+  float* part_stats = reinterpret_cast<float*>(static_cast<char*>(workspace) + 2 * list_bytes);
   dim3 grid(nc, n_rows);
   if (vec_ok && chunk <= TOPK_REG_ELEMS)
     topk_partial_reg_kernel<true><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(scores, row_stride, vocab, chunk, nc, part_val,
-                                                                 part_idx, part_stats);
+                                                                 part_idx, part_stats, nullptr, nullptr);
   else
     topk_partial_kernel<true><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
-                                                             part_idx, part_stats);
+                                                             part_idx, part_stats, nullptr, nullptr);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
   return launch_dependent(rank_features_finish_kernel, dim3(ceil_div(n_rows, 8)), dim3(256), cs, n_rows, nc, vocab,

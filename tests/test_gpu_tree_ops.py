@@ -708,3 +708,16 @@ def test_fuse_project_selector_weights_and_host_errors():
         sb.sb_fuse_project(ct, et, qt, wt, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
     with pytest.raises(sb.SbError):
         sb.sb_fuse_project(ct, et, qt, wt, q_term_valid=True)                         # no q_term to read
+
+
+@pytest.mark.parametrize("n_starts,block_k", [(256, 4), (300, 4), (5, 7), (64, 16), (1, 1)])
+def test_expand_many_rows_and_other_block_lengths(n_starts, block_k):
+    """Up to 1024 rows one CTA per row finishes the expansion; beyond that a single CTA does
+    (256 x 4 = 1024 rows is the last size of the first kind, 300 x 4 the second kind)."""
+    rng = W.rng_for(200 + n_starts)
+    case = W.make_expand_case(rng, n_starts=n_starts, block_k=block_k, vocab=700, bmap=[2, 3, 4, 0],
+                              node_budget=128, existing_parent=W.random_tree(rng, 9, 3), tie_rows=3)
+    _check_expand(case)
+    roomy = W.make_expand_case(rng, n_starts=n_starts, block_k=block_k, vocab=90, bmap=[1, 2, 3, 1],
+                               node_budget=128 if n_starts > 20 else 4096)
+    _check_expand(roomy)
