@@ -22,8 +22,10 @@ __device__ inline void mbar_arrive(uint64_t* bar) {
 }
 // Bounded wait: gives up after two seconds of wall time, or as soon as another thread of the CTA
 // has given up, and returns false; the caller then skips its remaining work and the kernel ends.
-__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  const uint32_t addr = smem_u32(bar);
+// The first probe (which the hardware already holds for a while) is inline; the polling loop with its
+// clock and abort checks is one shared out-of-line copy, so that the dozens of waits of a kernel cost
+// a few instructions each in its code.
+static __device__ __noinline__ bool mbar_wait_poll(uint32_t addr, uint32_t parity, volatile int* abort_flag) {
   unsigned long long t0 = 0;
   for (int it = 0;; ++it) {
     uint32_t ok;
@@ -43,6 +45,17 @@ __device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* a
   }
   *abort_flag = 1;
   return false;
+}
+__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const uint32_t addr = smem_u32(bar);
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok)
+      : "r"(addr), "r"(parity)
+      : "memory");
+  if (ok) return true;
+  return mbar_wait_poll(addr, parity, abort_flag);
 }
 __device__ inline void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
