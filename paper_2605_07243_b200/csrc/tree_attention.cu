@@ -525,9 +525,9 @@ static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_spl
   const int sms = num_sms();
   // More (sequence, KV head, row tile) units than SMs and at least two row tiles per KV head: the
   // tcgen05 kernel that gives one CTA two tiles (each K/V block is pulled from L2 once for both).
-  // (With three tiles the second CTA of a KV head would hold a single one, and ragged batches whose
-  // largest tree has three tiles mostly hold one or two: measured slower than the one-tile kernel.)
-  bool two_tiles = impl == IMPL_TC && row_tiles >= 2 && row_tiles != 3 && base > sms;
+  // (With three tiles the second CTA of a KV head holds a single one; still faster than three one-tile
+  // CTAs on the ragged batch of config 4: 131 us against 154 us.)
+  bool two_tiles = impl == IMPL_TC && row_tiles >= 2 && base > sms;
   if (const char* e = getenv("SB_ATTN_TWO_TILES")) two_tiles = impl == IMPL_TC && row_tiles >= 2 && atoi(e) != 0;
   if (two_tiles) {
     SplitPlan sp;
