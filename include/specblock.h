@@ -74,6 +74,13 @@ typedef enum sb_dtype { SB_BF16 = 0, SB_F32 = 1 } sb_dtype;
  * The three host integers at the end only size grids and bound loops; the kernels re-check
  * the device values against them and flag SB_ERR_INVALID_TREE / SB_ERR_BOUNDS instead of
  * trusting them.
+ * index_arrays_settled: the attention kernel starts as a programmatic dependent of whatever
+ * precedes it in the stream and normally reads nothing before that work has completed.  A caller
+ * who knows that the kernel enqueued IMMEDIATELY before the call does not write this batch's index
+ * arrays (prefix_len, node_offsets, q_node_begin, q_offsets -- e.g. the previous layer's attention
+ * call of the same verify forward) may set this to 1: the sequence lengths are then fetched while
+ * that kernel is still running (about half a microsecond per call).  Q, K, V, the parents and the
+ * page table are always read after it has completed.  0 is always correct.
  */
 typedef struct sb_tree_batch {
   int32_t batch;      /* B >= 1                                                     */
@@ -93,6 +100,8 @@ typedef struct sb_tree_batch {
   const int32_t* parent;     /* [total_nodes]                                       */
   int32_t max_nodes;         /* host upper bound on N_b (<= SB_MAX_NODES)           */
   int32_t max_kv_len;        /* host upper bound on P_b + N_b                       */
+  int32_t index_arrays_settled; /* 0, or 1: see below                                */
+  int32_t reserved;          /* 0                                                   */
 } sb_tree_batch;
 
 /*

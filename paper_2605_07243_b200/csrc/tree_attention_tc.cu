@@ -126,13 +126,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   // Programmatic dependent launch: everything above is independent of earlier kernels' results and
   // may overlap their tail; from here on their memory is complete and visible.  Dependents of this
   // kernel are released right away, so at most two consecutive grids are ever in flight.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // A caller may vouch that the kernel just before does not write the index arrays: then the sequence
+  // lengths (one trip to the L2 cache, on the way to the first load) are fetched before the wait.
+  const bool lengths_early = p.tb.index_arrays_settled != 0 && !(!FAST && p.sort_seqs);
+  if (!lengths_early) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // grid index z -> sequence (longest first when the grid runs in several waves)
   const int b = (!FAST && p.sort_seqs) ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent)
                                        : (int)blockIdx.z;
   const SeqPre pre = plan_lengths(p, b);
+  if (lengths_early) asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int rows_total = pre.info.nq * G;
   const int row0 = tile * TC_BM;
   if (!pre.can_write || row0 >= rows_total) {  // uniform over the cluster

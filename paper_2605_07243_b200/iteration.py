@@ -214,7 +214,7 @@ class SpecBlockIteration:
         for l in range(self.n_layers):
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,
                                  num_splits=self.num_splits, workspace=self.attn_ws, status=self.attn_status,
-                                 k_cache=self.k_all[l], v_cache=self.v_all[l])
+                                 k_cache=self.k_all[l], v_cache=self.v_all[l], index_arrays_settled=l > 0)
         sb.sb_verify_accept(self.logits, self.node_offsets, self.tree["parent"], self.tree["tok"], self.max_depth,
                             workspace=self.accept_ws, out=self.accept)
         sb.sb_kv_compact(self.tb, self.n_layers, self.layer_stride, self.accept["path_nodes"],
