@@ -232,24 +232,23 @@ def run_ours(args):
         g_expand = capture(torch, step.run_expand)
         g_accept = capture(torch, step.run_accept)
         g_compact = capture(torch, step.run_compact)
-        step.run_rank_features()
-        g_features = capture(torch, step.run_rank_features)
-        step.run_signal()
-        g_signal = capture(torch, step.run_signal)
-        step.run_sample()
-        g_sample = capture(torch, step.run_sample)
-        step.run_shift_all()
-        g_shift = capture(torch, step.run_shift_all)
-        step.run_fuse_all()
-        g_fuse = capture(torch, step.run_fuse_all)
-        # one whole iteration (two drafter blocks growing the tree on the device, then the verify forward on it)
-        from paper_2605_07243_b200.iteration import build_8b_iteration
-        iteration = build_8b_iteration(layers, ver.logits, ver.max_depth, num_splits=args.num_splits)
-        iteration.run()
-        side.synchronize()
-        assert int(iteration.attn_status.max()) == 0 and int(iteration.accept["status"].max()) == 0
-        assert all(int(e["status"][0]) == 0 for e in iteration.blocks)
-        g_iter = capture(torch, iteration.run)
+        extras = []   # pieces outside the step (the "next" rows), timed on their own
+        if not args.step_only:
+            for name, fn in (("rank_features_not_in_step", step.run_rank_features),
+                             ("verifier_signal_not_in_step", step.run_signal),
+                             ("verify_sample_T1_not_in_step", step.run_sample),
+                             ("shift_project_32x4096_not_in_step", step.run_shift_all),
+                             ("fuse_project_8x4x4096_not_in_step", step.run_fuse_all)):
+                fn()
+                extras.append((name, capture(torch, fn)))
+            # one whole iteration (two drafter blocks growing the tree on the device, then the verify forward on it)
+            from paper_2605_07243_b200.iteration import build_8b_iteration
+            iteration = build_8b_iteration(layers, ver.logits, ver.max_depth, num_splits=args.num_splits)
+            iteration.run()
+            side.synchronize()
+            assert int(iteration.attn_status.max()) == 0 and int(iteration.accept["status"].max()) == 0
+            assert all(int(e["status"][0]) == 0 for e in iteration.blocks)
+            extras.append(("whole_iteration_2_blocks_32_layers_not_in_step", capture(torch, iteration.run)))
 
         for _ in range(max(args.warmup, 3)):
             g_step.replay()
@@ -277,17 +276,13 @@ def run_ours(args):
         keep_busy(0.4)
         clocks = sampler.stop()
         parts_ms = {}
-        for name, g in (("expand", g_expand), ("accept", g_accept), ("compact", g_compact),
-                        ("rank_features_not_in_step", g_features), ("verifier_signal_not_in_step", g_signal),
-                        ("verify_sample_T1_not_in_step", g_sample),
-                        ("shift_project_32x4096_not_in_step", g_shift),
-                        ("fuse_project_8x4x4096_not_in_step", g_fuse),
-                        ("whole_iteration_2_blocks_32_layers_not_in_step", g_iter)):
+        for name, g in [("expand", g_expand), ("accept", g_accept), ("compact", g_compact)] + extras:
             for _ in range(3):
                 g.replay()
             parts_ms[name] = time_graph(torch, g, 20, False) / 20
-        parts_ms["shift_project_32x4096_not_in_step"] /= step.SHIFT_SETS   # one graph = one call per weight set
-        parts_ms["fuse_project_8x4x4096_not_in_step"] /= step.FUSE_SETS
+        if "shift_project_32x4096_not_in_step" in parts_ms:   # one graph = one call per weight set
+            parts_ms["shift_project_32x4096_not_in_step"] /= step.SHIFT_SETS
+            parts_ms["fuse_project_8x4x4096_not_in_step"] /= step.FUSE_SETS
 
         # end to end: inputs in pinned host memory, results back to pinned host memory
         e2e_steps = 1 if args.quick else max(3, min(args.steps, 5))
@@ -367,6 +362,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--num-splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--step-only", action="store_true",
+                    help="profiling aid: leave out the pieces timed outside the step (their kernels then do not appear)")
     ap.add_argument("--quick", action="store_true",
                     help="profiling aid: no clock-sampling busy loops, a single end-to-end step, no CPU baseline")
     args = ap.parse_args()
