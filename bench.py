@@ -346,6 +346,22 @@ def run_ours(args):
                                 "kind": "oracle", "seconds": dt,
                                 "sample": "one whole step (all 32 attention layers, acceptance, expansion, "
                                           "compaction) on the fp64 oracle, once"}
+    if rank == 0 and world == 1 and args.oracle_configs:
+        # The oracle's tree attention on each of the five benchmark configurations, once, on the host
+        # cores (the counterpart of `python -m paper_2605_07243_b200.time_configs`); a baseline only.
+        import oracle
+        from paper_2605_07243_b200 import workloads as W
+        makers = {1: lambda: W.config1_tiny()[0], 2: W.config2_verify_layer, 3: lambda: W.config3_drafter()[0],
+                  4: lambda: W.config4_batched(with_logits=False)[0], 5: lambda: W.config5_long(with_logits=False)[0]}
+        by_config = {}
+        for c in [int(x) for x in args.oracle_configs.split(",")]:
+            case = makers[c]()
+            t0 = time.perf_counter()
+            oracle.tree_attention(**case.oracle_kwargs())
+            dt = time.perf_counter() - t0
+            by_config[str(c)] = {"seconds": dt, "GB/s": case.algorithmic_bytes() / dt / 1e9,
+                                 "GFLOP/s": case.flops() / dt / 1e9}
+        line["cpu_baseline_attention_by_config"] = {"cores": oracle.num_threads(), "kind": "oracle", "configs": by_config}
     if dist_on:
         torch.distributed.barrier()
         torch.distributed.destroy_process_group()
@@ -362,6 +378,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--num-splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--oracle-configs", default="",
+                    help="also time the CPU oracle's tree attention on these benchmark configurations (e.g. 1,2,3,4,5)")
     ap.add_argument("--step-only", action="store_true",
                     help="profiling aid: leave out the pieces timed outside the step (their kernels then do not appear)")
     ap.add_argument("--quick", action="store_true",
