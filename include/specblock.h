@@ -279,7 +279,9 @@ size_t sb_fuse_project_workspace_bytes(int32_t n_starts, int32_t block_k, int32_
  *   out_tokens = accepted tokens then the bonus, bonus).
  *   status int32 [batch]: SB_OK, SB_ERR_INVALID_TREE, or SB_ERR_BOUNDS when an inner node of the walk
  *   has no valid child_row (outputs of that sequence: accept_len 0, -1 elsewhere).
- *   workspace: sb_verify_sample_workspace_bytes(batch, vocab) = batch * 2 * vocab floats, 16-byte aligned.
+ *   workspace: sb_verify_sample_workspace_bytes(batch, vocab, total_nodes, n_rows) bytes, 256-byte aligned (vocab
+ *   floats per sequence for the residual distribution after a rejection, and the per-chunk softmax statistics of
+ *   every target and draft row, which a first pair of kernels computes over the whole GPU).
  *   Probabilities and sums are fp32; a decision whose two sides differ by less than about 1e-5
  *   relative may fall either way.
  */
@@ -290,7 +292,7 @@ sb_status sb_verify_sample(const void* logits, sb_dtype dtype, int64_t row_strid
                            const float* u_accept, const float* u_bonus, int32_t max_depth, int32_t* accept_len,
                            int32_t* path_nodes, int32_t* out_tokens, int32_t* bonus, void* workspace,
                            size_t workspace_bytes, int32_t* status, void* stream);
-size_t sb_verify_sample_workspace_bytes(int32_t batch, int32_t vocab);
+size_t sb_verify_sample_workspace_bytes(int32_t batch, int32_t vocab, int32_t total_nodes, int32_t n_rows);
 
 /*
  * sb_verifier_signal -- one iteration's term of the verifier-derived update signal

@@ -280,8 +280,9 @@ def sb_verifier_signal(scores, node_offsets, child_row, path_nodes, accept_len, 
     return dict(r_prob=r_prob, signal=signal, status=status)
 
 
-def sb_verify_sample_workspace_bytes(batch: int, vocab: int) -> int:
-    return int(load().sb_verify_sample_workspace_bytes(C.c_int32(batch), C.c_int32(vocab)))
+def sb_verify_sample_workspace_bytes(batch: int, vocab: int, total_nodes: int, n_rows: int) -> int:
+    return int(load().sb_verify_sample_workspace_bytes(C.c_int32(batch), C.c_int32(vocab), C.c_int32(total_nodes),
+                                                       C.c_int32(n_rows)))
 
 
 def sb_verify_sample(logits, scores, node_offsets, parent, tok, child_row, temperature, u_accept, u_bonus, max_depth,
@@ -300,7 +301,8 @@ def sb_verify_sample(logits, scores, node_offsets, parent, tok, child_row, tempe
                    out_tokens=torch.empty((batch, max_depth + 1), **i32), bonus=torch.empty(batch, **i32),
                    status=torch.empty(batch, **i32))
     if workspace is None:
-        workspace = torch.empty(max(sb_verify_sample_workspace_bytes(batch, vocab), 16), dtype=torch.uint8, device=dev)
+        workspace = torch.empty(max(sb_verify_sample_workspace_bytes(batch, vocab, total, n_rows), 256), dtype=torch.uint8,
+                                device=dev)
     rc = load().sb_verify_sample(
         _ptr(logits), C.c_int(dt), C.c_int64(stride), C.c_int32(vocab), _ptr(scores, torch.float32), C.c_int64(sstride),
         C.c_int32(n_rows), C.c_int32(batch), C.c_int32(total), _ptr(node_offsets, torch.int32),

@@ -158,7 +158,8 @@ class VerifyStep:
             e["u_accept"] = torch.rand(n, generator=gen).to(self.device)
             e["u_bonus"] = torch.rand(B, generator=gen).to(self.device)
             V = self.logits.shape[1]
-            e["sample_ws"] = torch.empty(max(16, sb.sb_verify_sample_workspace_bytes(B, V)), dtype=torch.uint8,
+            e["sample_ws"] = torch.empty(max(256, sb.sb_verify_sample_workspace_bytes(B, V, n, e["scores"].shape[0])),
+                                         dtype=torch.uint8,
                                          device=self.device)
             i32 = dict(dtype=torch.int32, device=self.device)
             e["sample_out"] = dict(accept_len=torch.empty(B, **i32),
