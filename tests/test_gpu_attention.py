@@ -330,3 +330,17 @@ def test_random_shapes_against_oracle(seed, monkeypatch):
         monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
     check_attention(case, f"random shape {seed}: B={B} Hkv={hkv} G={G} D={D} page={page} splits={splits}",
                     num_splits=splits)
+
+
+def test_index_arrays_settled_gives_the_same_bits():
+    """The flag only moves the fetch of the sequence lengths ahead of the dependency wait: same results,
+    on the compile-time variant (config 2), a paged ragged batch and a drafter call with cached nodes."""
+    rng = W.rng_for(431)
+    ragged = W.make_attn_case(rng, parents=[W.random_tree(rng, 40, 6), W.chain_tree(7), W.random_tree(rng, 90, 9)],
+                              prefix_lens=[700, 33, 0], n_q_heads=16, n_kv_heads=4, head_dim=128, page_size=64)
+    for case in (W.config2_verify_layer(prefix=600), ragged, W.config3_drafter(prefix=900)[0]):
+        plain = gpu_attention(case)
+        flagged = gpu_attention(case, index_arrays_settled=True)
+        for a, b in zip(plain, flagged):
+            np.testing.assert_array_equal(a, b)
+        assert (plain[2] == 0).all()
