@@ -235,6 +235,7 @@ def run_ours(args):
         extras = []   # pieces outside the step (the "next" rows), timed on their own
         if not args.step_only:
             for name, fn in (("rank_features_not_in_step", step.run_rank_features),
+                             ("expand_and_rank_features_one_pass_not_in_step", step.run_expand_features),
                              ("verifier_signal_not_in_step", step.run_signal),
                              ("verify_sample_T1_not_in_step", step.run_sample),
                              ("shift_project_32x4096_not_in_step", step.run_shift_all),

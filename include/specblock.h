@@ -11,6 +11,7 @@
  *   sb_tree_attention  tree-masked attention over prefix KV + ancestors (Sec. 3.1, App. A.2, Alg. 1 "verify")
  *   sb_tree_expand     per-row top-k + bucket-driven branching          (Sec. 3.2, App. A.5, Alg. 1 "attach")
  *   sb_rank_features   15-dim summary of each draft distribution        (Sec. 3.2, App. B)
+ *   sb_tree_expand_features  both of the above from one pass over the scores
  *   sb_verifier_signal verifier-derived update signal s = sum (1 - r)   (Sec. 3.4, Alg. 2)
  *   sb_verify_sample   stochastic (temperature > 0) tree verification   (Sec. 4.1, Sec. 4.2)
  *   sb_shift_project   layer-wise shift projection between drafter layers (Sec. 3.1)
@@ -197,6 +198,20 @@ size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab);
 sb_status sb_rank_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
                            float* features, void* workspace, size_t workspace_bytes, void* stream);
 size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
+
+/*
+ * sb_tree_expand_features -- sb_tree_expand and sb_rank_features of the same scores in ONE pass over them:
+ * the scan that finds the per-chunk top-16 also accumulates the chunk statistics of psi(p), and both
+ * finishing kernels follow it.  Arguments as sb_tree_expand plus features fp32 [n_rows][15] as
+ * sb_rank_features; results identical to the two separate calls.
+ *   workspace : sb_rank_features_workspace_bytes(n_rows, vocab) bytes, 256-byte aligned.
+ */
+sb_status sb_tree_expand_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                                  int32_t block_k, const uint8_t* bucket, const int32_t* bmap /*host[4]*/,
+                                  const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
+                                  int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
+                                  int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features,
+                                  void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 
 /*
  * sb_shift_project -- the layer-wise shift between consecutive decoder layers of the drafter

@@ -69,7 +69,7 @@ def load(build_if_missing: bool = True):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
                  "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal", "sb_verify_sample",
-                 "sb_shift_project", "sb_fuse_project"):
+                 "sb_shift_project", "sb_fuse_project", "sb_tree_expand_features"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -80,7 +80,7 @@ EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspa
             "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
             "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_verifier_signal", "sb_verify_sample",
             "sb_verify_sample_workspace_bytes", "sb_shift_project", "sb_shift_project_workspace_bytes",
-            "sb_fuse_project", "sb_fuse_project_workspace_bytes", "sb_status_string",
+            "sb_fuse_project", "sb_fuse_project_workspace_bytes", "sb_tree_expand_features", "sb_status_string",
             "sb_version",
             "sb_kernel_launch_count")
 
@@ -413,10 +413,12 @@ def sb_tree_expand_workspace_bytes(n_rows: int, vocab: int) -> int:
 
 
 def sb_tree_expand(scores, block_k, bucket, bmap, start_parent, node_budget, tree, *, vocab=None,
-                   workspace=None, topk_tok=None, topk_val=None, status=None):
+                   workspace=None, topk_tok=None, topk_val=None, status=None, features=None):
     """scores fp32 [R, stride]; bucket uint8 [R]; bmap: 4 host ints; tree: dict of int32 device
     tensors n_nodes [1], tok, parent, depth, node_row, node_rank (capacity node_budget), updated
-    in place.  -> (topk_tok [R,16], topk_val [R,16], status [1])."""
+    in place.  -> (topk_tok [R,16], topk_val [R,16], status [1]).
+    features fp32 [R, 15]: also filled (sb_tree_expand_features: one pass over the scores for both);
+    the workspace must then hold sb_rank_features_workspace_bytes."""
     n_rows, stride = scores.shape
     vocab = stride if vocab is None else vocab
     dev = scores.device
@@ -425,16 +427,19 @@ def sb_tree_expand(scores, block_k, bucket, bmap, start_parent, node_budget, tre
     status = torch.empty(1, dtype=torch.int32, device=dev) if status is None else status
     lib = load()
     if workspace is None:
-        need = sb_tree_expand_workspace_bytes(n_rows, vocab)
+        need = (sb_tree_expand_workspace_bytes if features is None else sb_rank_features_workspace_bytes)(n_rows, vocab)
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     bm = (C.c_int32 * 4)(*[int(x) for x in bmap])
-    rc = lib.sb_tree_expand(_ptr(scores, torch.float32), C.c_int64(stride), C.c_int32(n_rows),
-                            C.c_int32(vocab), C.c_int32(block_k), _ptr(bucket, torch.uint8), bm,
-                            _ptr(start_parent, torch.int32), C.c_int32(node_budget),
-                            _ptr(tree["n_nodes"], torch.int32), _ptr(tree["tok"], torch.int32),
-                            _ptr(tree["parent"], torch.int32), _ptr(tree["depth"], torch.int32),
-                            _ptr(tree["node_row"], torch.int32), _ptr(tree["node_rank"], torch.int32),
-                            _ptr(topk_tok, torch.int32), _ptr(topk_val, torch.float32), _ptr(workspace),
-                            C.c_size_t(workspace.numel()), _ptr(status, torch.int32), _stream())
-    _check(rc, "sb_tree_expand")
+    head = (_ptr(scores, torch.float32), C.c_int64(stride), C.c_int32(n_rows),
+            C.c_int32(vocab), C.c_int32(block_k), _ptr(bucket, torch.uint8), bm,
+            _ptr(start_parent, torch.int32), C.c_int32(node_budget),
+            _ptr(tree["n_nodes"], torch.int32), _ptr(tree["tok"], torch.int32),
+            _ptr(tree["parent"], torch.int32), _ptr(tree["depth"], torch.int32),
+            _ptr(tree["node_row"], torch.int32), _ptr(tree["node_rank"], torch.int32),
+            _ptr(topk_tok, torch.int32), _ptr(topk_val, torch.float32))
+    tail = (_ptr(workspace), C.c_size_t(workspace.numel()), _ptr(status, torch.int32), _stream())
+    if features is None:
+        _check(lib.sb_tree_expand(*head, *tail), "sb_tree_expand")
+    else:
+        _check(lib.sb_tree_expand_features(*head, _ptr(features, torch.float32), *tail), "sb_tree_expand_features")
     return topk_tok, topk_val, status

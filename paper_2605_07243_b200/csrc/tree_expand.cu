@@ -843,12 +843,13 @@ extern "C" size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab) 
   return 2 * sb::topk_list_bytes(n_rows, vocab) + 256;  // value lists, id lists, the snapshot of the node count
 }
 
-extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
-                                    int32_t block_k, const uint8_t* bucket, const int32_t* bmap,
-                                    const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
-                                    int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
-                                    int32_t* node_rank, int32_t* topk_tok, float* topk_val, void* workspace,
-                                    size_t workspace_bytes, int32_t* status, void* stream) {
+// sb_tree_expand, and with `features` the distribution summaries of sb_rank_features from the same scan.
+static sb_status expand_impl(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                             int32_t block_k, const uint8_t* bucket, const int32_t* bmap,
+                             const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
+                             int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
+                             int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features, void* workspace,
+                             size_t workspace_bytes, int32_t* status, void* stream) {
   using namespace sb;
   if (!scores || !bucket || !bmap || !start_parent || !n_nodes || !tok || !parent || !depth || !node_row ||
       !node_rank || !topk_tok || !topk_val || !status || n_rows < 1 || vocab < 1 || row_stride < vocab ||
@@ -857,7 +858,7 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
   for (int m = 0; m < 4; ++m)
     if (bmap[m] < 0 || bmap[m] > SB_KMAX) return SB_ERR_INVALID_ARG;
   if (n_rows > 65535 || block_k > FINISH_THREADS) return SB_ERR_UNSUPPORTED;
-  const size_t need = sb_tree_expand_workspace_bytes(n_rows, vocab);
+  const size_t need = features ? sb_rank_features_workspace_bytes(n_rows, vocab) : sb_tree_expand_workspace_bytes(n_rows, vocab);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255))
     return SB_ERR_WORKSPACE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
@@ -869,25 +870,62 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
   float* part_val = static_cast<float*>(workspace);
   int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + list_bytes);
   int* n0_snapshot = reinterpret_cast<int*>(static_cast<char*>(workspace) + 2 * list_bytes);
+  float* part_stats = features ? reinterpret_cast<float*>(static_cast<char*>(workspace) + 2 * list_bytes + 256) : nullptr;
   const bool by_rows = n_rows <= ROWS_MAX;  // else the single-CTA finishing kernel, which reads the counter itself
+  int* snap = by_rows ? n0_snapshot : nullptr;
   dim3 grid(nc, n_rows);
-  if (vec_ok && chunk <= TOPK_REG_ELEMS)
-    topk_partial_reg_kernel<false><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(
-        scores, row_stride, vocab, chunk, nc, part_val, part_idx, nullptr, n_nodes, by_rows ? n0_snapshot : nullptr);
+  const bool reg = vec_ok && chunk <= TOPK_REG_ELEMS;
+  if (reg && features)
+    topk_partial_reg_kernel<true><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(scores, row_stride, vocab, chunk, nc,
+                                                                                    part_val, part_idx, part_stats, n_nodes, snap);
+  else if (reg)
+    topk_partial_reg_kernel<false><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(scores, row_stride, vocab, chunk, nc,
+                                                                                     part_val, part_idx, nullptr, n_nodes, snap);
+  else if (features)
+    topk_partial_kernel<true><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val, part_idx,
+                                                             part_stats, n_nodes, snap);
   else
-    topk_partial_kernel<false><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val,
-                                                              part_idx, nullptr, n_nodes,
-                                                              by_rows ? n0_snapshot : nullptr);
+    topk_partial_kernel<false><<<grid, TOPK_THREADS, 0, cs>>>(scores, row_stride, vocab, chunk, nc, vec_ok, part_val, part_idx,
+                                                              nullptr, n_nodes, snap);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
   if (by_rows)
-    return launch_dependent(expand_rows_kernel, dim3(n_rows), dim3(ROWS_THREADS), cs, n_rows, nc, part_val, part_idx,
-                            block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
-                            vocab, n0_snapshot, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val,
-                            status);
-  return launch_dependent(expand_finish_kernel, dim3(1), dim3(FINISH_THREADS), cs, n_rows, nc, part_val, part_idx,
+    st = launch_dependent(expand_rows_kernel, dim3(n_rows), dim3(ROWS_THREADS), cs, n_rows, nc, part_val, part_idx,
+                          block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
+                          vocab, n0_snapshot, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val,
+                          status);
+  else
+    st = launch_dependent(expand_finish_kernel, dim3(1), dim3(FINISH_THREADS), cs, n_rows, nc, part_val, part_idx,
                           block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
                           vocab, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val, status);
+  if (st != SB_OK || !features) return st;
+  // the summaries read the same chunk lists and the chunk statistics; as a dependent of the finishing kernel
+  // (which waited for the scan) their wait covers the scan too
+  return launch_dependent(rank_features_finish_kernel, dim3(ceil_div(n_rows, 8)), dim3(256), cs, n_rows, nc, vocab,
+                          part_val, part_idx, part_stats, features);
+}
+
+extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                                    int32_t block_k, const uint8_t* bucket, const int32_t* bmap,
+                                    const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
+                                    int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
+                                    int32_t* node_rank, int32_t* topk_tok, float* topk_val, void* workspace,
+                                    size_t workspace_bytes, int32_t* status, void* stream) {
+  return expand_impl(scores, row_stride, n_rows, vocab, block_k, bucket, bmap, start_parent, node_budget, n_nodes, tok,
+                     parent, depth, node_row, node_rank, topk_tok, topk_val, nullptr, workspace, workspace_bytes, status,
+                     stream);
+}
+
+extern "C" sb_status sb_tree_expand_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
+                                             int32_t block_k, const uint8_t* bucket, const int32_t* bmap,
+                                             const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
+                                             int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
+                                             int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features,
+                                             void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+  if (!features) return SB_ERR_INVALID_ARG;
+  return expand_impl(scores, row_stride, n_rows, vocab, block_k, bucket, bmap, start_parent, node_budget, n_nodes, tok,
+                     parent, depth, node_row, node_rank, topk_tok, topk_val, features, workspace, workspace_bytes, status,
+                     stream);
 }
 
 extern "C" size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab) {
@@ -911,7 +949,7 @@ extern "C" sb_status sb_rank_features(const float* scores, int64_t row_stride, i
   const size_t list_bytes = topk_list_bytes(n_rows, vocab);
   float* part_val = static_cast<float*>(workspace);
   int* part_idx = reinterpret_cast<int*>(static_cast<char*>(workspace) + list_bytes);
-  float* part_stats = reinterpret_cast<float*>(static_cast<char*>(workspace) + 2 * list_bytes);
+  float* part_stats = reinterpret_cast<float*>(static_cast<char*>(workspace) + 2 * list_bytes + 256);
   dim3 grid(nc, n_rows);
   if (vec_ok && chunk <= TOPK_REG_ELEMS)
     topk_partial_reg_kernel<true><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(scores, row_stride, vocab, chunk, nc, part_val,

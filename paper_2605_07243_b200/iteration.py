@@ -12,8 +12,8 @@ Per drafter block m (Algorithm 1, the loop over m):
     W_fuse        per-position inputs from c, the embedding and the position queries  (sb_fuse_project)
     L_d layers    tree attention over the drafter's cache, then the layer-wise shift  (sb_tree_attention,
                   sb_shift_project)
-    psi(p)        the rank head's distribution summary of every row                   (sb_rank_features)
-    attach        top-b tokens of every row under the block's starts                  (sb_tree_expand)
+    psi(p)        the rank head's distribution summary of every row   } one pass over  (sb_tree_expand_features)
+    attach        top-b tokens of every row under the block's starts  } the scores
 then  verify:     ancestor masks, tree attention of every target layer, greedy acceptance, compaction.
 
 The pieces that need trained weights are not in the library (the decoder layers' own projections
@@ -205,9 +205,10 @@ class SpecBlockIteration:
             if l < len(e.get("hidden", [])):
                 sb.sb_shift_project(e["hidden"][l], w["w_shift"][l], self.block_k, out=e["shifted"][l],
                                     workspace=e["shift_ws"], status=e["shift_status"])
-        sb.sb_rank_features(e["scores"], features=e["features"], workspace=e["features_ws"])
+        # psi(p) and the expansion read the same scores: one pass over them serves both
         sb.sb_tree_expand(e["scores"], self.block_k, e["bucket"], self.bmap, e["start_parent"], self.budget, self.tree,
-                          workspace=e["ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"], status=e["status"])
+                          workspace=e["features_ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"], status=e["status"],
+                          features=e["features"])
 
     def run_verify(self):
         sb.sb_tree_ancestors(self.node_offsets, self.tree["parent"], self.budget, self.anc, self.depth, self.anc_status)

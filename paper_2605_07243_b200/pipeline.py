@@ -127,6 +127,19 @@ class VerifyStep:
                                            device=self.device)
         return sb.sb_rank_features(e["scores"], features=e["features"], workspace=e["features_ws"])
 
+    def run_expand_features(self):
+        """The expansion and psi(p) of the same scores from ONE pass over them (sb_tree_expand_features); not part
+        of run_device(), timed on its own beside run_expand() and run_rank_features()."""
+        e = self.expand
+        if e is None:
+            return None
+        self.run_rank_features() if "features" not in e else None
+        e["n_nodes"].copy_(e["n_nodes0"])
+        tree = dict(e["tree"], n_nodes=e["n_nodes"])
+        sb.sb_tree_expand(e["scores"], e["block_k"], e["bucket"], e["bmap"], e["start_parent"], e["budget"], tree,
+                          workspace=e["features_ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"], status=e["status"],
+                          features=e["features"])
+
     def run_signal(self):
         """One iteration's term of the verifier-derived update signal, chained after run_accept() (not
         part of run_device(): a 'next' row, timed on its own).  The benchmark's tree and drafter rows

@@ -721,3 +721,41 @@ def test_expand_many_rows_and_other_block_lengths(n_starts, block_k):
     roomy = W.make_expand_case(rng, n_starts=n_starts, block_k=block_k, vocab=90, bmap=[1, 2, 3, 1],
                                node_budget=128 if n_starts > 20 else 4096)
     _check_expand(roomy)
+
+
+def test_expand_with_features_in_one_pass():
+    """sb_tree_expand_features = sb_tree_expand + sb_rank_features from one scan: same tree, same summaries."""
+    for case in (W.config3_drafter()[1],
+                 W.make_expand_case(W.rng_for(230), n_starts=5, block_k=3, vocab=777, bmap=[2, 3, 4, 0], node_budget=40,
+                                    existing_parent=W.random_tree(W.rng_for(231), 6, 3), tie_rows=2)):
+        R, V = case.scores.shape
+        scores = torch.from_numpy(case.scores).cuda()
+
+        def fresh_tree():
+            n0 = 0 if case.tree is None else len(case.tree["tok"])
+            t = {k: torch.full((case.node_budget,), -1, dtype=torch.int32, device="cuda")
+                 for k in ("tok", "parent", "depth", "node_row", "node_rank")}
+            if case.tree is not None:
+                for k in t:
+                    t[k][:n0] = dev.i32_tensor(case.tree[k])
+            t["n_nodes"] = torch.tensor([n0], dtype=torch.int32, device="cuda")
+            return t
+
+        args = (scores, case.block_k, torch.from_numpy(case.bucket).cuda(), case.bmap, dev.i32_tensor(case.start_parent),
+                case.node_budget)
+        t_sep, t_fused = fresh_tree(), fresh_tree()
+        tok_a, val_a, st_a = sb.sb_tree_expand(*args, t_sep)
+        feat_sep = sb.sb_rank_features(scores)
+        feat_fused = torch.full((R, 15), float("nan"), dtype=torch.float32, device="cuda")
+        tok_b, val_b, st_b = sb.sb_tree_expand(*args, t_fused, features=feat_fused)
+        torch.cuda.synchronize()
+        assert int(st_a.cpu()[0]) == 0 and int(st_b.cpu()[0]) == 0
+        assert torch.equal(tok_a, tok_b) and torch.equal(val_a, val_b)
+        for k in t_sep:
+            assert torch.equal(t_sep[k], t_fused[k]), k
+        assert torch.equal(feat_sep.view(torch.int32), feat_fused.view(torch.int32))
+        ref = oracle.rank_features(case.scores)
+        got = feat_fused.cpu().numpy().astype(np.float64)
+        fin = np.isfinite(ref)
+        assert (np.abs(got[fin] - ref[fin]) <= 2e-5 * np.maximum(1, np.abs(ref[fin]))).all()
+        assert (got[~fin] == ref[~fin]).all()
