@@ -759,3 +759,15 @@ def test_expand_with_features_in_one_pass():
         fin = np.isfinite(ref)
         assert (np.abs(got[fin] - ref[fin]) <= 2e-5 * np.maximum(1, np.abs(ref[fin]))).all()
         assert (got[~fin] == ref[~fin]).all()
+
+
+@pytest.mark.parametrize("vocab,dtype,pad", [(131071, "f32", 3), (130000, "bf16", 5), (131072, "f32", 0), (200000, "bf16", 0)])
+def test_verify_sample_large_vocabularies_and_unaligned_rows(vocab, dtype, pad):
+    """Segments of exactly 512 tokens take the register-resident runs (with 16-byte loads only where the
+    rows allow them: odd vocabularies and padded strides fall back to scalar loads inside the run);
+    more than 131072 tokens take the scalar passes."""
+    rng = W.rng_for(240 + pad + vocab % 97)
+    parents = [W.random_tree(rng, 14, 4), W.chain_tree(5)]
+    case = _sample_case(rng, parents, vocab, dtype, stride_pad=pad)
+    for rep in range(2):
+        _check_sample(rng, *case, temperature=1.0, max_depth=5, vocab=vocab)
