@@ -204,6 +204,11 @@ size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
  * the scan that finds the per-chunk top-16 also accumulates the chunk statistics of psi(p), and both
  * finishing kernels follow it.  Arguments as sb_tree_expand plus features fp32 [n_rows][15] as
  * sb_rank_features; results identical to the two separate calls.
+ *   child_row int32 [node_budget] or NULL: for every row of this call that emits nodes under an existing
+ *   node, child_row[that node] = row_base + row -- the row of the drafter's scores that proposed the node's
+ *   children, as sb_verifier_signal and sb_verify_sample want it (row_base = rows of the earlier blocks when
+ *   the blocks' scores lie one after the other in one matrix).  Entries of nodes without children are left
+ *   as they are (initialise the array to -1); if several rows attach under one node, one of them is recorded.
  *   workspace : sb_rank_features_workspace_bytes(n_rows, vocab) bytes, 256-byte aligned.
  */
 sb_status sb_tree_expand_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
@@ -211,7 +216,8 @@ sb_status sb_tree_expand_features(const float* scores, int64_t row_stride, int32
                                   const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
                                   int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
                                   int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features,
-                                  void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+                                  int32_t* child_row, int32_t row_base, void* workspace, size_t workspace_bytes,
+                                  int32_t* status, void* stream);
 
 /*
  * sb_shift_project -- the layer-wise shift between consecutive decoder layers of the drafter

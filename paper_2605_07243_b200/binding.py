@@ -413,12 +413,15 @@ def sb_tree_expand_workspace_bytes(n_rows: int, vocab: int) -> int:
 
 
 def sb_tree_expand(scores, block_k, bucket, bmap, start_parent, node_budget, tree, *, vocab=None,
-                   workspace=None, topk_tok=None, topk_val=None, status=None, features=None):
+                   workspace=None, topk_tok=None, topk_val=None, status=None, features=None, child_row=None,
+                   row_base=0):
     """scores fp32 [R, stride]; bucket uint8 [R]; bmap: 4 host ints; tree: dict of int32 device
     tensors n_nodes [1], tok, parent, depth, node_row, node_rank (capacity node_budget), updated
     in place.  -> (topk_tok [R,16], topk_val [R,16], status [1]).
     features fp32 [R, 15]: also filled (sb_tree_expand_features: one pass over the scores for both);
-    the workspace must then hold sb_rank_features_workspace_bytes."""
+    the workspace must then hold sb_rank_features_workspace_bytes.  With features, child_row int32
+    [node_budget] (initialised to -1 by the caller) receives row_base + row for the nodes whose children a row
+    of this call proposes."""
     n_rows, stride = scores.shape
     vocab = stride if vocab is None else vocab
     dev = scores.device
@@ -441,5 +444,6 @@ def sb_tree_expand(scores, block_k, bucket, bmap, start_parent, node_budget, tre
     if features is None:
         _check(lib.sb_tree_expand(*head, *tail), "sb_tree_expand")
     else:
-        _check(lib.sb_tree_expand_features(*head, _ptr(features, torch.float32), *tail), "sb_tree_expand_features")
+        _check(lib.sb_tree_expand_features(*head, _ptr(features, torch.float32), _ptr(child_row, torch.int32),
+                                           C.c_int32(row_base), *tail), "sb_tree_expand_features")
     return topk_tok, topk_val, status

@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
     const uint8_t* __restrict__ bucket, int4 bmap, const int* __restrict__ start_parent, int node_budget,
     int vocab, int* __restrict__ n_nodes, int* __restrict__ tok, int* __restrict__ parent, int* __restrict__ depth,
     int* __restrict__ node_row, int* __restrict__ node_rank, int* __restrict__ topk_tok,
-    float* __restrict__ topk_val, int* __restrict__ status) {
+    float* __restrict__ topk_val, int* __restrict__ child_row, int row_base, int* __restrict__ status) {
   __shared__ int s_bad;
   __shared__ int s_warp_sum[FINISH_THREADS / 32];
   __shared__ int s_first[FINISH_THREADS + 1];  // first node id of each row of the current slab
@@ -564,6 +564,7 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
         node_row[n] = r;
         node_rank[n] = j;
       }
+      if (child_row && par >= 0 && first < node_budget) child_row[par] = row_base + r;  // this row proposed par's children
     }
     __syncthreads();
     if (tid == 0) s_carry = carry + s_warp_sum[FINISH_THREADS / 32 - 1];
@@ -595,7 +596,8 @@ __global__ void __launch_bounds__(ROWS_THREADS) expand_rows_kernel(
     const uint8_t* __restrict__ bucket, int4 bmap, const int* __restrict__ start_parent, int node_budget,
     int vocab, const int* __restrict__ n0_snapshot, int* __restrict__ n_nodes, int* __restrict__ tok,
     int* __restrict__ parent, int* __restrict__ depth, int* __restrict__ node_row, int* __restrict__ node_rank,
-    int* __restrict__ topk_tok, float* __restrict__ topk_val, int* __restrict__ status) {
+    int* __restrict__ topk_tok, float* __restrict__ topk_val, int* __restrict__ child_row, int row_base,
+    int* __restrict__ status) {
   __shared__ __align__(16) unsigned long long s_key[MERGE_MAX];
   __shared__ float s_val[MERGE_MAX];
   __shared__ int s_rank[MERGE_MAX];
@@ -715,6 +717,8 @@ __global__ void __launch_bounds__(ROWS_THREADS) expand_rows_kernel(
       node_rank[n] = rank;
     }
   }
+  // this row proposed the children of `par`: recorded for the calls that need the draft distribution of a node
+  if (tid == 0 && child_row && !any_bad && width > 0 && first < node_budget && par >= 0) child_row[par] = row_base + rr;
   if (rr == 0 && tid == 0) {
     if (any_bad) {
       *status = SB_ERR_INVALID_ARG;
@@ -848,8 +852,9 @@ static sb_status expand_impl(const float* scores, int64_t row_stride, int32_t n_
                              int32_t block_k, const uint8_t* bucket, const int32_t* bmap,
                              const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
                              int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
-                             int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features, void* workspace,
-                             size_t workspace_bytes, int32_t* status, void* stream) {
+                             int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features,
+                             int32_t* child_row, int32_t row_base, void* workspace, size_t workspace_bytes,
+                             int32_t* status, void* stream) {
   using namespace sb;
   if (!scores || !bucket || !bmap || !start_parent || !n_nodes || !tok || !parent || !depth || !node_row ||
       !node_rank || !topk_tok || !topk_val || !status || n_rows < 1 || vocab < 1 || row_stride < vocab ||
@@ -893,11 +898,12 @@ static sb_status expand_impl(const float* scores, int64_t row_stride, int32_t n_
     st = launch_dependent(expand_rows_kernel, dim3(n_rows), dim3(ROWS_THREADS), cs, n_rows, nc, part_val, part_idx,
                           block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
                           vocab, n0_snapshot, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val,
-                          status);
+                          child_row, (int)row_base, status);
   else
     st = launch_dependent(expand_finish_kernel, dim3(1), dim3(FINISH_THREADS), cs, n_rows, nc, part_val, part_idx,
                           block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent, node_budget,
-                          vocab, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val, status);
+                          vocab, n_nodes, tok, parent, depth, node_row, node_rank, topk_tok, topk_val, child_row,
+                          (int)row_base, status);
   if (st != SB_OK || !features) return st;
   // the summaries read the same chunk lists and the chunk statistics; as a dependent of the finishing kernel
   // (which waited for the scan) their wait covers the scan too
@@ -912,8 +918,8 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
                                     int32_t* node_rank, int32_t* topk_tok, float* topk_val, void* workspace,
                                     size_t workspace_bytes, int32_t* status, void* stream) {
   return expand_impl(scores, row_stride, n_rows, vocab, block_k, bucket, bmap, start_parent, node_budget, n_nodes, tok,
-                     parent, depth, node_row, node_rank, topk_tok, topk_val, nullptr, workspace, workspace_bytes, status,
-                     stream);
+                     parent, depth, node_row, node_rank, topk_tok, topk_val, nullptr, nullptr, 0, workspace,
+                     workspace_bytes, status, stream);
 }
 
 extern "C" sb_status sb_tree_expand_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
@@ -921,11 +927,12 @@ extern "C" sb_status sb_tree_expand_features(const float* scores, int64_t row_st
                                              const int32_t* start_parent, int32_t node_budget, int32_t* n_nodes,
                                              int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
                                              int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features,
-                                             void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
-  if (!features) return SB_ERR_INVALID_ARG;
+                                             int32_t* child_row, int32_t row_base, void* workspace,
+                                             size_t workspace_bytes, int32_t* status, void* stream) {
+  if (!features || row_base < 0) return SB_ERR_INVALID_ARG;
   return expand_impl(scores, row_stride, n_rows, vocab, block_k, bucket, bmap, start_parent, node_budget, n_nodes, tok,
-                     parent, depth, node_row, node_rank, topk_tok, topk_val, features, workspace, workspace_bytes, status,
-                     stream);
+                     parent, depth, node_row, node_rank, topk_tok, topk_val, features, child_row, row_base, workspace,
+                     workspace_bytes, status, stream);
 }
 
 extern "C" size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab) {

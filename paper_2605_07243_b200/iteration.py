@@ -14,7 +14,8 @@ Per drafter block m (Algorithm 1, the loop over m):
                   sb_shift_project)
     psi(p)        the rank head's distribution summary of every row   } one pass over  (sb_tree_expand_features)
     attach        top-b tokens of every row under the block's starts  } the scores
-then  verify:     ancestor masks, tree attention of every target layer, greedy acceptance, compaction.
+then  verify:     ancestor masks, tree attention of every target layer, greedy acceptance, the verifier-derived
+                  signal of the iteration, compaction.
 
 The pieces that need trained weights are not in the library (the decoder layers' own projections
 and MLPs, the lm_head, the rank head, the choice of next-block starts): their outputs are inputs
@@ -98,11 +99,19 @@ class SpecBlockIteration:
             d = w.w_fuse.shape[0]
             self.q_term = torch.empty((block_k, d), dtype=torch.float32, device=device)
             self.q_term_valid = False
+        # the blocks' scores lie one after the other in ONE matrix: a node's draft distribution is then a row of it
+        self.scores_all = torch.from_numpy(np.ascontiguousarray(np.concatenate([b.scores for b in blocks]), np.float32)).to(device)
+        self.child_row = torch.empty(node_budget, **i32)      # per node: the row that proposed its children (-1: none)
+        self._child_row0 = torch.full((node_budget,), -1, **i32)
+        self.signal = torch.zeros(1, dtype=torch.float32, device=device)   # verifier-derived signal, summed over iterations
+        self.r_prob = torch.empty(1, dtype=torch.float32, device=device)
+        self.signal_status = torch.empty(1, **i32)
         self.blocks = []
+        row_base = 0
         for m, b in enumerate(blocks):
             R, V = b.scores.shape
             S = R // block_k
-            e = dict(scores=torch.from_numpy(np.ascontiguousarray(b.scores, np.float32)).to(device),
+            e = dict(scores=self.scores_all[row_base:row_base + R], row_base=row_base,
                      bucket=torch.from_numpy(np.ascontiguousarray(b.bucket, np.uint8)).to(device),
                      start_parent=dev.i32_tensor(b.start_parent, device), R=R, S=S,
                      topk_tok=torch.empty((R, sb.SB_KMAX), **i32),
@@ -144,6 +153,7 @@ class SpecBlockIteration:
                                             device=device)
                 e["shift_status"] = torch.zeros(1, **i32)
             self.blocks.append(e)
+            row_base += R
         # ---- the target's verify forward ------------------------------------------------------------------
         c0 = target_layers[0]
         assert c0.batch == 1 and int(c0.node_offsets[-1]) == node_budget and c0.q_node_begin is None
@@ -185,6 +195,7 @@ class SpecBlockIteration:
         for k, t0 in self._tree0.items():
             self.tree[k].copy_(t0)
         self.node_offsets.copy_(self._offsets0)
+        self.child_row.copy_(self._child_row0)
 
     def run_block(self, m: int):
         e, w = self.blocks[m], self.weights
@@ -208,7 +219,7 @@ class SpecBlockIteration:
         # psi(p) and the expansion read the same scores: one pass over them serves both
         sb.sb_tree_expand(e["scores"], self.block_k, e["bucket"], self.bmap, e["start_parent"], self.budget, self.tree,
                           workspace=e["features_ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"], status=e["status"],
-                          features=e["features"])
+                          features=e["features"], child_row=self.child_row, row_base=e["row_base"])
 
     def run_verify(self):
         sb.sb_tree_ancestors(self.node_offsets, self.tree["parent"], self.budget, self.anc, self.depth, self.anc_status)
@@ -218,6 +229,12 @@ class SpecBlockIteration:
                                  k_cache=self.k_all[l], v_cache=self.v_all[l], index_arrays_settled=l > 0)
         sb.sb_verify_accept(self.logits, self.node_offsets, self.tree["parent"], self.tree["tok"], self.max_depth,
                             workspace=self.accept_ws, out=self.accept)
+        # the verifier-derived signal of this iteration (Algorithm 2, line 2): the drafter's probability of the
+        # bonus token in the row that proposed the children of the last accepted node -- found through child_row,
+        # which the expansions filled in on the device
+        sb.sb_verifier_signal(self.scores_all, self.node_offsets, self.child_row, self.accept["path_nodes"],
+                              self.accept["accept_len"], self.accept["bonus"], self.max_depth, self.signal,
+                              r_prob=self.r_prob, status=self.signal_status)
         sb.sb_kv_compact(self.tb, self.n_layers, self.layer_stride, self.accept["path_nodes"],
                          self.accept["accept_len"], self.max_depth, self.new_len, self.compact_status)
 

@@ -121,6 +121,20 @@ def _check_against_oracle(it, blocks, tree2, n, logits, target, weights, planted
     for key in ("accept_len", "path_nodes", "out_tokens", "bonus", "status"):
         np.testing.assert_array_equal(it.accept[key].cpu().numpy(), ref[key], err_msg=key)
     np.testing.assert_array_equal(it.accept["amax"].cpu().numpy()[:n], ref["amax"])
+    # the row that proposed each node's children, recorded by the expansions, and the verifier-derived signal
+    child_row = np.full(n, -1, np.int32)
+    row_base = np.cumsum([0] + [b.scores.shape[0] for b in blocks])
+    first_new = 1
+    for m, b in enumerate(blocks):                      # nodes are appended block by block, in row order
+        res_m, _ = _oracle_tree(blocks[:m + 1])
+        for c in range(first_new, res_m["n_nodes"]):
+            child_row[tree2["parent"][c]] = row_base[m] + tree2["node_row"][c]
+        first_new = res_m["n_nodes"]
+    np.testing.assert_array_equal(it.child_row.cpu().numpy()[:n], child_row)
+    scores_all = np.concatenate([b.scores for b in blocks])
+    sig = oracle.verifier_signal(scores_all, offs, child_row, ref["path_nodes"], ref["accept_len"], ref["bonus"], 2 * K)
+    assert int(it.signal_status.cpu()[0]) == int(sig["status"][0]) == 0
+    assert abs(float(it.r_prob.cpu()[0]) - sig["r_prob"][0]) <= 2e-5 * max(sig["r_prob"][0], 1e-3)
     c0 = target[0]
     for name, got_all in (("k", it.k_all), ("v", it.v_all)):
         cache = np.stack([getattr(c, name) for c in target]).reshape(-1)

@@ -727,7 +727,10 @@ def test_expand_with_features_in_one_pass():
     """sb_tree_expand_features = sb_tree_expand + sb_rank_features from one scan: same tree, same summaries."""
     for case in (W.config3_drafter()[1],
                  W.make_expand_case(W.rng_for(230), n_starts=5, block_k=3, vocab=777, bmap=[2, 3, 4, 0], node_budget=40,
-                                    existing_parent=W.random_tree(W.rng_for(231), 6, 3), tie_rows=2)):
+                                    existing_parent=W.random_tree(W.rng_for(231), 6, 3), tie_rows=2),
+                 W.make_expand_case(W.rng_for(232), n_starts=300, block_k=4, vocab=90, bmap=[1, 2, 1, 0], node_budget=4000,
+                                    existing_parent=np.concatenate([[-1], np.zeros(299, np.int32)]),
+                                    start_parent=np.arange(300, dtype=np.int32))):   # > 1024 rows: one finishing CTA
         R, V = case.scores.shape
         scores = torch.from_numpy(case.scores).cuda()
 
@@ -747,13 +750,26 @@ def test_expand_with_features_in_one_pass():
         tok_a, val_a, st_a = sb.sb_tree_expand(*args, t_sep)
         feat_sep = sb.sb_rank_features(scores)
         feat_fused = torch.full((R, 15), float("nan"), dtype=torch.float32, device="cuda")
-        tok_b, val_b, st_b = sb.sb_tree_expand(*args, t_fused, features=feat_fused)
+        child_row = torch.full((case.node_budget,), -1, dtype=torch.int32, device="cuda")
+        tok_b, val_b, st_b = sb.sb_tree_expand(*args, t_fused, features=feat_fused, child_row=child_row, row_base=1000)
         torch.cuda.synchronize()
         assert int(st_a.cpu()[0]) == 0 and int(st_b.cpu()[0]) == 0
         assert torch.equal(tok_a, tok_b) and torch.equal(val_a, val_b)
         for k in t_sep:
             assert torch.equal(t_sep[k], t_fused[k]), k
         assert torch.equal(feat_sep.view(torch.int32), feat_fused.view(torch.int32))
+        # the row that proposed each node's children: derived from the oracle's tree
+        ref_t = oracle.tree_expand(case.scores, case.block_k, case.bucket, case.bmap, case.start_parent, case.node_budget,
+                                   tree=case.tree)
+        n0 = 0 if case.tree is None else len(case.tree["tok"])
+        want_rows = np.full(case.node_budget, -1, np.int32)
+        for c in range(n0, ref_t["n_nodes"]):
+            if ref_t["parent"][c] >= 0:
+                want_rows[ref_t["parent"][c]] = 1000 + ref_t["node_row"][c]
+        unique_starts = len(set(int(x) for x in case.start_parent if x >= 0)) == sum(1 for x in case.start_parent if x >= 0)
+        assert unique_starts or R == 15                 # only the small random case may let two starts share a node
+        if unique_starts:
+            np.testing.assert_array_equal(child_row.cpu().numpy(), want_rows)
         ref = oracle.rank_features(case.scores)
         got = feat_fused.cpu().numpy().astype(np.float64)
         fin = np.isfinite(ref)
