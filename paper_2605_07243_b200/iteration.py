@@ -71,10 +71,12 @@ def _bf16(x, device):
 class SpecBlockIteration:
     def __init__(self, *, block_k: int, bmap, node_budget: int, root_tok: int, blocks: List[DraftBlock],
                  target_layers: List, logits: np.ndarray, max_depth: int, weights: Optional[DrafterWeights] = None,
-                 device="cuda", num_splits=0):
+                 device="cuda", num_splits=0, temperature: float = 0.0, u_accept=None, u_bonus=None):
         """target_layers: one workloads.AttnCase per target layer over ONE sequence whose tree has
         `node_budget` nodes (their K/V rows and Q rows are used; the tree itself is built here);
-        logits: [node_budget, V] fp32 or bf16 bits (the target's scores per tree node)."""
+        logits: [node_budget, V] fp32 or bf16 bits (the target's scores per tree node).
+        temperature > 0: the tree is verified by rejection sampling (sb_verify_sample) with the given uniforms
+        (u_accept fp32 [node_budget], u_bonus fp32 [1]) instead of greedy acceptance."""
         self.device, self.block_k, self.budget, self.max_depth = device, block_k, node_budget, max_depth
         self.bmap = [int(x) for x in bmap]
         self.num_splits = num_splits
@@ -187,6 +189,12 @@ class SpecBlockIteration:
                                      dtype=torch.uint8, device=device)
         self.new_len = torch.empty(1, **i32)
         self.compact_status = torch.empty(1, **i32)
+        self.temperature = float(temperature)
+        if self.temperature > 0.0:
+            self.u_accept = torch.as_tensor(np.asarray(u_accept, np.float32)).to(device)
+            self.u_bonus = torch.as_tensor(np.asarray(u_bonus, np.float32)).to(device)
+            self.sample_ws = torch.empty(max(256, sb.sb_verify_sample_workspace_bytes(
+                1, self.logits.shape[1], node_budget, self.scores_all.shape[0])), dtype=torch.uint8, device=device)
 
     # ---- the chain ---------------------------------------------------------------------------------------
 
@@ -227,8 +235,13 @@ class SpecBlockIteration:
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,
                                  num_splits=self.num_splits, workspace=self.attn_ws, status=self.attn_status,
                                  k_cache=self.k_all[l], v_cache=self.v_all[l], index_arrays_settled=l > 0)
-        sb.sb_verify_accept(self.logits, self.node_offsets, self.tree["parent"], self.tree["tok"], self.max_depth,
-                            workspace=self.accept_ws, out=self.accept)
+        if self.temperature > 0.0:   # rejection sampling against the target: the drafter rows come through child_row
+            sb.sb_verify_sample(self.logits, self.scores_all, self.node_offsets, self.tree["parent"], self.tree["tok"],
+                                self.child_row, self.temperature, self.u_accept, self.u_bonus, self.max_depth,
+                                workspace=self.sample_ws, out=self.accept)
+        else:
+            sb.sb_verify_accept(self.logits, self.node_offsets, self.tree["parent"], self.tree["tok"], self.max_depth,
+                                workspace=self.accept_ws, out=self.accept)
         # the verifier-derived signal of this iteration (Algorithm 2, line 2): the drafter's probability of the
         # bonus token in the row that proposed the children of the last accepted node -- found through child_row,
         # which the expansions filled in on the device

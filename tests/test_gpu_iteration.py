@@ -224,3 +224,44 @@ def test_iteration_without_the_drafter_side_and_budget_cut():
         _check_against_oracle(*built)
     finally:
         BUDGET = old
+
+
+def test_iteration_with_stochastic_verification():
+    """Temperature 1: the tree grown on the device is verified by rejection sampling, the drafter's rows found
+    through the child_row array the expansions filled in; walk and signal against the oracle on the same tree."""
+    from test_gpu_tree_ops import _robust_uniforms
+    it, blocks, tree2, n, logits, target, weights, planted = _build(9004, n_target_layers=1, with_drafter=False)
+    rng = W.rng_for(9005)
+    offs = np.array([0, n], np.int32)
+    child_row = np.full(n, -1, np.int32)
+    row_base = np.cumsum([0] + [b.scores.shape[0] for b in blocks])
+    first_new = 1
+    for m in range(len(blocks)):
+        res_m, _ = _oracle_tree(blocks[:m + 1])
+        for c in range(first_new, res_m["n_nodes"]):
+            child_row[tree2["parent"][c]] = row_base[m] + tree2["node_row"][c]
+        first_new = res_m["n_nodes"]
+    scores_all = np.concatenate([b.scores for b in blocks])
+    args = (logits[:n], scores_all, offs, tree2["parent"], tree2["tok"], child_row)
+    u_a, u_b, ref = _robust_uniforms(rng, args, 1.0, 2 * K, n, 1)
+    u_full = np.zeros(BUDGET, np.float32)
+    u_full[:n] = u_a
+    it2 = SpecBlockIteration(block_k=K, bmap=BMAP, node_budget=BUDGET, root_tok=ROOT_TOK, blocks=blocks,
+                             target_layers=target, logits=logits, max_depth=2 * K, temperature=1.0, u_accept=u_full,
+                             u_bonus=u_b)
+    it2.run()
+    torch.cuda.synchronize()
+    for key in ("status", "accept_len", "path_nodes"):
+        np.testing.assert_array_equal(it2.accept[key].cpu().numpy(), ref[key], err_msg=key)
+    a = int(ref["accept_len"][0])
+    np.testing.assert_array_equal(it2.accept["out_tokens"].cpu().numpy()[0, :a], ref["out_tokens"][0, :a])
+    lo = oracle.verify_sample(*args, 1.0, u_a, (u_b * np.float32(1 - 1e-3)).astype(np.float32), 2 * K)["bonus"][0]
+    hi = oracle.verify_sample(*args, 1.0, u_a, (u_b * np.float32(1 + 1e-3)).astype(np.float32), 2 * K)["bonus"][0]
+    got_bonus = int(it2.accept["bonus"].cpu()[0])
+    assert lo <= got_bonus <= hi
+    # the signal follows the sampled path and bonus (compared when the device drew the oracle's own bonus token,
+    # which it does unless u_bonus falls within 1e-3 of a cell boundary)
+    sig = oracle.verifier_signal(scores_all, offs, child_row, ref["path_nodes"], ref["accept_len"], ref["bonus"], 2 * K)
+    assert int(it2.signal_status.cpu()[0]) == int(sig["status"][0])
+    if got_bonus == int(ref["bonus"][0]) and sig["r_prob"][0] >= 0:
+        assert abs(float(it2.r_prob.cpu()[0]) - sig["r_prob"][0]) <= 2e-5 * max(sig["r_prob"][0], 1e-3)
