@@ -480,14 +480,18 @@ static int max_active_clusters(int D, int cluster) {
 // clusters of 8 full-SM CTAs keep only 120 of the 148 SMs busy, clusters of 2 all of them, and the
 // extra fp32 partials (one per cluster) cost less than the idle SMs (measured on the long-context
 // configuration: 1072 us against 1227 us).
-static SplitPlan plan_for(int s, bool oversubscribed) {
+// The tcgen05 kernel also runs clusters of 9 and 10 (beyond the portable 8: allowed per kernel), which the
+// single-wave chooser below takes when they fit -- 15 clusters of 9 or 11 of 10 full-SM CTAs on a B200.
+constexpr int kMaxClusterTc = 10;
+static SplitPlan plan_for(int s, bool oversubscribed, bool wide = false) {
   SplitPlan sp;
   sp.two_tiles = false;
   sp.cluster = 1;
-  int cmax = oversubscribed ? 2 : kMaxCluster;
+  const int climit = wide ? kMaxClusterTc : kMaxCluster;
+  int cmax = oversubscribed ? 2 : climit;
   if (const char* e = getenv("SB_ATTN_MAX_CLUSTER")) {  // experiment knob
     const int v = atoi(e);
-    if (v >= 1 && v <= kMaxCluster) cmax = v;
+    if (v >= 1 && v <= climit) cmax = v;
   }
   for (int c = cmax; c >= 1; --c)
     if (s % c == 0) { sp.cluster = c; break; }
@@ -589,7 +593,7 @@ static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_spl
   SplitPlan best = plan_for(1, false);
   double best_cost = 1.2 * max_blocks;
   for (int s = 2; s <= s_max; ++s) {
-    const SplitPlan sp = plan_for(s, false);
+    const SplitPlan sp = plan_for(s, false, impl == IMPL_TC);
     if (sp.outer > 1 && sp.cluster < 4) continue;  // partial traffic for little gain
     const int fit = impl == IMPL_TC ? attn_tc_max_active_clusters(tb->head_dim, sp.cluster)
                                     : max_active_clusters(tb->head_dim, sp.cluster);

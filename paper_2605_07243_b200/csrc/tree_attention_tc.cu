@@ -45,7 +45,8 @@ constexpr int TC_VLOAD_WARP = 10;    // lane 0 issues the V loads; the warp zero
 constexpr int TC_THREADS = 384;      // 12 warps (warp 11 only takes part in the barriers)
 constexpr int TC_TMEM_COLS = 512;
 constexpr int TC_SMALL_BYTES = 8192; // ancestor masks, parents, barriers, softmax exchange
-constexpr int TC_MERGE_SLOTS = TC_BM + 8;  // receive slots: S * ceil(128 / S) <= 135 for S <= 8
+constexpr int TC_MAX_CLUSTER = 10;          // chunks merged in one cluster (9 and 10 are beyond the portable size)
+constexpr int TC_MERGE_SLOTS = TC_BM + 8;  // receive slots: S * ceil(128 / S) <= 135 for S <= 10
 
 enum TcBar { K_FULL0, K_FULL1, K_EMPTY0, K_EMPTY1, V_FULL0, V_FULL1, V_EMPTY0, V_EMPTY1, S_FULL0, S_FULL1,
              S_EMPTY0, S_EMPTY1, P_FULL, PV_FULL, V_TMA0, V_TMA1, Q_FULL, MERGE_BAR, ACK_BAR, TC_NUM_BARS };
@@ -63,8 +64,8 @@ constexpr size_t attn_tc_smem_bytes() {
 // index z = sequence.  The general instantiation decides all of that at run time (paged caches, a
 // gathered Q tile, partials for attn_merge_kernel, sequences taken longest first).  Code that is
 // never executed still costs a kernel this short: an untaken branch to the sequence ranking alone
-// was 0.1 us per launch, and knowing the cluster size (CS = 1..8, the chunks of a tile) at compile
-// time another 0.4 us.  CS = 0 is the general instantiation.
+// was 0.1 us per launch, and knowing the cluster size (CS = 1..10, the chunks of a tile) at compile
+// time another 0.4 us.  CS = 0 is the general instantiation; 9 and 10 are beyond the portable cluster size.
 template <int D, int CS>
 __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams p,
                                                                 const __grid_constant__ CUtensorMap kmap,
@@ -549,13 +550,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       const int Rr = row0 + my_first + t;
       if (Rr >= rows_total) continue;
       const bool has_cols = col8 < D / 8;
-      float w[8];
-      uint4 raw[8];
+      constexpr int SRC = FAST ? CS : TC_MAX_CLUSTER;  // sources: known at compile time in the common case
+      float w[SRC];
+      uint4 raw[SRC];
       float M = -INFINITY, Lsum = 0.f;
       {
-        float mc[8], lc[8];
+        float mc[SRC], lc[SRC];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < SRC; ++c) {
           const uint8_t* rowp = src + ((size_t)(c < S ? c : 0) * rows_per + t) * ROWB;
           mc[c] = c < S ? *reinterpret_cast<const float*>(rowp + D * 2) : -INFINITY;
           lc[c] = c < S ? *reinterpret_cast<const float*>(rowp + D * 2 + 4) : 0.f;
@@ -563,7 +565,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
           M = fmaxf(M, mc[c]);
         }
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < SRC; ++c) {
           w[c] = mc[c] == -INFINITY ? 0.f : fast_exp2(mc[c] - M) * lc[c];  // 2^(m_c - M) * l_c
           Lsum += w[c];
         }
@@ -573,7 +575,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = 0.f;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int c = 0; c < SRC; ++c) {
         const uint32_t q4[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -643,8 +645,12 @@ static bool tc_prepare() {
   all = all && cudaFuncSetAttribute(attn_tc_kernel<D, cs_>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
                                     (int)attn_tc_smem_bytes<D>()) == cudaSuccess;
     SB_TC_PREPARE(0) SB_TC_PREPARE(1) SB_TC_PREPARE(2) SB_TC_PREPARE(3) SB_TC_PREPARE(4)
-    SB_TC_PREPARE(5) SB_TC_PREPARE(6) SB_TC_PREPARE(7) SB_TC_PREPARE(8)
+    SB_TC_PREPARE(5) SB_TC_PREPARE(6) SB_TC_PREPARE(7) SB_TC_PREPARE(8) SB_TC_PREPARE(9) SB_TC_PREPARE(10)
 #undef SB_TC_PREPARE
+    // clusters of 9 and 10 CTAs are beyond the portable size: allowed per kernel
+    all = all && cudaFuncSetAttribute(attn_tc_kernel<D, 0>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    all = all && cudaFuncSetAttribute(attn_tc_kernel<D, 9>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    all = all && cudaFuncSetAttribute(attn_tc_kernel<D, 10>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
     if (!all) {
       cudaGetLastError();
       return false;
@@ -655,10 +661,10 @@ static bool tc_prepare() {
 }
 
 int attn_tc_max_active_clusters(int D, int cluster) {
-  static int cache[2][9];
-  static bool have[2][9];
+  static int cache[2][TC_MAX_CLUSTER + 1];
+  static bool have[2][TC_MAX_CLUSTER + 1];
   const int di = D == 64 ? 0 : 1;
-  if (cluster < 1 || cluster > 8) return 0;
+  if (cluster < 1 || cluster > TC_MAX_CLUSTER) return 0;
   if (!have[di][cluster]) {
     int n = 0;
     cudaLaunchAttribute attr[2];
@@ -701,7 +707,7 @@ static sb_status launch_tc(const AttnParams& p, dim3 grid, int cluster, cudaStre
 #define SB_TC_LAUNCH(cs_) \
   case cs_: le = cudaLaunchKernelEx(&cfg, attn_tc_kernel<D, cs_>, p, kmap, vmap, qmap, box_rows, q_tma); break;
     SB_TC_LAUNCH(0) SB_TC_LAUNCH(1) SB_TC_LAUNCH(2) SB_TC_LAUNCH(3) SB_TC_LAUNCH(4)
-    SB_TC_LAUNCH(5) SB_TC_LAUNCH(6) SB_TC_LAUNCH(7) SB_TC_LAUNCH(8)
+    SB_TC_LAUNCH(5) SB_TC_LAUNCH(6) SB_TC_LAUNCH(7) SB_TC_LAUNCH(8) SB_TC_LAUNCH(9) SB_TC_LAUNCH(10)
 #undef SB_TC_LAUNCH
     default: break;
   }
