@@ -120,14 +120,20 @@ __global__ void __launch_bounds__(VS_STATS_THREADS) vs_stats_kernel(const T* __r
                                                                     bool p_vec, int total_nodes,
                                                                     const float* __restrict__ scores,
                                                                     long long score_stride, bool q_vec, int vocab,
-                                                                    int chunk, int n_chunks, float k,
+                                                                    int chunk_p, int n_chunks_p, int chunk_q,
+                                                                    int n_chunks_q, float k,
                                                                     float* __restrict__ stats_p,
                                                                     float* __restrict__ stats_q) {
   __shared__ float s_red[VS_STATS_THREADS / 32];
   pdl_release();  // the walk may set itself up
   const int row = blockIdx.y;
-  if (row < total_nodes) vs_chunk_stats<T>(logits, row_stride, row, vocab, chunk, n_chunks, p_vec, k, stats_p, s_red);
-  else vs_chunk_stats<float>(scores, score_stride, row - total_nodes, vocab, chunk, n_chunks, q_vec, k, stats_q, s_red);
+  // the grid is as wide as the matrix with more chunks per row; a row of the other one leaves its spare CTAs idle
+  if (row < total_nodes) {
+    if ((int)blockIdx.x < n_chunks_p)
+      vs_chunk_stats<T>(logits, row_stride, row, vocab, chunk_p, n_chunks_p, p_vec, k, stats_p, s_red);
+  } else if ((int)blockIdx.x < n_chunks_q) {
+    vs_chunk_stats<float>(scores, score_stride, row - total_nodes, vocab, chunk_q, n_chunks_q, q_vec, k, stats_q, s_red);
+  }
 }
 
 // (M, Z) of a row from its chunk statistics (at most 32 chunks): lane c fetches chunk c, the warp combines
@@ -248,8 +254,8 @@ __global__ void __launch_bounds__(VS_THREADS) verify_sample_kernel(
     const T* __restrict__ logits, long long row_stride, int vocab, const float* __restrict__ scores,
     long long score_stride, int n_rows, int total_nodes, const int* __restrict__ node_offsets,
     const int* __restrict__ parent, const int* __restrict__ tok, const int* __restrict__ child_row, float inv_t,
-    const float* __restrict__ u_accept, const float* __restrict__ u_bonus, int max_depth, int n_chunks,
-    const float* __restrict__ stats_p, const float* __restrict__ stats_q, int* __restrict__ accept_len,
+    const float* __restrict__ u_accept, const float* __restrict__ u_bonus, int max_depth, int n_chunks_p,
+    int n_chunks_q, const float* __restrict__ stats_p, const float* __restrict__ stats_q, int* __restrict__ accept_len,
     int* __restrict__ path_nodes, int* __restrict__ out_tokens, int* __restrict__ bonus, float* work,
     int* __restrict__ status) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -311,7 +317,7 @@ __global__ void __launch_bounds__(VS_THREADS) verify_sample_kernel(
   const T* prow = logits + (long long)o * row_stride;  // target row of the current node
   bool p_plain = true;      // p = softmax of prow (else: pw / zp)
   float Mp, zp;             // maximum of prow; normaliser of p in either form
-  vs_row_stats(stats_p + (long long)o * n_chunks * 2, n_chunks, vocab, k, Mp, zp);
+  vs_row_stats(stats_p + (long long)o * n_chunks_p * 2, n_chunks_p, vocab, k, Mp, zp);
   auto p_unnorm = [&](int v) { return p_plain ? vs_unnorm(vs_value<T>(prow, v), Mp, k) : pw[v]; };
   auto p_run = [&](float (&y)[VS_RUN]) {  // this lane's run of unnormalised p
     if (p_plain) {
@@ -333,7 +339,7 @@ __global__ void __launch_bounds__(VS_THREADS) verify_sample_kernel(
     if (row < 0 || row >= n_rows) { err = SB_ERR_BOUNDS; break; }
     const float* qrow = scores + (long long)row * score_stride;
     float Mq, zq;  // q = (unnormalised draft value, 0 for the removed tokens) / zq
-    vs_row_stats(stats_q + (long long)row * n_chunks * 2, n_chunks, vocab, k, Mq, zq);
+    vs_row_stats(stats_q + (long long)row * n_chunks_q * 2, n_chunks_q, vocab, k, Mq, zq);
     int n_removed = 0;
     int accepted = -1;
     for (; c < n; ++c) {
@@ -404,7 +410,7 @@ __global__ void __launch_bounds__(VS_THREADS) verify_sample_kernel(
     if (writer) { path[depth] = a; otok[depth - 1] = s_tok[a]; }
     prow = logits + (long long)(o + a) * row_stride;
     p_plain = true;
-    vs_row_stats(stats_p + (long long)(o + a) * n_chunks * 2, n_chunks, vocab, k, Mp, zp);
+    vs_row_stats(stats_p + (long long)(o + a) * n_chunks_p * 2, n_chunks_p, vocab, k, Mp, zp);
   }
   if (err) {  // uniform over the cluster
     __syncthreads();
@@ -522,11 +528,12 @@ __global__ void __launch_bounds__(VS_THREADS) verify_sample_kernel(
   }
 }
 
-// Chunks per row of the statistics kernels: enough for one sweep per CTA (256 threads x 8 loads of 16
-// bytes = 8192 floats; the same count is used for bf16 rows) and for a grid of a few hundred CTAs.
-static int vs_chunks(int rows, int vocab) {
-  int nc = ceil_div(vocab, 8192);
-  const int fill = ceil_div(2 * 148, rows > 0 ? rows : 1), max_nc = ceil_div(vocab, 2048);
+// Chunks per row of the statistics kernel for rows of `elem_bytes`-wide elements: one sweep per CTA (256 threads x
+// 8 loads of 16 bytes), and at least a few hundred CTAs in the grid when the matrix is small.
+static int vs_chunks(int rows_total, int vocab, int elem_bytes) {
+  const int sweep = VS_STATS_THREADS * 8 * (16 / elem_bytes);
+  int nc = ceil_div(vocab, sweep);
+  const int fill = ceil_div(2 * 148, rows_total > 0 ? rows_total : 1), max_nc = ceil_div(vocab, 2048);
   if (nc < fill) nc = fill < max_nc ? fill : max_nc;
   if (nc > VS_MAX_CHUNKS) nc = VS_MAX_CHUNKS;
   if (nc < 1) nc = 1;
@@ -539,9 +546,10 @@ static size_t vs_align(size_t x) { return (x + 255) & ~(size_t)255; }
 extern "C" size_t sb_verify_sample_workspace_bytes(int32_t batch, int32_t vocab, int32_t total_nodes, int32_t n_rows) {
   if (batch < 1 || vocab < 1 || total_nodes < 1 || n_rows < 1) return 0;
   using namespace sb;
-  const size_t nc = (size_t)vs_chunks(total_nodes + n_rows, vocab);
-  return vs_align((size_t)batch * vocab * sizeof(float)) + vs_align((size_t)total_nodes * nc * 2 * sizeof(float)) +
-         vs_align((size_t)n_rows * nc * 2 * sizeof(float));
+  // the statistics of the target rows are sized for 2-byte logits (the larger count covers fp32 ones too)
+  return vs_align((size_t)batch * vocab * sizeof(float)) +
+         vs_align((size_t)total_nodes * VS_MAX_CHUNKS * 2 * sizeof(float)) +
+         vs_align((size_t)n_rows * VS_MAX_CHUNKS * 2 * sizeof(float));
 }
 
 extern "C" sb_status sb_verify_sample(const void* logits, sb_dtype dtype, int64_t row_stride, int32_t vocab,
@@ -565,23 +573,25 @@ extern "C" sb_status sb_verify_sample(const void* logits, sb_dtype dtype, int64_
   const float inv_t = 1.0f / temperature, k = inv_t * kVsLog2e;
   char* ws = static_cast<char*>(workspace);
   float* work = reinterpret_cast<float*>(ws);
-  const int nc = vs_chunks(total_nodes + n_rows, vocab);
-  float* stats_p = reinterpret_cast<float*>(ws + vs_align((size_t)batch * vocab * sizeof(float)));
-  float* stats_q = reinterpret_cast<float*>(reinterpret_cast<char*>(stats_p) + vs_align((size_t)total_nodes * nc * 2 * sizeof(float)));
-  // statistics of every target row and every draft row, one grid
   const int esz = dtype == SB_BF16 ? 2 : 4;
-  const int chunk = ceil_div(ceil_div(vocab, nc), 8) * 8;
+  const int ncp = vs_chunks(total_nodes + n_rows, vocab, esz), ncq = vs_chunks(total_nodes + n_rows, vocab, 4);
+  float* stats_p = reinterpret_cast<float*>(ws + vs_align((size_t)batch * vocab * sizeof(float)));
+  float* stats_q = reinterpret_cast<float*>(reinterpret_cast<char*>(stats_p) +
+                                            vs_align((size_t)total_nodes * VS_MAX_CHUNKS * 2 * sizeof(float)));
+  // statistics of every target row and every draft row, one grid
+  const int chunk_p = ceil_div(ceil_div(vocab, ncp), 8) * 8, chunk_q = ceil_div(ceil_div(vocab, ncq), 8) * 8;
   const bool p_vec = (reinterpret_cast<uintptr_t>(logits) & 15) == 0 && (row_stride * esz) % 16 == 0;
   const bool q_vec = (reinterpret_cast<uintptr_t>(scores) & 15) == 0 && score_stride % 4 == 0;
-  const dim3 sgrid(nc, total_nodes + n_rows);
+  const dim3 sgrid(ncp > ncq ? ncp : ncq, total_nodes + n_rows);
   if (dtype == SB_BF16)
     vs_stats_kernel<uint16_t><<<sgrid, VS_STATS_THREADS, 0, cs>>>(static_cast<const uint16_t*>(logits), (long long)row_stride,
                                                                 p_vec, (int)total_nodes, scores, (long long)score_stride,
-                                                                q_vec, (int)vocab, chunk, nc, k, stats_p, stats_q);
+                                                                q_vec, (int)vocab, chunk_p, ncp, chunk_q, ncq, k, stats_p,
+                                                                stats_q);
   else
     vs_stats_kernel<float><<<sgrid, VS_STATS_THREADS, 0, cs>>>(static_cast<const float*>(logits), (long long)row_stride, p_vec,
                                                              (int)total_nodes, scores, (long long)score_stride, q_vec,
-                                                             (int)vocab, chunk, nc, k, stats_p, stats_q);
+                                                             (int)vocab, chunk_p, ncp, chunk_q, ncq, k, stats_p, stats_q);
   sb_status st = launch_check();
   if (st != SB_OK) return st;
   cudaLaunchConfig_t cfg = {};
@@ -601,13 +611,13 @@ extern "C" sb_status sb_verify_sample(const void* logits, sb_dtype dtype, int64_
   if (dtype == SB_BF16)
     e = cudaLaunchKernelEx(&cfg, verify_sample_kernel<uint16_t>, static_cast<const uint16_t*>(logits), (long long)row_stride,
                            (int)vocab, scores, (long long)score_stride, (int)n_rows, (int)total_nodes, node_offsets, parent,
-                           tok, child_row, inv_t, u_accept, u_bonus, (int)max_depth, nc,
+                           tok, child_row, inv_t, u_accept, u_bonus, (int)max_depth, ncp, ncq,
                            static_cast<const float*>(stats_p), static_cast<const float*>(stats_q), accept_len, path_nodes,
                            out_tokens, bonus, work, status);
   else
     e = cudaLaunchKernelEx(&cfg, verify_sample_kernel<float>, static_cast<const float*>(logits), (long long)row_stride,
                            (int)vocab, scores, (long long)score_stride, (int)n_rows, (int)total_nodes, node_offsets, parent,
-                           tok, child_row, inv_t, u_accept, u_bonus, (int)max_depth, nc,
+                           tok, child_row, inv_t, u_accept, u_bonus, (int)max_depth, ncp, ncq,
                            static_cast<const float*>(stats_p), static_cast<const float*>(stats_q), accept_len, path_nodes,
                            out_tokens, bonus, work, status);
   if (e != cudaSuccess) {
