@@ -34,6 +34,23 @@ def test_host_only_entry_points():
     assert binding.sb_verify_accept_workspace_bytes(60, 128256) > 0
     assert binding.sb_tree_expand_workspace_bytes(32, 128256) > 0
     assert lib.sb_tree_attention_workspace_bytes(None, 1, 0) == 0
+    # every other query: positive and 256-byte granular for valid shapes, 0 for shapes the call refuses
+    expand = binding.sb_tree_expand_workspace_bytes(32, 128256)
+    feats = binding.sb_rank_features_workspace_bytes(32, 128256)
+    assert feats > expand and expand % 256 == 0 and feats % 256 == 0          # the fused call uses the larger one
+    assert binding.sb_tree_expand_workspace_bytes(0, 128256) == 0
+    sample = binding.sb_verify_sample_workspace_bytes(2, 128256, 120, 36)
+    assert sample >= 2 * 128256 * 4 and sample % 256 == 0                      # a residual row per sequence + statistics
+    assert binding.sb_verify_sample_workspace_bytes(2, 128256, 0, 36) == 0
+    shift = binding.sb_shift_project_workspace_bytes(32, 4096, 4096, 4)
+    plain = binding.sb_shift_project_workspace_bytes(32, 4096, 4096, 0)
+    assert shift >= plain > 0 and shift % 256 == 0                             # fp32 partials of the K splits + a word
+    assert binding.sb_shift_project_workspace_bytes(32, 4000, 4096, 4) == 0    # d not a multiple of 64
+    assert binding.sb_shift_project_workspace_bytes(129, 4096, 4096, 4) == 0   # more than 128 rows
+    fuse3 = binding.sb_fuse_project_workspace_bytes(8, 4, 4096, 4096, False)
+    fuse2 = binding.sb_fuse_project_workspace_bytes(8, 4, 4096, 4096, True)
+    assert fuse3 > fuse2 > 0                                                   # the cached query term saves a third
+    assert binding.sb_fuse_project_workspace_bytes(8, 4, 4096, 100, False) == 0
 
 
 def test_binding_struct_matches_header_layout():
