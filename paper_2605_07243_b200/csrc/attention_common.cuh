@@ -22,12 +22,13 @@ struct AttnParams {
   float scale_log2;  // softmax scale * log2(e): scores are kept in the base-2 domain
   int num_splits;   // KV chunks per (sequence, KV head, row tile) = cluster size * outer
   int outer;        // clusters per (sequence, KV head, row tile); > 1 needs the merge kernel
-  float* part_o;    // [outer][total_q*Hq][D] normalised partial outputs
+  float* part_o;    // [outer][total_q*Hq][D] normalised partial outputs (fp32, or bf16 when part_bf16)
   float* part_lse;  // [outer][total_q*Hq]    base-2 log-sum-exp of each partial
   int* status;
   int G;            // query heads per KV head
   int row_tiles;    // 128-row query tiles per (sequence, KV head) in the grid
   int sort_seqs;    // 1: grid index z is the rank of a sequence by length, longest first
+  int part_bf16;    // 1: part_o holds bf16 (the writer's rows are already rounded to bf16 when it stores them)
 };
 
 constexpr float kLn2 = 0.6931471805599453f;

@@ -354,7 +354,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
 // One warp per (node, head) row.
 // ----------------------------------------------------------------------------------------------
 
-template <int D>
+template <int D, bool PB16>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
   constexpr int E = D / 32;
   const int b = blockIdx.y;
@@ -374,20 +374,49 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
   const long long rows_all = (long long)p.total_q * Hq;
   const long long grow = (long long)q_off * Hq + rr;
   float M = -INFINITY;
-  for (int s = 0; s < p.outer; ++s) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
+  for (int s = lane; s < p.outer; s += 32) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
   float acc[E];
 #pragma unroll
   for (int e = 0; e < E; ++e) acc[e] = 0.f;
   float denom = 0.f;
   if (M != -INFINITY) {
+    // no branch around the loads, so that several chunks' rows are in flight at once
+#pragma unroll 4
     for (int s = 0; s < p.outer; ++s) {
       const float ls = p.part_lse[s * rows_all + grow];
-      if (ls == -INFINITY) continue;  // that chunk saw no key for this row: its O is not written
-      const float w = exp2f(ls - M);
+      const bool live = ls != -INFINITY;  // a chunk that saw no key for this row did not write its O
+      const float w = live ? exp2f(ls - M) : 0.f;
       denom += w;
-      const float* po = p.part_o + (s * rows_all + grow) * D + lane * E;
+      float v[E];
+      if (PB16) {
+        const bf16* po = reinterpret_cast<const bf16*>(p.part_o) + (s * rows_all + grow) * D + lane * E;
+        uint32_t raw[E / 2];
+        if (E == 4) {
+          const uint2 t = live ? *reinterpret_cast<const uint2*>(po) : make_uint2(0u, 0u);
+          raw[0] = t.x;
+          raw[E / 2 - 1] = t.y;
+        } else {
+          raw[0] = live ? *reinterpret_cast<const uint32_t*>(po) : 0u;
+        }
 #pragma unroll
-      for (int e = 0; e < E; ++e) acc[e] += w * po[e];
+        for (int e = 0; e < E / 2; ++e) {
+          v[2 * e] = __uint_as_float(raw[e] << 16);
+          v[2 * e + 1] = __uint_as_float(raw[e] & 0xffff0000u);
+        }
+      } else {
+        const float* po = p.part_o + (s * rows_all + grow) * D + lane * E;
+        if (E == 4) {
+          const float4 t = live ? *reinterpret_cast<const float4*>(po) : make_float4(0.f, 0.f, 0.f, 0.f);
+          v[0] = t.x, v[1] = t.y, v[E - 2] = t.z, v[E - 1] = t.w;
+        } else {
+          const float2 t = live ? *reinterpret_cast<const float2*>(po) : make_float2(0.f, 0.f);
+          v[0] = t.x, v[1] = t.y;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[e] += w * v[e];
     }
   }
   const float inv = denom > 0.f ? 1.f / denom : 0.f;
@@ -684,6 +713,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   p.G = tb->n_q_heads / tb->n_kv_heads;
   p.part_o = nullptr;
   p.sort_seqs = 0;
+  p.part_bf16 = 0;
   p.part_lse = nullptr;
 
   const AttnImpl impl = attn_impl();
@@ -711,6 +741,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   }
   const int row_tiles = max_row_tiles(tb, total_q);
   p.row_tiles = row_tiles;
+  p.part_bf16 = plan.two_tiles ? 1 : 0;
   // ragged batches that run in waves start their longest sequences first
   p.sort_seqs = (impl == IMPL_TC && tb->batch > 1 && tb->batch <= 128 &&
                  (long long)tb->batch * tb->n_kv_heads * row_tiles > num_sms()) ? 1 : 0;
@@ -721,7 +752,12 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   else st = D == 64 ? launch_attn_mma<64>(p, grid, plan.cluster, cs) : launch_attn_mma<128>(p, grid, plan.cluster, cs);
   if (st != SB_OK || plan.outer == 1) return st;
   dim3 mgrid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);
-  if (D == 64) attn_merge_kernel<64><<<mgrid, 256, 0, cs>>>(p);
-  else attn_merge_kernel<128><<<mgrid, 256, 0, cs>>>(p);
+  if (p.part_bf16) {
+    if (D == 64) attn_merge_kernel<64, true><<<mgrid, 256, 0, cs>>>(p);
+    else attn_merge_kernel<128, true><<<mgrid, 256, 0, cs>>>(p);
+  } else {
+    if (D == 64) attn_merge_kernel<64, false><<<mgrid, 256, 0, cs>>>(p);
+    else attn_merge_kernel<128, false><<<mgrid, 256, 0, cs>>>(p);
+  }
   return launch_check();
 }

@@ -483,16 +483,9 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
         *reinterpret_cast<uint4*>(p.out + grow * D + col8 * 8) = raw;
         if (p.lse && col8 == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
       } else {
-        const uint32_t q4[4] = {raw.x, raw.y, raw.z, raw.w};
-        float f[8];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          f[2 * e] = __uint_as_float(q4[e] << 16);
-          f[2 * e + 1] = __uint_as_float(q4[e] & 0xffff0000u);
-        }
-        float* po = p.part_o + ((long long)split * rows_all + grow) * D + col8 * 8;
-        *reinterpret_cast<float4*>(po) = make_float4(f[0], f[1], f[2], f[3]);
-        *reinterpret_cast<float4*>(po + 4) = make_float4(f[4], f[5], f[6], f[7]);
+        // the staged row is bf16 already: partials keep that width (half the bytes of fp32, same values)
+        bf16* po = reinterpret_cast<bf16*>(p.part_o) + ((long long)split * rows_all + grow) * D + col8 * 8;
+        *reinterpret_cast<uint4*>(po) = raw;
         if (col8 == 0) p.part_lse[(long long)split * rows_all + grow] = lse2;
       }
     }
