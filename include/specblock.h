@@ -82,6 +82,12 @@ typedef enum sb_dtype { SB_BF16 = 0, SB_F32 = 1 } sb_dtype;
  * call of the same verify forward) may set this to 1: the sequence lengths are then fetched while
  * that kernel is still running (about half a microsecond per call).  Q, K, V, the parents and the
  * page table are always read after it has completed.  0 is always correct.
+ * prefix_rows_settled (only with index_arrays_settled = 1): the same vouch for the cache rows of
+ * the committed prefix -- the kernel enqueued immediately before does not write K or V at positions
+ * below prefix_len[b] (a projection that appends the tree's rows, or the previous layer's
+ * attention, qualifies).  Key blocks that lie wholly inside the prefix may then be requested
+ * before that kernel has completed; rows from prefix_len on, Q, V, the parents and the page table
+ * are still read afterwards.  Used by the contiguous-cache single-wave kernel; 0 is always correct.
  */
 typedef struct sb_tree_batch {
   int32_t batch;      /* B >= 1                                                     */
@@ -102,7 +108,7 @@ typedef struct sb_tree_batch {
   int32_t max_nodes;         /* host upper bound on N_b (<= SB_MAX_NODES)           */
   int32_t max_kv_len;        /* host upper bound on P_b + N_b                       */
   int32_t index_arrays_settled; /* 0, or 1: see below                                */
-  int32_t reserved;          /* 0                                                   */
+  int32_t prefix_rows_settled;  /* 0, or 1: see below (needs index_arrays_settled)   */
 } sb_tree_batch;
 
 /*

@@ -39,7 +39,7 @@ class _TreeBatch(C.Structure):
         ("num_pages", C.c_int32), ("total_nodes", C.c_int32), ("page_table", C.c_void_p),
         ("prefix_len", C.c_void_p), ("node_offsets", C.c_void_p), ("parent", C.c_void_p),
         ("max_nodes", C.c_int32), ("max_kv_len", C.c_int32),
-        ("index_arrays_settled", C.c_int32), ("reserved", C.c_int32),
+        ("index_arrays_settled", C.c_int32), ("prefix_rows_settled", C.c_int32),
     ]
 
 
@@ -139,7 +139,7 @@ class TreeBatch:
     num_pages: int = 0
     max_pages: int = 0
 
-    def c_struct(self, k_cache=None, v_cache=None, settled=False) -> _TreeBatch:
+    def c_struct(self, k_cache=None, v_cache=None, settled=False, prefix_settled=False) -> _TreeBatch:
         k = self.k_cache if k_cache is None else k_cache
         v = self.v_cache if v_cache is None else v_cache
         s = _TreeBatch()
@@ -154,7 +154,8 @@ class TreeBatch:
         s.node_offsets = _ptr(self.node_offsets, torch.int32).value
         s.parent = _ptr(self.parent, torch.int32).value
         s.max_nodes, s.max_kv_len = self.max_nodes, self.max_kv_len
-        s.index_arrays_settled, s.reserved = (1 if settled else 0), 0
+        s.index_arrays_settled = 1 if settled else 0
+        s.prefix_rows_settled = 1 if (settled and prefix_settled) else 0
         return s
 
 
@@ -181,18 +182,20 @@ def sb_tree_attention_workspace_bytes(tb: TreeBatch, total_q: int, num_splits: i
 
 def sb_tree_attention(tb: TreeBatch, q, out=None, lse=None, *, q_node_begin=None, q_offsets=None,
                       scale=0.0, num_splits=0, workspace=None, status=None, want_lse=True,
-                      k_cache=None, v_cache=None, index_arrays_settled=False):
+                      k_cache=None, v_cache=None, index_arrays_settled=False, prefix_rows_settled=False):
     """q bf16 [total_q, Hq, D] -> (out bf16 like q, lse fp32 [total_q, Hq] or None, status [B]).
     k_cache / v_cache override the batch's layer (same layout) without rebuilding it.
     index_arrays_settled: the kernel enqueued just before this call does not write the batch's index
-    arrays (e.g. it is the previous layer's attention): the lengths may be fetched under its tail."""
+    arrays (e.g. it is the previous layer's attention): the lengths may be fetched under its tail.
+    prefix_rows_settled (with index_arrays_settled): nor does it write cache rows below prefix_len: key
+    blocks inside the prefix may be requested under its tail too."""
     total_q = q.shape[0]
     dev = q.device
     out = torch.empty_like(q) if out is None else out
     if lse is None and want_lse:
         lse = torch.empty((total_q, tb.n_q_heads), dtype=torch.float32, device=dev)
     status = torch.empty(tb.prefix_len.numel(), dtype=torch.int32, device=dev) if status is None else status
-    s = tb.c_struct(k_cache, v_cache, index_arrays_settled)
+    s = tb.c_struct(k_cache, v_cache, index_arrays_settled, prefix_rows_settled)
     lib = load()
     if workspace is None:
         need = int(lib.sb_tree_attention_workspace_bytes(C.byref(s), C.c_int32(total_q),

@@ -136,11 +136,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const int b = (!FAST && p.sort_seqs) ? sequence_of_rank(p.tb, blockIdx.z, reinterpret_cast<int*>(s_anc), s_parent)
                                        : (int)blockIdx.z;
   const SeqPre pre = plan_lengths(p, b);
-  if (lengths_early) asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // A second vouch, for the committed prefix's cache rows (positions below prefix_len): the K blocks of this
+  // CTA's first two stages that lie wholly inside the prefix are requested before the wait as well, so that
+  // they are on their way from HBM while the predecessor finishes (Q, a fresh product of that predecessor,
+  // comes from L2 and is faster anyway).  Contiguous single-wave variant only.
+  const bool kv_early = FAST && lengths_early && p.tb.prefix_rows_settled != 0;
+  if (lengths_early && !kv_early) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!kv_early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int rows_total = pre.info.nq * G;
   const int row0 = tile * TC_BM;
   if (!pre.can_write || row0 >= rows_total) {  // uniform over the cluster
+    if (kv_early) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
     // the designated CTA always owns rows unless the sequence has none; its status is still due
     if (split == 0 && blockIdx.y == 0 && tid == 0) p.status[b] = pre.info.err;
     if (warp == TC_MMA_WARP)
@@ -220,6 +229,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   // the K side (Q, K blocks 0 and 1) is requested at once; the V blocks, needed a softmax later,
   // follow when K block 0 has landed, so they do not queue in front of it in the memory system.
   if (nb > 0 && lane == 0 && warp == TC_KLOAD_WARP) {
+    bool k0e = false, k1e = false;
+    if (kv_early) {
+      if (key_begin + TC_BN <= pre.info.P) {
+        issue_block(0, &kmap, smem_u32(sK), &s_bar[K_FULL0]);
+        k0e = true;
+      }
+      if (nb > 1 && key_begin + 2 * TC_BN <= pre.info.P) {
+        issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
+        k1e = true;
+      }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
     if (q_tma) {
       mbar_expect_tx(&s_bar[Q_FULL], (uint32_t)(TC_BM * D * 2));
 #pragma unroll
@@ -227,8 +249,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
         tma_load_3d(smem_u32(sQ) + h * (TC_BM * 128), &qmap, h * 64, g * G, pre.info.q_off + tile * (TC_BM / G),
                     &s_bar[Q_FULL]);
     }
-    issue_block(0, &kmap, smem_u32(sK), &s_bar[K_FULL0]);
-    if (nb > 1) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
+    if (!k0e) issue_block(0, &kmap, smem_u32(sK), &s_bar[K_FULL0]);
+    if (nb > 1 && !k1e) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
+  } else if (kv_early) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
 
   const SeqPlan sp = plan_tree(p, b, split == 0 && blockIdx.y == 0, pre, s_parent, s_anc);

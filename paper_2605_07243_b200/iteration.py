@@ -234,7 +234,8 @@ class SpecBlockIteration:
         for l in range(self.n_layers):
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,
                                  num_splits=self.num_splits, workspace=self.attn_ws, status=self.attn_status,
-                                 k_cache=self.k_all[l], v_cache=self.v_all[l], index_arrays_settled=l > 0)
+                                 k_cache=self.k_all[l], v_cache=self.v_all[l], index_arrays_settled=l > 0,
+                                 prefix_rows_settled=l > 0)
         if self.temperature > 0.0:   # rejection sampling against the target: the drafter rows come through child_row
             sb.sb_verify_sample(self.logits, self.scores_all, self.node_offsets, self.tree["parent"], self.tree["tok"],
                                 self.child_row, self.temperature, self.u_accept, self.u_bonus, self.max_depth,

@@ -246,10 +246,11 @@ class VerifyStep:
         first = True
         for l in range(self.n_layers) if layers is None else layers:
             # from the second layer on the kernel just before is the previous layer's attention, which
-            # writes none of the index arrays: the lengths may be read under its tail
+            # writes neither the index arrays nor the cache: lengths and prefix keys may be read under its tail
             sb.sb_tree_attention(self.tb, self.q_all[l], self.out_all[l], self.lse_all[l], scale=self.scale,
                                  num_splits=self.num_splits, workspace=self.attn_ws, status=self.attn_status,
                                  k_cache=self.k_all[l], v_cache=self.v_all[l], index_arrays_settled=not first,
+                                 prefix_rows_settled=not first,
                                  **self.kw)
             first = False
 

@@ -332,15 +332,20 @@ def test_random_shapes_against_oracle(seed, monkeypatch):
                     num_splits=splits)
 
 
-def test_index_arrays_settled_gives_the_same_bits():
-    """The flag only moves the fetch of the sequence lengths ahead of the dependency wait: same results,
-    on the compile-time variant (config 2), a paged ragged batch and a drafter call with cached nodes."""
+def test_settled_flags_give_the_same_bits():
+    """The flags only move the fetch of the sequence lengths, and of key blocks inside the prefix, ahead of
+    the dependency wait: same results, on the compile-time variant (config 2, with chunks that lie inside
+    the prefix, straddle its end, or hold tree rows only), a paged ragged batch and a drafter call with
+    cached nodes."""
     rng = W.rng_for(431)
     ragged = W.make_attn_case(rng, parents=[W.random_tree(rng, 40, 6), W.chain_tree(7), W.random_tree(rng, 90, 9)],
                               prefix_lens=[700, 33, 0], n_q_heads=16, n_kv_heads=4, head_dim=128, page_size=64)
-    for case in (W.config2_verify_layer(prefix=600), ragged, W.config3_drafter(prefix=900)[0]):
+    for case in (W.config2_verify_layer(prefix=600), W.config2_verify_layer(prefix=130), W.config2_verify_layer(),
+                 ragged, W.config3_drafter(prefix=900)[0]):
         plain = gpu_attention(case)
-        flagged = gpu_attention(case, index_arrays_settled=True)
-        for a, b in zip(plain, flagged):
-            np.testing.assert_array_equal(a, b)
+        for flags in (dict(index_arrays_settled=True), dict(index_arrays_settled=True, prefix_rows_settled=True),
+                      dict(prefix_rows_settled=True)):
+            flagged = gpu_attention(case, **flags)
+            for a, b in zip(plain, flagged):
+                np.testing.assert_array_equal(a, b)
         assert (plain[2] == 0).all()

@@ -60,7 +60,7 @@ def test_binding_struct_matches_header_layout():
     assert names == ["batch", "n_q_heads", "n_kv_heads", "head_dim", "k_cache", "v_cache",
                      "page_size", "max_pages", "kv_capacity", "num_pages", "total_nodes",
                      "page_table", "prefix_len", "node_offsets", "parent", "max_nodes",
-                     "max_kv_len", "index_arrays_settled", "reserved"]
+                     "max_kv_len", "index_arrays_settled", "prefix_rows_settled"]
     assert s.k_cache.offset == 16 and s.kv_capacity.offset == 40 and s.page_table.offset == 56
     assert s.max_nodes.offset == 88 and s.index_arrays_settled.offset == 96
     assert ctypes.sizeof(s) == 104
