@@ -570,16 +570,17 @@ static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_spl
       sp.outer = num_splits < max_blocks ? num_splits : max_blocks;
       return sp;
     }
-    // CTAs run in waves; a CTA costs its blocks (two tiles each) plus a fixed start-up worth about
-    // five, and every chunk beyond the first writes and re-reads an fp32 partial of all rows, here
-    // in units of one block-time (1.2 us) at 6 TB/s.
+    // CTAs run in waves; a CTA costs its blocks (two tiles each) plus a fixed start-up and epilogue
+    // (about 11 us measured on the long-context configuration: nine block-times), and every chunk beyond
+    // the first writes and re-reads a bf16 partial of all rows, here in units of one block-time
+    // (1.2 us) at 6 TB/s.
     const long long units = (long long)tb->batch * tb->n_kv_heads * ceil_div(row_tiles, 2);
-    const double partial = 2.0 * (double)total_q * tb->n_q_heads * tb->head_dim * 4.0 / 6e12 / 1.2e-6;
+    const double partial = 2.0 * (double)total_q * tb->n_q_heads * tb->head_dim * 2.0 / 6e12 / 1.2e-6;
     int best = 1;
     double best_cost = 0.0;
     for (int s = 1; s <= 8 && s <= max_blocks; ++s) {
       const long long waves = (units * s + sms - 1) / sms;
-      const double cost = (double)waves * (2 * ceil_div(max_blocks, s) + 5) + (s > 1 ? partial * s + 3.0 : 0.0);
+      const double cost = (double)waves * (2 * ceil_div(max_blocks, s) + 9) + (s > 1 ? partial * s + 3.0 : 0.0);
       if (s == 1 || cost < best_cost) {
         best = s;
         best_cost = cost;

@@ -16,8 +16,8 @@
 //   order, so S_{v+2} overwrites P_v only after PV_v has read it, and S_{v+1} (the other tile) is
 //   computed while the softmax warps work on v.
 // Everything else (TMA loaders, visibility windows, lazy reference maximum, bounded waits) is as in
-// attn_tc_kernel.  CTAs are not clustered: with more than one KV chunk every CTA writes an fp32
-// partial and attn_merge_kernel merges them.
+// attn_tc_kernel.  CTAs are not clustered: with more than one KV chunk every CTA writes a bf16
+// partial (its rows are rounded to bf16 when they are staged anyway) and attn_merge_kernel merges them.
 #include <cstdio>
 #include <cstdlib>
 
@@ -435,7 +435,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
   // ---- normalise and store, one tile after the other ------------------------------------------------
   // The softmax threads stage the tile's rows as [O / l in bf16 (D) | m | l | pad] over the idle Q
   // tiles; then half a warp per row writes whole rows: the output row and its log-sum-exp, or, with
-  // several KV chunks, this chunk's fp32 partial for attn_merge_kernel.
+  // several KV chunks, this chunk's bf16 partial for attn_merge_kernel.
   constexpr int ROWB = D * 2 + 16;  // bytes per staged row (16-byte multiple)
   tc_fence_before();
   __syncthreads();  // every role is done: no async access to Q/K/V stages is in flight any more
