@@ -220,7 +220,10 @@ class SpecBlockIteration:
         for l in range(n_layers):
             if l < len(e.get("attn", [])):
                 a = e["attn"][l]
-                sb.sb_tree_attention(a["tb"], a["q"], a["out"], a["lse"], workspace=a["ws"], status=a["status"], **a["kw"])
+                # the block's index arrays and its drafter cache are inputs that no kernel of the chain writes:
+                # whatever was enqueued just before, lengths and prefix keys may be fetched under its tail
+                sb.sb_tree_attention(a["tb"], a["q"], a["out"], a["lse"], workspace=a["ws"], status=a["status"],
+                                     index_arrays_settled=True, prefix_rows_settled=True, **a["kw"])
             if l < len(e.get("hidden", [])):
                 sb.sb_shift_project(e["hidden"][l], w["w_shift"][l], self.block_k, out=e["shifted"][l],
                                     workspace=e["shift_ws"], status=e["shift_status"])
