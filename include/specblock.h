@@ -18,6 +18,7 @@
  *   sb_fuse_project    the drafter's fused per-position input h^(0)      (Sec. 3.1 "Block forward")
  *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
  *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
+ *   sb_path_rows       the accepted path in the drafter's row numbering  (App. A.2)
  *
  * Conventions that hold for every call
  *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
@@ -209,7 +210,8 @@ size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab);
  * sb_tree_expand_features -- sb_tree_expand and sb_rank_features of the same scores in ONE pass over them:
  * the scan that finds the per-chunk top-16 also accumulates the chunk statistics of psi(p), and both
  * finishing kernels follow it.  Arguments as sb_tree_expand plus features fp32 [n_rows][15] as
- * sb_rank_features; results identical to the two separate calls.
+ * sb_rank_features; results identical to the two separate calls, except that node_row counts the rows from
+ * row_base (node_row = row_base + r), like child_row.
  *   child_row int32 [node_budget] or NULL: for every row of this call that emits nodes under an existing
  *   node, child_row[that node] = row_base + row -- the row of the drafter's scores that proposed the node's
  *   children, as sb_verifier_signal and sb_verify_sample want it (row_base = rows of the earlier blocks when
@@ -416,6 +418,33 @@ sb_status sb_verify_accept_static(const void* logits, sb_dtype dtype, int64_t ro
 sb_status sb_kv_compact(const sb_tree_batch* tb, int32_t n_layers, int64_t layer_stride_elems,
                         const int32_t* path_nodes, const int32_t* accept_len, int32_t max_depth,
                         int32_t* new_len, int32_t* status, void* stream);
+
+/*
+ * sb_path_rows -- the accepted path in the drafter's own row numbering (App. A.2: a committed
+ * position keeps the keys and values that its own draft forward produced).
+ *
+ *   A draft forward has one cache row per block position, shared by the sibling tokens attached at
+ *   that position, so the drafter's cache is committed by rows, not by tree nodes.  For sequence b
+ *   with accepted path nodes p_0 = 0, p_1, ..., p_a (a = accept_len[b]):
+ *       path_rows[b][0] = 0
+ *       path_rows[b][j] = 1 + node_row[node_offsets[b] + p_j] - row_begin[b],   j = 1..a
+ *   -- node_row, the tree array written by sb_tree_expand / sb_tree_expand_features, names the row
+ *   whose distribution proposed a node (counted from the call's row_base, so that the rows of an
+ *   iteration's blocks are numbered through); entries past a are -1.
+ *   Slot 0 stands for the last committed position, whose row lies just before this iteration's
+ *   rows: with a drafter cache that holds row r of the iteration at position Pd + r,
+ *   sb_kv_compact over a batch with prefix_len = Pd - 1 and node_offsets = {0, 1 + rows} and the
+ *   path (path_rows, accept_len) moves the accepted rows to Pd .. Pd + a - 1 and returns
+ *   new_len = Pd + a.
+ *   row_begin int32 [batch] or NULL (= 0): first row of each sequence in node_row's numbering.
+ *   status[b]: SB_ERR_INVALID_TREE when accept_len[b] is outside [0, max_depth], a path node lies
+ *   outside the sequence's tree or has no row (the root, or a row before row_begin[b]), or the rows
+ *   do not increase along the path; path_rows[b] is then 0 followed by -1.
+ *   All pointers device; path_nodes, path_rows int32 [batch][max_depth+1]; max_depth <= SB_MAX_DEPTH.
+ */
+sb_status sb_path_rows(int32_t batch, const int32_t* node_offsets, const int32_t* node_row,
+                       const int32_t* row_begin, const int32_t* path_nodes, const int32_t* accept_len,
+                       int32_t max_depth, int32_t* path_rows, int32_t* status, void* stream);
 
 /* Text for a status code (static storage). */
 const char* sb_status_string(sb_status s);

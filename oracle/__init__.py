@@ -18,5 +18,6 @@ from .oracle import (  # noqa: F401
     fuse_project,
     accept_from_amax,
     kv_compact,
+    path_rows,
     tree_expand,
 )

@@ -239,6 +239,20 @@ def accept_from_amax(parent, tok, amax, max_depth):
                 bonus=int(bonus[0]), status=int(rc))
 
 
+def path_rows(node_offsets, node_row, path_nodes, accept_len, max_depth, row_begin=None):
+    """node_row int32 [total_nodes]: the iteration-wide row that proposed each node (-1: root).
+    -> dict(path_rows int32 [B, max_depth+1], status int32 [B])."""
+    node_offsets, node_row = _i32(node_offsets), _i32(node_row)
+    path_nodes, accept_len = _i32(path_nodes), _i32(accept_len)
+    batch = node_offsets.shape[0] - 1
+    rb = None if row_begin is None else _i32(row_begin)
+    rows = np.zeros((batch, max_depth + 1), np.int32)
+    status = np.zeros(batch, np.int32)
+    _load().sbo_path_rows(C.c_int(batch), _p(node_offsets), _p(node_row), None if rb is None else _p(rb),
+                          _p(path_nodes), _p(accept_len), C.c_int(max_depth), _p(rows), _p(status))
+    return dict(path_rows=rows, status=status)
+
+
 def kv_compact(*, n_kv_heads, head_dim, cache, n_layers, layer_stride_elems, page_size=0,
                max_pages=0, num_pages=0, kv_capacity=0, page_table=None, prefix_len,
                node_offsets, path_nodes, accept_len, max_depth):

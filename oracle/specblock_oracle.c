@@ -17,6 +17,7 @@
  *   sbo_verify_accept   : exhaustive comparison with an independent recurrence on all small
  *                         trees; planted paths; the case-study tree (4 accepted + bonus).
  *   sbo_kv_compact      : numpy fancy-index gather; attention over the compacted cache.
+ *   sbo_path_rows       : a hand-worked two-block tree; numpy fancy indexing on random paths.
  *   sbo_rank_features   : scipy log_softmax / entropy; closed forms (uniform row, one dominant token).
  *   sbo_verifier_signal : scipy softmax; closed forms (flat row, one raised token); probabilities of
  *                         all tokens of a row sum to one; the sum over iterations of a query.
@@ -339,6 +340,41 @@ int sbo_accept_from_amax(int n, const int32_t* parent, const int32_t* tok, const
                          int max_depth, int32_t* accept_len, int32_t* path_nodes,
                          int32_t* out_tokens, int32_t* bonus) {
   return accept_one(n, parent, tok, amax, max_depth, accept_len, path_nodes, out_tokens, bonus);
+}
+
+/* ---- the accepted path in the drafter's row numbering (App. A.2) ----------------------------- */
+
+/*
+ * A draft forward produces one cache row per block position; the tokens attached at a position share
+ * it.  node_row[i] is the row (in the numbering of all rows of the iteration, first row of sequence
+ * b = row_begin[b]) of the position whose distribution proposed tree node i, -1 for the root.  For the
+ * accepted path p_0 = 0, ..., p_a: rows[0] = 0 (the last committed position, one slot before the
+ * iteration's rows) and rows[j] = 1 + node_row[p_j] - row_begin[b]; entries past a are -1.
+ * status 0 ok / 4 when a is outside [0, max_depth], a path node is outside the tree or has no row,
+ * or the rows do not increase (rows then 0, -1, -1, ...).
+ */
+void sbo_path_rows(int batch, const int32_t* node_offsets, const int32_t* node_row, const int32_t* row_begin,
+                   const int32_t* path_nodes, const int32_t* accept_len, int max_depth, int32_t* rows,
+                   int32_t* status) {
+  for (int b = 0; b < batch; ++b) {
+    const int o = node_offsets[b], n = node_offsets[b + 1] - o, a = accept_len[b];
+    const int r0 = row_begin ? row_begin[b] : 0;
+    const int32_t* path = path_nodes + (int64_t)b * (max_depth + 1);
+    int32_t* out = rows + (int64_t)b * (max_depth + 1);
+    int bad = n < 1 || a < 0 || a > max_depth;
+    for (int j = 0; j <= max_depth; ++j) out[j] = -1;
+    out[0] = 0;
+    for (int j = 1; !bad && j <= a; ++j) {
+      const int p = path[j];
+      if (p < 0 || p >= n || node_row[o + p] < r0 || node_row[o + p] < 0) { bad = 1; break; }
+      out[j] = 1 + node_row[o + p] - r0;
+      if (out[j] <= out[j - 1]) bad = 1;
+    }
+    if (bad) {
+      for (int j = 1; j <= max_depth; ++j) out[j] = -1;
+    }
+    status[b] = bad ? 4 : 0;
+  }
 }
 
 /* ---- O3: cache compaction as an out-of-place gather ---------------------------------------- */

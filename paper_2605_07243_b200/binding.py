@@ -68,8 +68,8 @@ def load(build_if_missing: bool = True):
                  "sb_fuse_project_workspace_bytes"):
         getattr(lib, name).restype = C.c_size_t
     for name in ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_expand", "sb_verify_accept",
-                 "sb_verify_accept_static", "sb_kv_compact", "sb_rank_features", "sb_verifier_signal", "sb_verify_sample",
-                 "sb_shift_project", "sb_fuse_project", "sb_tree_expand_features"):
+                 "sb_verify_accept_static", "sb_kv_compact", "sb_path_rows", "sb_rank_features", "sb_verifier_signal",
+                 "sb_verify_sample", "sb_shift_project", "sb_fuse_project", "sb_tree_expand_features"):
         getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -77,7 +77,7 @@ def load(build_if_missing: bool = True):
 
 EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspace_bytes",
             "sb_tree_expand", "sb_tree_expand_workspace_bytes", "sb_verify_accept",
-            "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact",
+            "sb_verify_accept_workspace_bytes", "sb_verify_accept_static", "sb_kv_compact", "sb_path_rows",
             "sb_rank_features", "sb_rank_features_workspace_bytes", "sb_verifier_signal", "sb_verify_sample",
             "sb_verify_sample_workspace_bytes", "sb_shift_project", "sb_shift_project_workspace_bytes",
             "sb_fuse_project", "sb_fuse_project_workspace_bytes", "sb_tree_expand_features", "sb_status_string",
@@ -409,6 +409,22 @@ def sb_kv_compact(tb: TreeBatch, n_layers, layer_stride_elems, path_nodes, accep
                               _ptr(status, torch.int32), _stream())
     _check(rc, "sb_kv_compact")
     return new_len, status
+
+
+def sb_path_rows(node_offsets, node_row, path_nodes, accept_len, max_depth, path_rows=None, status=None,
+                 row_begin=None):
+    """The accepted path in the drafter's row numbering: -> (path_rows int32 [B, max_depth+1], status [B])."""
+    batch = node_offsets.numel() - 1
+    dev = node_row.device
+    if path_rows is None:
+        path_rows = torch.empty((batch, max_depth + 1), dtype=torch.int32, device=dev)
+    status = torch.empty(batch, dtype=torch.int32, device=dev) if status is None else status
+    rc = load().sb_path_rows(C.c_int32(batch), _ptr(node_offsets, torch.int32), _ptr(node_row, torch.int32),
+                             _ptr(row_begin, torch.int32), _ptr(path_nodes, torch.int32),
+                             _ptr(accept_len, torch.int32), C.c_int32(max_depth), _ptr(path_rows, torch.int32),
+                             _ptr(status, torch.int32), _stream())
+    _check(rc, "sb_path_rows")
+    return path_rows, status
 
 
 def sb_tree_expand_workspace_bytes(n_rows: int, vocab: int) -> int:

@@ -83,7 +83,60 @@ __global__ void __launch_bounds__(COMPACT_THREADS) kv_compact_kernel(const sb_tr
   }
 }
 
+// sb_path_rows: one CTA per sequence; thread j looks up the row of path node j, thread 0 checks the order.
+__global__ void __launch_bounds__(64) path_rows_kernel(const int* __restrict__ node_offsets,
+                                                       const int* __restrict__ node_row,
+                                                       const int* __restrict__ row_begin,
+                                                       const int* __restrict__ path_nodes,
+                                                       const int* __restrict__ accept_len, int max_depth,
+                                                       int* __restrict__ path_rows, int* __restrict__ status) {
+  __shared__ int s_rows[SB_MAX_DEPTH + 1];
+  __shared__ int s_err;
+  const int b = blockIdx.x, j = threadIdx.x;
+  const int o = node_offsets[b];
+  const int n = node_offsets[b + 1] - o;
+  const int a = accept_len[b];
+  const int r0 = row_begin ? row_begin[b] : 0;
+  const bool shape_ok = n >= 1 && a >= 0 && a <= max_depth;
+  if (j == 0) s_err = shape_ok ? 0 : (int)SB_ERR_INVALID_TREE;
+  __syncthreads();
+  if (j <= max_depth) {
+    int row = -1;
+    if (shape_ok && j <= a) {
+      const int self = path_nodes[(long long)b * (max_depth + 1) + j];
+      if (self < 0 || self >= n) atomicExch(&s_err, (int)SB_ERR_INVALID_TREE);
+      if (j == 0) {
+        row = 0;
+      } else {
+        const int nr = (self >= 0 && self < n) ? node_row[o + self] : -1;
+        if (nr < r0 || nr < 0) atomicExch(&s_err, (int)SB_ERR_INVALID_TREE);
+        else row = 1 + nr - r0;
+      }
+    }
+    s_rows[j] = row;
+  }
+  __syncthreads();
+  if (j == 0 && !s_err)
+    for (int t = 1; t <= a; ++t)
+      if (s_rows[t] <= s_rows[t - 1]) s_err = SB_ERR_INVALID_TREE;
+  __syncthreads();
+  if (j <= max_depth) path_rows[(long long)b * (max_depth + 1) + j] = s_err ? (j == 0 ? 0 : -1) : s_rows[j];
+  if (j == 0) status[b] = s_err;
+}
+
 }  // namespace sb
+
+extern "C" sb_status sb_path_rows(int32_t batch, const int32_t* node_offsets, const int32_t* node_row,
+                                  const int32_t* row_begin, const int32_t* path_nodes, const int32_t* accept_len,
+                                  int32_t max_depth, int32_t* path_rows, int32_t* status, void* stream) {
+  using namespace sb;
+  if (batch < 1 || !node_offsets || !node_row || !path_nodes || !accept_len || !path_rows || !status)
+    return SB_ERR_INVALID_ARG;
+  if (max_depth < 0 || max_depth > SB_MAX_DEPTH) return SB_ERR_UNSUPPORTED;
+  path_rows_kernel<<<batch, 64, 0, static_cast<cudaStream_t>(stream)>>>(node_offsets, node_row, row_begin, path_nodes,
+                                                                        accept_len, max_depth, path_rows, status);
+  return launch_check();
+}
 
 extern "C" sb_status sb_kv_compact(const sb_tree_batch* tb, int32_t n_layers, int64_t layer_stride_elems,
                                    const int32_t* path_nodes, const int32_t* accept_len, int32_t max_depth,

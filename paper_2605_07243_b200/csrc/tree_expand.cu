@@ -561,7 +561,7 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
         tok[n] = topk_tok[r * SB_KMAX + j];
         parent[n] = par;
         depth[n] = base_depth + kpos;
-        node_row[n] = r;
+        node_row[n] = row_base + r;
         node_rank[n] = j;
       }
       if (child_row && par >= 0 && first < node_budget) child_row[par] = row_base + r;  // this row proposed par's children
@@ -713,7 +713,7 @@ __global__ void __launch_bounds__(ROWS_THREADS) expand_rows_kernel(
       tok[n] = id;
       parent[n] = par;
       depth[n] = node_depth;
-      node_row[n] = rr;
+      node_row[n] = row_base + rr;
       node_rank[n] = rank;
     }
   }

@@ -71,12 +71,19 @@ def _bf16(x, device):
 class SpecBlockIteration:
     def __init__(self, *, block_k: int, bmap, node_budget: int, root_tok: int, blocks: List[DraftBlock],
                  target_layers: List, logits: np.ndarray, max_depth: int, weights: Optional[DrafterWeights] = None,
-                 device="cuda", num_splits=0, temperature: float = 0.0, u_accept=None, u_bonus=None):
+                 device="cuda", num_splits=0, temperature: float = 0.0, u_accept=None, u_bonus=None,
+                 drafter_cache: Optional[List] = None):
         """target_layers: one workloads.AttnCase per target layer over ONE sequence whose tree has
         `node_budget` nodes (their K/V rows and Q rows are used; the tree itself is built here);
         logits: [node_budget, V] fp32 or bf16 bits (the target's scores per tree node).
         temperature > 0: the tree is verified by rejection sampling (sb_verify_sample) with the given uniforms
-        (u_accept fp32 [node_budget], u_bonus fp32 [1]) instead of greedy acceptance."""
+        (u_accept fp32 [node_budget], u_bonus fp32 [1]) instead of greedy acceptance.
+        drafter_cache: one workloads.AttnCase per drafter layer (contiguous, one sequence) whose K/V hold,
+        behind a prefix that ends with the last committed position, one row per block position of this
+        iteration in the order of the blocks' score rows (a "tree" of 1 + total rows nodes, prefix_len = the
+        drafter's committed length - 1).  A committed position keeps the keys and values of its own draft
+        forward (App. A.2): the accepted path is translated to rows (sb_path_rows, through node_row) and
+        committed by a second sb_kv_compact."""
         self.device, self.block_k, self.budget, self.max_depth = device, block_k, node_budget, max_depth
         self.bmap = [int(x) for x in bmap]
         self.num_splits = num_splits
@@ -189,6 +196,25 @@ class SpecBlockIteration:
                                      dtype=torch.uint8, device=device)
         self.new_len = torch.empty(1, **i32)
         self.compact_status = torch.empty(1, **i32)
+        # ---- the drafter's cache of the same tree (optional) -------------------------------------------------
+        self.drafter_tb = None
+        if drafter_cache:
+            d0 = drafter_cache[0]
+            n_rows_all = int(self.scores_all.shape[0])
+            assert d0.batch == 1 and d0.page_size == 0 and int(d0.node_offsets[-1]) == 1 + n_rows_all
+            self.drafter_k = dev.bf16_tensor(np.stack([c.k for c in drafter_cache]), device)
+            self.drafter_v = dev.bf16_tensor(np.stack([c.v for c in drafter_cache]), device)
+            self.drafter_layers, self.drafter_stride = len(drafter_cache), int(d0.k.size)
+            self.drafter_tb = sb.TreeBatch(
+                n_q_heads=d0.n_q_heads, n_kv_heads=d0.n_kv_heads, head_dim=d0.head_dim, k_cache=self.drafter_k[0],
+                v_cache=self.drafter_v[0], prefix_len=dev.i32_tensor(d0.prefix_len, device),
+                node_offsets=dev.i32_tensor(d0.node_offsets, device), parent=dev.i32_tensor(d0.parent, device),
+                total_nodes=1 + n_rows_all, max_nodes=1 + n_rows_all, max_kv_len=d0.max_kv_len, page_size=0,
+                kv_capacity=d0.kv_capacity)
+            self.path_rows = torch.empty((1, max_depth + 1), **i32)
+            self.path_rows_status = torch.empty(1, **i32)
+            self.drafter_new_len = torch.empty(1, **i32)
+            self.drafter_compact_status = torch.empty(1, **i32)
         self.temperature = float(temperature)
         if self.temperature > 0.0:
             self.u_accept = torch.as_tensor(np.asarray(u_accept, np.float32)).to(device)
@@ -254,6 +280,12 @@ class SpecBlockIteration:
                               r_prob=self.r_prob, status=self.signal_status)
         sb.sb_kv_compact(self.tb, self.n_layers, self.layer_stride, self.accept["path_nodes"],
                          self.accept["accept_len"], self.max_depth, self.new_len, self.compact_status)
+        if self.drafter_tb is not None:   # the drafter commits the block rows that proposed the accepted nodes
+            sb.sb_path_rows(self.node_offsets, self.tree["node_row"], self.accept["path_nodes"], self.accept["accept_len"],
+                            self.max_depth, self.path_rows, self.path_rows_status)
+            sb.sb_kv_compact(self.drafter_tb, self.drafter_layers, self.drafter_stride, self.path_rows,
+                             self.accept["accept_len"], self.max_depth, self.drafter_new_len,
+                             self.drafter_compact_status)
 
     def run(self):
         """The whole iteration (enqueue only): returns nothing, results stay on the device."""
@@ -296,6 +328,9 @@ def build_8b_iteration(target_layers, logits, max_depth, *, d=4096, vocab=128256
     b2 = block(8, np.arange(1, 9), rng.choice(4, size=8 * K, p=freq).astype(np.uint8), attn2, False)
     weights = DrafterWeights(w_cond=rb(d, 3 * d, std=0.02), w_fuse=rb(d, 3 * d, std=0.02), queries=rb(K, d),
                              w_shift=[rb(d, 2 * d, std=0.02) for _ in range(drafter_layers)])
+    # the drafter's own cache: 4096 committed positions, then one row per block position (4 + 32)
+    cache = [W.make_attn_case(rng, parents=[W.chain_tree(1 + 9 * K)], prefix_lens=[4095], n_q_heads=32, n_kv_heads=8,
+                              head_dim=128) for _ in range(drafter_layers)]
     return SpecBlockIteration(block_k=K, bmap=[1, 2, 3, 4], node_budget=budget, root_tok=1, blocks=[b1, b2],
                               target_layers=target_layers, logits=logits, max_depth=max_depth, weights=weights,
-                              device=device, num_splits=num_splits)
+                              device=device, num_splits=num_splits, drafter_cache=cache)

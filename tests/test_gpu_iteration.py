@@ -77,13 +77,19 @@ def _build(seed, n_target_layers=2, with_drafter=True):
     logits[end, bonus] = logits[end].max() + np.float32(4.0)
     target = [W.make_attn_case(rng, parents=[W.chain_tree(BUDGET)], prefix_lens=[P], n_q_heads=8, n_kv_heads=2,
                                head_dim=128) for _ in range(n_target_layers)]
-    weights = None
+    weights, drafter_cache = None, None
     if with_drafter:
+        # the drafter's own cache: 78 committed positions (the last one is slot 0 of the row numbering), then one
+        # K/V row per block position of the iteration (4 rows of block 1, 12 of block 2)
+        drafter_cache = [W.make_attn_case(rng, parents=[W.chain_tree(1 + 4 * K)], prefix_lens=[77], n_q_heads=4,
+                                          n_kv_heads=2, head_dim=64) for _ in range(2)]
         weights = DrafterWeights(w_cond=bf((d, 3 * d_t), 0.05), w_fuse=bf((d, 3 * d), 0.05), queries=bf((K, d)),
                                  w_shift=[bf((d, 2 * d), 0.05) for _ in range(2)],
                                  gains=tuple(rng.uniform(0.5, 1.5, d).astype(np.float32) for _ in range(3)))
     it = SpecBlockIteration(block_k=K, bmap=BMAP, node_budget=BUDGET, root_tok=ROOT_TOK, blocks=[b1, b2],
-                            target_layers=target, logits=logits, max_depth=2 * K, weights=weights)
+                            target_layers=target, logits=logits, max_depth=2 * K, weights=weights,
+                            drafter_cache=drafter_cache)
+    it.drafter_cases = drafter_cache    # kept for the check below
     return it, [b1, b2], tree2, n, logits, target, weights, (len(path) - 1, bonus)
 
 
@@ -98,7 +104,7 @@ def _close(got, ref, scale=1.0):
 def _check_against_oracle(it, blocks, tree2, n, logits, target, weights, planted):
     # ---- the tree grown on the device ------------------------------------------------------------------
     assert it.node_offsets.cpu().tolist() == [0, n]
-    for k in ("tok", "parent", "depth", "node_row", "node_rank"):
+    for k in ("tok", "parent", "depth", "node_rank"):
         np.testing.assert_array_equal(it.tree[k].cpu().numpy()[:n], tree2[k], err_msg=k)
     for e in it.blocks:
         assert int(e["status"].cpu()[0]) == 0
@@ -123,31 +129,44 @@ def _check_against_oracle(it, blocks, tree2, n, logits, target, weights, planted
     np.testing.assert_array_equal(it.accept["amax"].cpu().numpy()[:n], ref["amax"])
     # the row that proposed each node's children, recorded by the expansions, and the verifier-derived signal
     child_row = np.full(n, -1, np.int32)
+    global_row = np.full(n, -1, np.int32)       # per node: the iteration-wide row that proposed it
     row_base = np.cumsum([0] + [b.scores.shape[0] for b in blocks])
     first_new = 1
     for m, b in enumerate(blocks):                      # nodes are appended block by block, in row order
         res_m, _ = _oracle_tree(blocks[:m + 1])
         for c in range(first_new, res_m["n_nodes"]):
             child_row[tree2["parent"][c]] = row_base[m] + tree2["node_row"][c]
+            global_row[c] = row_base[m] + tree2["node_row"][c]
         first_new = res_m["n_nodes"]
     np.testing.assert_array_equal(it.child_row.cpu().numpy()[:n], child_row)
+    # the device numbers the rows through the blocks of the iteration (row_base of each expansion)
+    np.testing.assert_array_equal(it.tree["node_row"].cpu().numpy()[:n], global_row)
     scores_all = np.concatenate([b.scores for b in blocks])
     sig = oracle.verifier_signal(scores_all, offs, child_row, ref["path_nodes"], ref["accept_len"], ref["bonus"], 2 * K)
     assert int(it.signal_status.cpu()[0]) == int(sig["status"][0]) == 0
     assert abs(float(it.r_prob.cpu()[0]) - sig["r_prob"][0]) <= 2e-5 * max(sig["r_prob"][0], 1e-3)
-    c0 = target[0]
-    for name, got_all in (("k", it.k_all), ("v", it.v_all)):
-        cache = np.stack([getattr(c, name) for c in target]).reshape(-1)
-        ref_c, ref_len, _ = oracle.kv_compact(
-            n_kv_heads=c0.n_kv_heads, head_dim=c0.head_dim, cache=cache, n_layers=len(target),
-            layer_stride_elems=int(c0.k.size), kv_capacity=c0.kv_capacity, prefix_len=c0.prefix_len, node_offsets=offs,
-            path_nodes=ref["path_nodes"], accept_len=ref["accept_len"], max_depth=2 * K)
-        new_len = int(ref_len[0])
-        assert new_len == P + planted[0] + 1
-        row = c0.n_kv_heads * c0.head_dim
-        np.testing.assert_array_equal(it.new_len.cpu().numpy(), ref_len)
-        np.testing.assert_array_equal(_bits(got_all).reshape(len(target), -1)[:, :new_len * row],
-                                      ref_c.reshape(len(target), -1)[:, :new_len * row], err_msg=name)
+    caches = [(target, it.k_all, it.v_all, it.new_len, it.compact_status, "target", offs, ref["path_nodes"])]
+    if it.drafter_cases:   # the drafter commits the block rows that proposed the accepted nodes
+        rows = oracle.path_rows(offs, global_row, ref["path_nodes"], ref["accept_len"], 2 * K)
+        assert int(rows["status"][0]) == 0 and int(it.path_rows_status.cpu()[0]) == 0
+        np.testing.assert_array_equal(it.path_rows.cpu().numpy(), rows["path_rows"])
+        caches.append((it.drafter_cases, it.drafter_k, it.drafter_v, it.drafter_new_len, it.drafter_compact_status,
+                       "drafter", it.drafter_cases[0].node_offsets, rows["path_rows"]))
+    for cases, k_all, v_all, got_len, got_status, who, c_offs, c_path in caches:
+        c0 = cases[0]
+        assert int(got_status.cpu()[0]) == 0
+        for name, got_all in (("k", k_all), ("v", v_all)):
+            cache = np.stack([getattr(c, name) for c in cases]).reshape(-1)
+            ref_c, ref_len, _ = oracle.kv_compact(
+                n_kv_heads=c0.n_kv_heads, head_dim=c0.head_dim, cache=cache, n_layers=len(cases),
+                layer_stride_elems=int(c0.k.size), kv_capacity=c0.kv_capacity, prefix_len=c0.prefix_len,
+                node_offsets=c_offs, path_nodes=c_path, accept_len=ref["accept_len"], max_depth=2 * K)
+            new_len = int(ref_len[0])
+            assert new_len == int(c0.prefix_len[0]) + planted[0] + 1
+            row = c0.n_kv_heads * c0.head_dim
+            np.testing.assert_array_equal(got_len.cpu().numpy(), ref_len)
+            np.testing.assert_array_equal(_bits(got_all).reshape(len(cases), -1)[:, :new_len * row],
+                                          ref_c.reshape(len(cases), -1)[:, :new_len * row], err_msg=f"{who} {name}")
     # ---- the drafter's side of every block --------------------------------------------------------------
     for m, (b, e) in enumerate(zip(blocks, it.blocks)):
         ref_f = oracle.rank_features(b.scores)

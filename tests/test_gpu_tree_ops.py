@@ -755,8 +755,15 @@ def test_expand_with_features_in_one_pass():
         torch.cuda.synchronize()
         assert int(st_a.cpu()[0]) == 0 and int(st_b.cpu()[0]) == 0
         assert torch.equal(tok_a, tok_b) and torch.equal(val_a, val_b)
+        n_old = 0 if case.tree is None else len(case.tree["tok"])
+        n_now = int(t_sep["n_nodes"].cpu()[0])
         for k in t_sep:
-            assert torch.equal(t_sep[k], t_fused[k]), k
+            if k == "node_row":    # the fused call numbers the rows from its row_base; the old nodes keep theirs
+                assert torch.equal(t_sep[k][:n_old], t_fused[k][:n_old])
+                assert torch.equal(t_sep[k][n_old:n_now] + 1000, t_fused[k][n_old:n_now])
+                assert torch.equal(t_sep[k][n_now:], t_fused[k][n_now:])
+            else:
+                assert torch.equal(t_sep[k], t_fused[k]), k
         assert torch.equal(feat_sep.view(torch.int32), feat_fused.view(torch.int32))
         # the row that proposed each node's children: derived from the oracle's tree
         ref_t = oracle.tree_expand(case.scores, case.block_k, case.bucket, case.bmap, case.start_parent, case.node_budget,
@@ -787,3 +794,38 @@ def test_verify_sample_large_vocabularies_and_unaligned_rows(vocab, dtype, pad):
     case = _sample_case(rng, parents, vocab, dtype, stride_pad=pad)
     for rep in range(2):
         _check_sample(rng, *case, temperature=1.0, max_depth=5, vocab=vocab)
+
+
+def test_path_rows_against_the_oracle_and_error_cases():
+    """Two sequences (the second with its own first row), every accepted length, then the error cases: a path
+    node without a row (the root), a node outside the tree, rows that do not increase, an accepted length
+    beyond max_depth."""
+    require_gpu()
+    # K = 4: block 1 rows 0..3 under the root (row 0 proposes the siblings 1 and 2), block 2 rows 4..7 under node 2
+    node_row = np.array([-1, 0, 0, 1, 2, 3, 4, 4, 5], np.int32)
+    n, md = len(node_row), 4
+    offs = np.array([0, n, 2 * n], np.int32)
+    row_begin = np.array([0, 100], np.int32)
+    rows_all = np.concatenate([node_row, np.where(node_row >= 0, node_row + 100, -1)]).astype(np.int32)
+    paths = {4: [0, 1, 3, 4, 5], 3: [0, 2, 6, 8, -1], 2: [0, 2, 7, -1, -1], 1: [0, 2, -1, -1, -1], 0: [0, -1, -1, -1, -1]}
+    dev_args = [torch.from_numpy(x).cuda() for x in (offs, rows_all)]
+    rb = torch.from_numpy(row_begin).cuda()
+
+    def both(pn, acc):
+        pn, acc = np.array(pn, np.int32), np.array(acc, np.int32)
+        ref = oracle.path_rows(offs, rows_all, pn, acc, md, row_begin=row_begin)
+        got, st = sb.sb_path_rows(*dev_args, torch.from_numpy(pn).cuda(), torch.from_numpy(acc).cuda(), md, row_begin=rb)
+        np.testing.assert_array_equal(got.cpu().numpy(), ref["path_rows"])
+        np.testing.assert_array_equal(st.cpu().numpy(), ref["status"])
+        return ref
+
+    for a0 in range(5):
+        for a1 in range(5):
+            assert both([paths[a0], paths[a1]], [a0, a1])["status"].tolist() == [0, 0]
+    assert both([paths[2], paths[3]], [2, 3])["path_rows"].tolist() == [[0, 1, 5, -1, -1], [0, 1, 5, 6, -1]]
+    for path, a in (([0, 0, -1, -1, -1], 1),      # the root has no row
+                    ([0, 1, 9, -1, -1], 2),       # node 9 does not exist
+                    ([0, 3, 1, -1, -1], 2),       # rows 1 then 0
+                    ([0, 1, 3, 4, 5], 5)):        # longer than max_depth
+        ref = both([paths[4], path], [4, a])
+        assert ref["status"].tolist() == [0, 4] and ref["path_rows"][1].tolist() == [0, -1, -1, -1, -1]   # SB_ERR_INVALID_TREE

@@ -281,6 +281,57 @@ def _scores_with_known_ranking(rng, n_rows, vocab):
     return scores, ranking
 
 
+def test_path_rows_hand_worked_two_block_tree():
+    """K = 4.  Block 1 (rows 0..3) starts at the root: row 0 proposes nodes 1, 2 (siblings), row 1 node 3 under node 1,
+    row 2 node 4, row 3 node 5 (the chain 1-3-4-5).  Block 2 (rows 4..7) starts at sibling 2: row 4 proposes nodes
+    6, 7 under 2, row 5 node 8 under 6.  A committed position keeps the row of its own draft forward (App. A.2),
+    and slot 0 of the row numbering is the last committed position."""
+    offs = [0, 9]
+    node_row = [-1, 0, 0, 1, 2, 3, 4, 4, 5]
+    cases = [([0, 1, 3, 4, 5], 4, [0, 1, 2, 3, 4]),          # the whole first chain: rows 0..3 -> slots 1..4
+             ([0, 2, 7, -1, -1], 2, [0, 1, 5, -1, -1]),     # sibling 2 shares row 0 with node 1; node 7 shares row 4
+             ([0, 2, 6, 8, -1], 3, [0, 1, 5, 6, -1]),
+             ([0, -1, -1, -1, -1], 0, [0, -1, -1, -1, -1])]  # nothing drafted was accepted
+    for path, a, want in cases:
+        r = oracle.path_rows(offs, node_row, [path], [a], 4)
+        assert r["status"].tolist() == [0]
+        assert r["path_rows"][0].tolist() == want
+    # the rows must increase along a path, a path node must exist and must have a row, a must fit
+    for path, a in (([0, 3, 1, -1, -1], 2), ([0, 9, -1, -1, -1], 1), ([0, 0, -1, -1, -1], 1), ([0, 1, 3, 4, 5], 5)):
+        r = oracle.path_rows(offs, node_row, [path], [a], 4)
+        assert r["status"].tolist() == [4] and r["path_rows"][0].tolist() == [0, -1, -1, -1, -1]
+
+
+def test_path_rows_equals_numpy_fancy_indexing_on_random_batches():
+    rng = W.rng_for(5150)
+    for _ in range(50):
+        B, md = int(rng.integers(1, 5)), int(rng.integers(1, 9))
+        n = rng.integers(md + 1, 40, size=B)
+        offs = np.concatenate([[0], np.cumsum(n)]).astype(np.int32)
+        row_begin = np.cumsum(np.concatenate([[0], n[:-1] + 3])).astype(np.int32)   # any first row per sequence
+        node_row = np.full(offs[-1], -1, np.int32)
+        paths, acc, want = [], [], []
+        for b in range(B):
+            # rows never decrease with the node id; siblings share a row
+            rows_b = np.sort(rng.integers(0, n[b] + 3, size=n[b] - 1))
+            node_row[offs[b] + 1:offs[b + 1]] = row_begin[b] + rows_b
+            distinct = np.unique(rows_b)
+            a = int(rng.integers(0, min(md, len(distinct)) + 1))
+            # one node from each of `a` different rows, in row order: the rows increase along the path
+            picked = np.sort(rng.choice(distinct, size=a, replace=False))
+            nodes = np.array([1 + int(rng.choice(np.flatnonzero(rows_b == r))) for r in picked], np.int64)
+            path = np.full(md + 1, -1, np.int32)
+            path[0] = 0
+            path[1:a + 1] = nodes
+            w = np.full(md + 1, -1, np.int32)
+            w[0] = 0
+            w[1:a + 1] = 1 + node_row[offs[b] + nodes] - row_begin[b]
+            paths.append(path), acc.append(a), want.append(w)
+        r = oracle.path_rows(offs, node_row, np.stack(paths), acc, md, row_begin=row_begin)
+        assert not r["status"].any()
+        np.testing.assert_array_equal(r["path_rows"], np.stack(want))
+
+
 def test_expand_hand_derived_examples(golden_dir):
     """The two printed branching maps on hand-worked blocks, incl. a width-0 bucket that ends a
     block, a second block level, and the node budget cutting a row."""
