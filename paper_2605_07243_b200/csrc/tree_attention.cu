@@ -354,9 +354,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
 // One warp per (node, head) row.
 // ----------------------------------------------------------------------------------------------
 
+// One 16-byte load per lane and chunk: a row takes D/8 lanes with bf16 partials, D/4 with fp32 ones, so a
+// warp holds one, two or four rows; every lane finds the row's reference maximum itself (the log-sum-exps are
+// a few broadcast loads) and then has eight chunks' loads in flight at a time, none of them waiting for a
+// weight: a chunk that saw no key for the row did not write its partial, so what was loaded for it is
+// dropped by a select instead of being skipped by a branch.
+template <int D, bool PB16>
+constexpr int merge_rows_per_cta() { return 8 * (32 / (D / (PB16 ? 8 : 4))); }
+
 template <int D, bool PB16>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
-  constexpr int E = D / 32;
+  constexpr int EPL = PB16 ? 8 : 4;  // elements per lane
+  constexpr int LPR = D / EPL;       // lanes per row
+  constexpr int RPW = 32 / LPR;      // rows per warp
+  constexpr int UN = 8;
   const int b = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Sequences whose lengths are bad still own their rows (zero-filled by the empty partials).
@@ -369,61 +380,70 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
                        o >= 0 && (long long)o + n_raw <= p.tb.total_nodes;
   if (!rows_ok) return;
   const int Hq = p.tb.n_q_heads;
-  const int rr = blockIdx.x * 8 + warp;
+  const int rr = (blockIdx.x * 8 + warp) * RPW + lane / LPR;
+  const int col = lane % LPR;
   if (rr >= (n_raw - q0) * Hq) return;
   const long long rows_all = (long long)p.total_q * Hq;
   const long long grow = (long long)q_off * Hq + rr;
   float M = -INFINITY;
-  for (int s = lane; s < p.outer; s += 32) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
+  for (int s = 0; s < p.outer; ++s) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
+  float acc[EPL];
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
-  float acc[E];
-#pragma unroll
-  for (int e = 0; e < E; ++e) acc[e] = 0.f;
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
   float denom = 0.f;
   if (M != -INFINITY) {
-    // no branch around the loads, so that several chunks' rows are in flight at once
-#pragma unroll 4
-    for (int s = 0; s < p.outer; ++s) {
-      const float ls = p.part_lse[s * rows_all + grow];
-      const bool live = ls != -INFINITY;  // a chunk that saw no key for this row did not write its O
-      const float w = live ? exp2f(ls - M) : 0.f;
-      denom += w;
-      float v[E];
-      if (PB16) {
-        const bf16* po = reinterpret_cast<const bf16*>(p.part_o) + (s * rows_all + grow) * D + lane * E;
-        uint32_t raw[E / 2];
-        if (E == 4) {
-          const uint2 t = live ? *reinterpret_cast<const uint2*>(po) : make_uint2(0u, 0u);
-          raw[0] = t.x;
-          raw[E / 2 - 1] = t.y;
-        } else {
-          raw[0] = live ? *reinterpret_cast<const uint32_t*>(po) : 0u;
-        }
+    for (int s0 = 0; s0 < p.outer; s0 += UN) {
+      uint4 raw[UN];
+      float w[UN];
 #pragma unroll
-        for (int e = 0; e < E / 2; ++e) {
-          v[2 * e] = __uint_as_float(raw[e] << 16);
-          v[2 * e + 1] = __uint_as_float(raw[e] & 0xffff0000u);
-        }
-      } else {
-        const float* po = p.part_o + (s * rows_all + grow) * D + lane * E;
-        if (E == 4) {
-          const float4 t = live ? *reinterpret_cast<const float4*>(po) : make_float4(0.f, 0.f, 0.f, 0.f);
-          v[0] = t.x, v[1] = t.y, v[E - 2] = t.z, v[E - 1] = t.w;
-        } else {
-          const float2 t = live ? *reinterpret_cast<const float2*>(po) : make_float2(0.f, 0.f);
-          v[0] = t.x, v[1] = t.y;
+      for (int u = 0; u < UN; ++u) {
+        const int s = s0 + u;
+        if (s < p.outer) {
+          const char* src = reinterpret_cast<const char*>(p.part_o) +
+                            ((s * rows_all + grow) * D + col * EPL) * (PB16 ? 2 : 4);
+          raw[u] = *reinterpret_cast<const uint4*>(src);
         }
       }
 #pragma unroll
-      for (int e = 0; e < E; ++e) acc[e] += w * v[e];
+      for (int u = 0; u < UN; ++u) {
+        const int s = s0 + u;
+        const float ls = s < p.outer ? p.part_lse[s * rows_all + grow] : -INFINITY;
+        w[u] = ls != -INFINITY ? exp2f(ls - M) : 0.f;
+        denom += w[u];
+      }
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        if (s0 + u >= p.outer) break;
+        const uint32_t q4[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+        const bool live = w[u] != 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (PB16) {
+            acc[2 * e] += live ? w[u] * __uint_as_float(q4[e] << 16) : 0.f;
+            acc[2 * e + 1] += live ? w[u] * __uint_as_float(q4[e] & 0xffff0000u) : 0.f;
+          } else {
+            acc[e] += live ? w[u] * __uint_as_float(q4[e]) : 0.f;
+          }
+        }
+      }
     }
   }
   const float inv = denom > 0.f ? 1.f / denom : 0.f;
-  bf16* orow = p.out + grow * D + lane * E;
-#pragma unroll
-  for (int e = 0; e < E; ++e) orow[e] = __float2bfloat16(acc[e] * inv);
-  if (p.lse && lane == 0) p.lse[grow] = denom > 0.f ? (M + log2f(denom)) * kLn2 : 0.f;
+  bf16* orow = p.out + grow * D + col * EPL;
+  if (PB16) {
+    uint4 o4;
+    o4.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+    o4.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+    o4.z = pack_bf16(acc[EPL - 4] * inv, acc[EPL - 3] * inv);
+    o4.w = pack_bf16(acc[EPL - 2] * inv, acc[EPL - 1] * inv);
+    *reinterpret_cast<uint4*>(orow) = o4;
+  } else {
+    uint2 o2;
+    o2.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+    o2.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+    *reinterpret_cast<uint2*>(orow) = o2;
+  }
+  if (p.lse && col == 0) p.lse[grow] = denom > 0.f ? (M + log2f(denom)) * kLn2 : 0.f;
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -752,13 +772,14 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   else if (impl == IMPL_TC) st = launch_attn_tc(p, grid, plan.cluster, cs);
   else st = D == 64 ? launch_attn_mma<64>(p, grid, plan.cluster, cs) : launch_attn_mma<128>(p, grid, plan.cluster, cs);
   if (st != SB_OK || plan.outer == 1) return st;
-  dim3 mgrid(ceil_div(tb->max_nodes * tb->n_q_heads, 8), tb->batch);
+  const int rows_max = tb->max_nodes * tb->n_q_heads;
+  auto mgrid = [&](int rows_per_cta) { return dim3(ceil_div(rows_max, rows_per_cta), tb->batch); };
   if (p.part_bf16) {
-    if (D == 64) attn_merge_kernel<64, true><<<mgrid, 256, 0, cs>>>(p);
-    else attn_merge_kernel<128, true><<<mgrid, 256, 0, cs>>>(p);
+    if (D == 64) attn_merge_kernel<64, true><<<mgrid(merge_rows_per_cta<64, true>()), 256, 0, cs>>>(p);
+    else attn_merge_kernel<128, true><<<mgrid(merge_rows_per_cta<128, true>()), 256, 0, cs>>>(p);
   } else {
-    if (D == 64) attn_merge_kernel<64, false><<<mgrid, 256, 0, cs>>>(p);
-    else attn_merge_kernel<128, false><<<mgrid, 256, 0, cs>>>(p);
+    if (D == 64) attn_merge_kernel<64, false><<<mgrid(merge_rows_per_cta<64, false>()), 256, 0, cs>>>(p);
+    else attn_merge_kernel<128, false><<<mgrid(merge_rows_per_cta<128, false>()), 256, 0, cs>>>(p);
   }
   return launch_check();
 }
