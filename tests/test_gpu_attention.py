@@ -349,3 +349,18 @@ def test_settled_flags_give_the_same_bits():
             for a, b in zip(plain, flagged):
                 np.testing.assert_array_equal(a, b)
         assert (plain[2] == 0).all()
+
+
+@pytest.mark.parametrize("page_size", [0, 64])
+@pytest.mark.parametrize("num_splits", [0, 1, 3])
+def test_empty_sequences_inside_a_batch(page_size, num_splits, monkeypatch):
+    """Sequences without any tree node (and one whose query range is empty) between ordinary ones: they own no
+    output row, report status 0 and leave their neighbours' rows alone -- on the one-tile and the two-tile kernel."""
+    rng = W.rng_for(77 + page_size + num_splits)
+    none = np.zeros(0, np.int32)
+    parents = [none, W.random_tree(rng, 70, 6), none, W.chain_tree(9), W.random_tree(rng, 20, 4), none]
+    case = W.make_attn_case(rng, parents=parents, prefix_lens=[40, 300, 0, 0, 129, 5], n_q_heads=8, n_kv_heads=2,
+                            head_dim=128, page_size=page_size, q_node_begin=[0, 0, 0, 3, 20, 0])
+    for two in ("0", "1"):
+        monkeypatch.setenv("SB_ATTN_TWO_TILES", two)
+        check_attention(case, f"empty sequences, page {page_size}, splits {num_splits}, two tiles {two}", num_splits=num_splits)

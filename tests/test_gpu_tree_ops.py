@@ -829,3 +829,39 @@ def test_path_rows_against_the_oracle_and_error_cases():
                     ([0, 1, 3, 4, 5], 5)):        # longer than max_depth
         ref = both([paths[4], path], [4, a])
         assert ref["status"].tolist() == [0, 4] and ref["path_rows"][1].tolist() == [0, -1, -1, -1, -1]   # SB_ERR_INVALID_TREE
+
+
+def test_accept_and_compact_with_empty_sequences_in_the_batch():
+    """A sequence without nodes has no root: acceptance reports an invalid tree for it (accept_len 0, -1 elsewhere)
+    and compaction leaves its cache and length alone, while the neighbours are processed as usual."""
+    require_gpu()
+    rng = W.rng_for(78)
+    none = np.zeros(0, np.int32)
+    parents = [W.random_tree(rng, 12, 4), none, W.chain_tree(6), none]
+    total = sum(len(p) for p in parents)
+    offs = np.concatenate([[0], np.cumsum([len(p) for p in parents])]).astype(np.int32)
+    logits = rng.standard_normal((total, 97), dtype=np.float32)
+    tok = rng.integers(0, 97, total).astype(np.int32)
+    par = np.concatenate(parents).astype(np.int32)
+    for c in range(13, 18):                               # the chain accepts its first three tokens
+        if c - 12 <= 3:
+            logits[c - 1, tok[c]] = 50.0
+    case = W.VerifyCase(logits, tok, offs, par, 5, None, None, None)
+    got = _check_accept(case)
+    assert list(got["status"]) == [0, 4, 0, 4] and got["accept_len"][2] == 3
+    attn = W.make_attn_case(rng, parents=parents, prefix_lens=[10, 4, 33, 0], n_q_heads=4, n_kv_heads=2, head_dim=64)
+    tb, _q, _kw = dev.attention_args(attn)
+    k0 = attn.k.copy()
+    new_len, st = sb.sb_kv_compact(tb, 1, int(attn.k.size), torch.from_numpy(got["path_nodes"]).cuda(),
+                                   torch.from_numpy(got["accept_len"]).cuda(), 5)
+    torch.cuda.synchronize()
+    ref_c, ref_len, ref_st = oracle.kv_compact(
+        n_kv_heads=2, head_dim=64, cache=k0.reshape(-1), n_layers=1, layer_stride_elems=int(attn.k.size),
+        kv_capacity=attn.kv_capacity, prefix_len=attn.prefix_len, node_offsets=offs, path_nodes=got["path_nodes"],
+        accept_len=got["accept_len"], max_depth=5)
+    np.testing.assert_array_equal(st.cpu().numpy(), ref_st)
+    np.testing.assert_array_equal(new_len.cpu().numpy(), ref_len)
+    got_k = tb.k_cache.view(torch.int16).cpu().numpy().view(np.uint16).reshape(len(parents), -1)
+    row = 2 * 64
+    for b in range(len(parents)):
+        np.testing.assert_array_equal(got_k[b, :ref_len[b] * row], ref_c.reshape(len(parents), -1)[b, :ref_len[b] * row])
