@@ -7,6 +7,7 @@ if the library is missing or no CUDA device is present these calls raise.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes as C
 import os
 from dataclasses import dataclass
@@ -50,14 +51,7 @@ def lib_path() -> str:
     return _build.LIB
 
 
-def load(build_if_missing: bool = True):
-    """Load libspecblock.so (building it in-tree with nvcc when it is absent or stale)."""
-    global _lib
-    if _lib is not None:
-        return _lib
-    path = _build.build() if build_if_missing else _build.LIB
-    if not os.path.exists(path):
-        raise RuntimeError("libspecblock.so is not built: run python -m paper_2605_07243_b200.build")
+def _open(path: str):
     lib = C.CDLL(path)
     lib.sb_status_string.restype = C.c_char_p
     lib.sb_version.restype = C.c_int32
@@ -71,8 +65,40 @@ def load(build_if_missing: bool = True):
                  "sb_verify_accept_static", "sb_kv_compact", "sb_path_rows", "sb_rank_features", "sb_verifier_signal",
                  "sb_verify_sample", "sb_shift_project", "sb_fuse_project", "sb_tree_expand_features"):
         getattr(lib, name).restype = C.c_int
-    _lib = lib
     return lib
+
+
+def load(build_if_missing: bool = True):
+    """Load libspecblock.so (building it in-tree with nvcc when it is absent or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build() if build_if_missing else _build.LIB
+    if not os.path.exists(path):
+        raise RuntimeError("libspecblock.so is not built: run python -m paper_2605_07243_b200.build")
+    _lib = _open(path)
+    return _lib
+
+
+_variants = {}
+
+
+@contextlib.contextmanager
+def build_variant(name: str):
+    """Inside the block every call of this module goes to another build of the same sources:
+    "test" (libspecblock_test.so: the mma.sync and one-warp-per-row attention kernels as independent
+    cross-checks, the environment switches SB_ATTN_IMPL / SB_ATTN_TWO_TILES / SB_ATTN_MAX_CLUSTER /
+    SB_NO_PDL / SB_DEBUG, and the wait-expiry kernel) or "checked" (libspecblock_checked.so: every
+    computed index verified before use).  For tests; the library proper is what load() returns."""
+    global _lib
+    load()
+    if name not in _variants:
+        _variants[name] = _open(_build.build(variant=name))
+    saved, _lib = _lib, _variants[name]
+    try:
+        yield _lib
+    finally:
+        _lib = saved
 
 
 EXPORTED = ("sb_tree_ancestors", "sb_tree_attention", "sb_tree_attention_workspace_bytes",
@@ -466,3 +492,33 @@ def sb_tree_expand(scores, block_k, bucket, bmap, start_parent, node_budget, tre
         _check(lib.sb_tree_expand_features(*head, _ptr(features, torch.float32), _ptr(child_row, torch.int32),
                                            C.c_int32(row_base), *tail), "sb_tree_expand_features")
     return topk_tok, topk_val, status
+
+
+# ---- hooks of the test and checked builds (include/specblock_test.h); use inside build_variant(...) ----
+
+def sb_test_wait_expires(limit_ns: int):
+    """Test build: lets a bounded device wait run out.  -> (status int32[1], elapsed_ns int64[2]) tensors."""
+    lib = load()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    elapsed = torch.zeros(2, dtype=torch.int64, device="cuda")
+    lib.sb_test_wait_expires.restype = C.c_int
+    _check(lib.sb_test_wait_expires(C.c_int64(limit_ns), _ptr(status), _ptr(elapsed), _stream()), "sb_test_wait_expires")
+    return status, elapsed
+
+
+def sb_checked_violations() -> int:
+    """Checked build: accesses refused since the last call (synchronises the device, clears the counter)."""
+    lib = load()
+    lib.sb_checked_violations.restype = C.c_int
+    n = C.c_int64(-1)
+    _check(lib.sb_checked_violations(C.byref(n)), "sb_checked_violations")
+    return int(n.value)
+
+
+def sb_checked_selftest():
+    """Checked build: one refused access on purpose.  -> status int32[2] tensor."""
+    lib = load()
+    lib.sb_checked_selftest.restype = C.c_int
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    _check(lib.sb_checked_selftest(_ptr(status), _stream()), "sb_checked_selftest")
+    return status

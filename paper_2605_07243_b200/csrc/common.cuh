@@ -4,6 +4,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
+
+#include <atomic>
 
 #include "../../include/specblock.h"
 
@@ -18,6 +21,55 @@ inline sb_status launch_check() {
 }
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Experiment switches exist only in the test build (-DSB_TEST_KERNELS); the library proper reads no
+// environment variable, on the launch path or anywhere else.
+#ifdef SB_TEST_KERNELS
+inline const char* test_knob(const char* name) { return getenv(name); }
+#else
+inline const char* test_knob(const char*) { return nullptr; }
+#endif
+
+// Kernel attributes (dynamic shared memory, cluster size) and occupancy figures belong to a device,
+// not to the process: caches of them are arrays indexed by the current device.  -1: no usable device.
+constexpr int kMaxDevices = 64;
+inline int device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return -1;
+  }
+  return dev;
+}
+// One-time set-up of the current device (cudaFuncSetAttribute and the like).  `fn` returns true on
+// success and must be idempotent: two host threads that meet here for the first time may both run it.
+struct PerDeviceOnce {
+  std::atomic<int> done[kMaxDevices];
+  template <typename F>
+  bool run(F fn) {
+    const int dev = device_slot();
+    if (dev < 0) return false;
+    if (done[dev].load(std::memory_order_acquire)) return true;
+    if (!fn()) return false;
+    done[dev].store(1, std::memory_order_release);
+    return true;
+  }
+};
+// A small integer fact of the current device, computed on first use (-1 = not known yet).
+struct PerDeviceInt {
+  std::atomic<int> value_plus_1[kMaxDevices];  // zero-initialised: 0 = unknown
+  template <typename F>
+  int get(F compute, int fallback) {
+    const int dev = device_slot();
+    if (dev < 0) return fallback;
+    int v = value_plus_1[dev].load(std::memory_order_acquire);
+    if (v == 0) {
+      v = compute() + 1;
+      value_plus_1[dev].store(v, std::memory_order_release);
+    }
+    return v - 1;
+  }
+};
 
 // Programmatic dependent launch.  A kernel started with launch_dependent() may begin while its
 // predecessor in the stream is still running; it must execute pdl_wait() before it reads anything
@@ -43,6 +95,30 @@ inline sb_status launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bloc
     return SB_ERR_CUDA;
   }
   return launch_check();
+}
+
+// Checked build (-DSB_CHECKED, libspecblock_checked.so): every index a kernel computes from device
+// data -- page ids, cache slots, query/output rows, workspace offsets -- is verified against the extent
+// of what it indexes right before the access.  A violation sets SB_ERR_BOUNDS in the call's status
+// word and the access is skipped.  The library proper compiles the test away.  (This pool has no
+// compute-sanitizer; this build plus canary-padded buffers in the tests stand in for it.)
+#ifdef SB_CHECKED
+extern __device__ unsigned long long g_checked_violations;  // api.cu; read and cleared by sb_checked_violations()
+__device__ inline bool checked_access(long long idx, long long limit, int* status_word) {
+  if (idx >= 0 && idx < limit) return true;
+  atomicAdd(&g_checked_violations, 1ull);
+  if (status_word) atomicMax(status_word, (int)SB_ERR_BOUNDS);  // a kernel's own final status may overwrite this
+  return false;
+}
+#define SB_CHECKED_ACCESS(idx, limit, status_word) ::sb::checked_access((long long)(idx), (long long)(limit), (status_word))
+#else
+#define SB_CHECKED_ACCESS(idx, limit, status_word) true
+#endif
+
+// Elements of one layer of a K or V cache.
+__host__ __device__ inline long long kv_cache_elems(const sb_tree_batch& tb) {
+  const long long rows = tb.page_size == 0 ? (long long)tb.batch * tb.kv_capacity : (long long)tb.num_pages * tb.page_size;
+  return rows * tb.n_kv_heads * tb.head_dim;
 }
 
 // Per-sequence facts every CTA of a sequence derives identically from device data.

@@ -71,14 +71,18 @@ __global__ void __launch_bounds__(COMPACT_THREADS) kv_compact_kernel(const sb_tr
 #pragma unroll
     for (int t = 0; t < COMPACT_GROUP; ++t) {
       const int j = j0 + t;
-      if (j <= a)
-        regs[t] = *reinterpret_cast<const uint4*>(cache + kv_row_elem_offset(tb, b, P + s_path[j]) + u * 8);
+      if (j <= a) {
+        const long long src = kv_row_elem_offset(tb, b, P + s_path[j]) + u * 8;
+        if (SB_CHECKED_ACCESS(src + 7, kv_cache_elems(tb), &status[b])) regs[t] = *reinterpret_cast<const uint4*>(cache + src);
+      }
     }
 #pragma unroll
     for (int t = 0; t < COMPACT_GROUP; ++t) {
       const int j = j0 + t;
-      if (j <= a && s_path[j] != j)
-        *reinterpret_cast<uint4*>(cache + kv_row_elem_offset(tb, b, P + j) + u * 8) = regs[t];
+      if (j <= a && s_path[j] != j) {
+        const long long dst = kv_row_elem_offset(tb, b, P + j) + u * 8;
+        if (SB_CHECKED_ACCESS(dst + 7, kv_cache_elems(tb), &status[b])) *reinterpret_cast<uint4*>(cache + dst) = regs[t];
+      }
     }
   }
 }

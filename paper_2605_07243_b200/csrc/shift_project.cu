@@ -217,8 +217,8 @@ static bool shift_plan(int n_rows, int d, int d_out, int segments, ShiftPlan* pl
   const bool two_per_sm = stage <= 24 * 1024;
   int cta_target = two_per_sm ? 320 : 160;
   size_t budget = two_per_sm ? 110 * 1024 : 200 * 1024;
-  if (const char* e = getenv("SB_SHIFT_CTAS")) cta_target = atoi(e);
-  if (const char* e = getenv("SB_SHIFT_SMEM_KB")) budget = (size_t)atoi(e) * 1024;
+  if (const char* e = test_knob("SB_SHIFT_CTAS")) cta_target = atoi(e);
+  if (const char* e = test_knob("SB_SHIFT_SMEM_KB")) budget = (size_t)atoi(e) * 1024;
   int ks = 1;
   // split_like: choose the K split as a problem of that many segments would (the same partial sums, hence the
   // same bits, whether or not a cached segment is left out)
@@ -251,14 +251,13 @@ static bool make_2d_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint6
 // Launches the GEMM of a plan (programmatic dependent of whatever precedes it in the stream).
 static sb_status launch_shift_gemm(const ShiftPlan& pl, const CUtensorMap& wmap, const CUtensorMap& xmap, int n_cols,
                                    int d, int d_out, int x_seg_rows, float* part, int* err_word, cudaStream_t cs) {
-  static bool prepared = false;
-  if (!prepared) {
-    if (cudaFuncSetAttribute(shift_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
-      cudaGetLastError();
-      return SB_ERR_CUDA;
-    }
-    prepared = true;
-  }
+  static PerDeviceOnce once;
+  if (!once.run([]() {
+        const bool ok = cudaFuncSetAttribute(shift_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) == cudaSuccess;
+        if (!ok) cudaGetLastError();
+        return ok;
+      }))
+    return SB_ERR_CUDA;
   if (pl.smem > 200 * 1024) return SB_ERR_UNSUPPORTED;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(d_out / SG_BM, pl.halves * pl.ksplit);
@@ -269,7 +268,7 @@ static sb_status launch_shift_gemm(const ShiftPlan& pl, const CUtensorMap& wmap,
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the kernel orders itself (pdl_wait)
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = getenv("SB_NO_PDL") ? 0 : 1;
+  cfg.numAttrs = test_knob("SB_NO_PDL") ? 0 : 1;
   if (cudaLaunchKernelEx(&cfg, shift_gemm_kernel, wmap, xmap, n_cols, pl.r_pad, d, d_out, pl.ksplit, pl.k_per,
                          pl.tmem_cols, pl.stages, x_seg_rows, part, err_word) != cudaSuccess) {
     cudaGetLastError();

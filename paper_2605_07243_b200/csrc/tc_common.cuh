@@ -25,7 +25,9 @@ __device__ inline void mbar_arrive(uint64_t* bar) {
 // The first probe (which the hardware already holds for a while) is inline; the polling loop with its
 // clock and abort checks is one shared out-of-line copy, so that the dozens of waits of a kernel cost
 // a few instructions each in its code.
-static __device__ __noinline__ bool mbar_wait_poll(uint32_t addr, uint32_t parity, volatile int* abort_flag) {
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // two seconds
+static __device__ __noinline__ bool mbar_wait_poll(uint32_t addr, uint32_t parity, volatile int* abort_flag,
+                                                   unsigned long long limit_ns = kWaitLimitNs) {
   unsigned long long t0 = 0;
   for (int it = 0;; ++it) {
     uint32_t ok;
@@ -40,7 +42,7 @@ static __device__ __noinline__ bool mbar_wait_poll(uint32_t addr, uint32_t parit
       unsigned long long now;
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
       if (t0 == 0) t0 = now;
-      else if (now - t0 > 2000000000ull) break;
+      else if (now - t0 > limit_ns) break;
     }
   }
   *abort_flag = 1;

@@ -11,12 +11,15 @@
 // cluster writes one partial and a second kernel merges the clusters' (out, log-sum-exp) pairs.
 //
 // Kernels in this file
-//   attn_simple_kernel : one warp per query row, fp32 FMA.  Slow, shape-agnostic check path
-//                        (environment SB_ATTN_IMPL=simple selects it).
+//   attn_merge_kernel  : log-sum-exp merge of the clusters' partials (only beyond one cluster of chunks).
+//   The attention itself runs on the tcgen05/TMEM kernels of tree_attention_tc.cu / tree_attention_tc2.cu;
+//   the library has this one backend and reads no environment variable.
+// Only in the test build (-DSB_TEST_KERNELS, libspecblock_test.so), as independent cross-checks of the
+// tcgen05 kernels and as switches that force a kernel variant onto a shape the planner would not give it:
+//   attn_simple_kernel : one warp per query row, fp32 FMA (SB_ATTN_IMPL=simple).
 //   attn_mma_kernel    : flash-decode with bf16 mma.sync (m16n8k16), fp32 accumulate, 3-stage cp.async
-//                        K/V pipeline in XOR-swizzled shared memory (SB_ATTN_IMPL=mma selects it).
-//   (default)          : the tcgen05/TMEM kernel in tree_attention_tc.cu.
-//   attn_merge_kernel  : log-sum-exp merge of the clusters' partials (only beyond 8 chunks).
+//                        K/V pipeline in XOR-swizzled shared memory (SB_ATTN_IMPL=mma).
+//   SB_ATTN_TWO_TILES, SB_ATTN_MAX_CLUSTER, SB_NO_PDL, SB_DEBUG.
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -30,6 +33,9 @@ sb_status launch_attn_tc(const AttnParams& p, dim3 grid, int cluster, cudaStream
 int attn_tc_max_active_clusters(int D, int cluster);
 sb_status launch_attn_tc2(const AttnParams& p, dim3 grid, cudaStream_t cs);
 
+constexpr int BM = 128;       // query rows per CTA tile
+
+#ifdef SB_TEST_KERNELS
 // ----------------------------------------------------------------------------------------------
 // Simple kernel: one warp per (node, head) row.
 // ----------------------------------------------------------------------------------------------
@@ -92,8 +98,7 @@ __global__ void __launch_bounds__(256) attn_simple_kernel(const AttnParams p) {
 // Tensor-core (mma.sync) flash-decode kernel.
 // ----------------------------------------------------------------------------------------------
 
-constexpr int BM = 128;       // query rows per CTA (8 warps x 16 rows)
-constexpr int BN = 64;        // keys per pipeline stage
+constexpr int BN = 64;        // keys per pipeline stage (BM = 8 warps x 16 rows)
 constexpr int NTHREADS = 256;
 constexpr int STAGES = 3;
 
@@ -349,6 +354,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_mma_kernel(const AttnParams 
   merge_reduce_and_store<D, BM>(p, mb, S, crank, split / S, row0, rows_total, g, si.q_off, rows_all, tid, NTHREADS);
 }
 
+#endif  // SB_TEST_KERNELS
+
 // ----------------------------------------------------------------------------------------------
 // Merge of split partials: out = sum_s w_s out_s, w_s = 2^(lse_s - M) / sum_s 2^(lse_s - M).
 // One warp per (node, head) row.
@@ -385,6 +392,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
   if (rr >= (n_raw - q0) * Hq) return;
   const long long rows_all = (long long)p.total_q * Hq;
   const long long grow = (long long)q_off * Hq + rr;
+  if (!SB_CHECKED_ACCESS(grow, rows_all, &p.status[b])) return;
   float M = -INFINITY;
   for (int s = 0; s < p.outer; ++s) M = fmaxf(M, p.part_lse[s * rows_all + grow]);
   float acc[EPL];
@@ -451,14 +459,16 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnParams p) {
 // ----------------------------------------------------------------------------------------------
 
 static int num_sms() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
+  static PerDeviceInt cache;
+  return cache.get([]() {
+    int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+      cudaGetLastError();
       sms = 148;
-  }
-  return sms;
+    }
+    return sms;
+  }, 148);
 }
 
 static sb_status check_batch(const sb_tree_batch* tb) {
@@ -483,20 +493,21 @@ static sb_status check_batch(const sb_tree_batch* tb) {
 
 constexpr int kMaxCluster = 8;  // portable thread-block cluster size
 
+
 struct SplitPlan {
   int cluster;     // chunk-CTAs merged through distributed shared memory
   int outer;       // clusters per (sequence, KV head, row tile)
   bool two_tiles;  // the two-tiles-per-CTA tcgen05 kernel (no clusters: outer = chunks)
 };
 
-// How many clusters of `cluster` CTAs of the attention kernel can be resident at once (0 when the
+#ifdef SB_TEST_KERNELS
+// How many clusters of `cluster` CTAs of the mma.sync kernel can be resident at once (0 when the
 // query fails).  Cached per (head_dim, cluster size); 8-CTA clusters of full-SM CTAs do not tile
 // the 148 SMs evenly, so this is what decides whether a grid runs as one wave.
 static int max_active_clusters(int D, int cluster) {
-  static int cache[2][kMaxCluster + 1];
-  static bool have[2][kMaxCluster + 1];
+  static PerDeviceInt cache[2][kMaxCluster + 1];
   const int di = D == 64 ? 0 : 1;
-  if (!have[di][cluster]) {
+  return cache[di][cluster].get([&]() {
     const size_t smem = 2560 + (size_t)BM * D * 2 + 2 * (size_t)STAGES * BN * D * 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cluster * 64, 1, 1);
@@ -519,11 +530,14 @@ static int max_active_clusters(int D, int cluster) {
       e = cudaOccupancyMaxActiveClusters(&n, attn_mma_kernel<128>, &cfg);
     }
     if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
-    cache[di][cluster] = n;
-    have[di][cluster] = true;
-  }
-  return cache[di][cluster];
+    return n;
+  }, 0);
 }
+constexpr int kCheckGranule = BN;
+#else
+static int max_active_clusters(int, int) { return 0; }
+constexpr int kCheckGranule = 64;
+#endif
 
 // `oversubscribed`: the grid has several waves of CTAs anyway.  Then clusters of 2 are preferred:
 // clusters of 8 full-SM CTAs keep only 120 of the 148 SMs busy, clusters of 2 all of them, and the
@@ -538,7 +552,7 @@ static SplitPlan plan_for(int s, bool oversubscribed, bool wide = false) {
   sp.cluster = 1;
   const int climit = wide ? kMaxClusterTc : kMaxCluster;
   int cmax = oversubscribed ? 2 : climit;
-  if (const char* e = getenv("SB_ATTN_MAX_CLUSTER")) {  // experiment knob
+  if (const char* e = test_knob("SB_ATTN_MAX_CLUSTER")) {
     const int v = atoi(e);
     if (v >= 1 && v <= climit) cmax = v;
   }
@@ -560,7 +574,7 @@ static int max_row_tiles(const sb_tree_batch* tb, int total_q) {
 }
 
 static AttnImpl attn_impl() {
-  const char* impl = getenv("SB_ATTN_IMPL");
+  const char* impl = test_knob("SB_ATTN_IMPL");
   if (impl && strcmp(impl, "simple") == 0) return IMPL_SIMPLE;
   if (impl && strcmp(impl, "mma") == 0) return IMPL_MMA;
   return IMPL_TC;
@@ -572,7 +586,7 @@ static AttnImpl attn_impl() {
 // clusters of the largest divisor <= 8.  `granule` is the kernel's key-block size.
 static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_splits, AttnImpl impl) {
   const int row_tiles = max_row_tiles(tb, total_q);
-  const int granule = impl == IMPL_TC ? 128 : BN;
+  const int granule = impl == IMPL_TC ? 128 : kCheckGranule;
   const int max_blocks = ceil_div(tb->max_kv_len, granule);
   const long long base = (long long)tb->batch * tb->n_kv_heads * row_tiles;
   const int sms = num_sms();
@@ -581,7 +595,7 @@ static SplitPlan choose_splits(const sb_tree_batch* tb, int total_q, int num_spl
   // (With three tiles the second CTA of a KV head holds a single one; still faster than three one-tile
   // CTAs on the ragged batch of config 4: 131 us against 154 us.)
   bool two_tiles = impl == IMPL_TC && row_tiles >= 2 && base > sms;
-  if (const char* e = getenv("SB_ATTN_TWO_TILES")) two_tiles = impl == IMPL_TC && row_tiles >= 2 && atoi(e) != 0;
+  if (const char* e = test_knob("SB_ATTN_TWO_TILES")) two_tiles = impl == IMPL_TC && row_tiles >= 2 && atoi(e) != 0;
   if (two_tiles) {
     SplitPlan sp;
     sp.two_tiles = true;
@@ -665,15 +679,17 @@ static size_t workspace_bytes_for(const sb_tree_batch* tb, int total_q, int oute
   return ((o + 255) & ~(size_t)255) + ((l + 255) & ~(size_t)255);
 }
 
+#ifdef SB_TEST_KERNELS
 template <int D>
 static sb_status launch_attn_mma(const AttnParams& p, dim3 grid, int cluster, cudaStream_t cs) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_mma_smem_bytes<D>()) != cudaSuccess)
-      return SB_ERR_CUDA;
-    attr_set = true;
-  }
+  static PerDeviceOnce once;
+  if (!once.run([]() {
+        const bool ok = cudaFuncSetAttribute(attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)attn_mma_smem_bytes<D>()) == cudaSuccess;
+        if (!ok) cudaGetLastError();
+        return ok;
+      }))
+    return SB_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(NTHREADS);
@@ -686,7 +702,7 @@ static sb_status launch_attn_mma(const AttnParams& p, dim3 grid, int cluster, cu
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (getenv("SB_DEBUG")) {
+  if (test_knob("SB_DEBUG")) {
     int max_clusters = -1;
     cudaOccupancyMaxActiveClusters(&max_clusters, attn_mma_kernel<D>, &cfg);
     fprintf(stderr, "[sb] attn_mma<%d> grid (%u,%u,%u) cluster %d outer %d: max active clusters %d\n", D, grid.x,
@@ -698,6 +714,7 @@ static sb_status launch_attn_mma(const AttnParams& p, dim3 grid, int cluster, cu
   }
   return launch_check();
 }
+#endif  // SB_TEST_KERNELS
 
 }  // namespace sb
 
@@ -738,6 +755,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   p.part_lse = nullptr;
 
   const AttnImpl impl = attn_impl();
+#ifdef SB_TEST_KERNELS
   if (impl == IMPL_SIMPLE) {
     p.num_splits = 1;
     p.outer = 1;
@@ -747,6 +765,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
     else attn_simple_kernel<128><<<grid, 256, 0, cs>>>(p);
     return launch_check();
   }
+#endif
 
   const SplitPlan plan = choose_splits(tb, total_q, num_splits, impl);
   p.num_splits = plan.cluster * plan.outer;
@@ -770,7 +789,11 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
   if (grid.y > 65535 || grid.z > 65535) return SB_ERR_UNSUPPORTED;
   if (plan.two_tiles) st = launch_attn_tc2(p, grid, cs);
   else if (impl == IMPL_TC) st = launch_attn_tc(p, grid, plan.cluster, cs);
+#ifdef SB_TEST_KERNELS
   else st = D == 64 ? launch_attn_mma<64>(p, grid, plan.cluster, cs) : launch_attn_mma<128>(p, grid, plan.cluster, cs);
+#else
+  else st = SB_ERR_UNSUPPORTED;
+#endif
   if (st != SB_OK || plan.outer == 1) return st;
   const int rows_max = tb->max_nodes * tb->n_q_heads;
   auto mgrid = [&](int rows_per_cta) { return dim3(ceil_div(rows_max, rows_per_cta), tb->batch); };

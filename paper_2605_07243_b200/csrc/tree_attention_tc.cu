@@ -184,7 +184,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     const int pieces = ceil_div(nj, box_rows);
 #pragma unroll 1
     for (int i = 0; i < MAX_PIECES; ++i)
-      if (i < pieces) pg[i] = p.tb.page_table[(long long)b * p.tb.max_pages + (k0 + i * box_rows) / (FAST ? 1 : page_size)];
+      if (i < pieces) {
+        const int lp = (k0 + i * box_rows) / (FAST ? 1 : page_size);
+        pg[i] = SB_CHECKED_ACCESS(lp, p.tb.max_pages, &p.status[b]) ? p.tb.page_table[(long long)b * p.tb.max_pages + lp] : 0;
+      }
   };
   auto issue_pieces = [&](int j, const int (&pg)[MAX_PIECES], const CUtensorMap* map, uint32_t stage_addr,
                           uint64_t* bar) {
@@ -278,7 +281,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
         const int node_l = valid ? R / G : 0;
         const int hh = valid ? R - node_l * G : 0;
         const long long off = ((long long)(si.q_off + node_l) * Hq + g * G + hh) * D + ch * 8;
-        cp_async_16_tc(qd + sw128_chunk_off(r, ch, TC_BM), p.q + (valid ? off : 0), valid ? 16 : 0);
+        const bool q_ok = valid && SB_CHECKED_ACCESS(off + 7, (long long)p.total_q * Hq * D, &p.status[b]);
+        cp_async_16_tc(qd + sw128_chunk_off(r, ch, TC_BM), p.q + (q_ok ? off : 0), q_ok ? 16 : 0);
       }
       asm volatile("cp.async.commit_group;\n" ::);
       asm volatile("cp.async.wait_group 0;\n" ::: "memory");
@@ -611,7 +615,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
       const int node_l = Rr / G, hh = Rr - node_l * G;
       const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
       const float lse2 = Lsum > 0.f ? M + log2f(Lsum) : -INFINITY;
-      if (has_cols) {
+      if (has_cols && SB_CHECKED_ACCESS(grow, rows_all, &p.status[b])) {
         if (FAST || p.outer == 1) {
           uint4 packed;
           packed.x = pack_bf16(acc[0] * inv, acc[1] * inv);
@@ -657,14 +661,14 @@ static cudaLaunchConfig_t tc_config(dim3 grid, int cluster, cudaStream_t cs, cud
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = getenv("SB_NO_PDL") ? 1 : 2;
+  cfg.numAttrs = test_knob("SB_NO_PDL") ? 1 : 2;
   return cfg;
 }
 
 template <int D>
 static bool tc_prepare() {
-  static bool done = false;
-  if (!done) {
+  static PerDeviceOnce once;  // kernel attributes belong to a device: a process may drive several
+  return once.run([]() {
     bool all = true;
 #define SB_TC_PREPARE(cs_)                                                                                       \
   all = all && cudaFuncSetAttribute(attn_tc_kernel<D, cs_>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
@@ -676,21 +680,16 @@ static bool tc_prepare() {
     all = all && cudaFuncSetAttribute(attn_tc_kernel<D, 0>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
     all = all && cudaFuncSetAttribute(attn_tc_kernel<D, 9>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
     all = all && cudaFuncSetAttribute(attn_tc_kernel<D, 10>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
-    if (!all) {
-      cudaGetLastError();
-      return false;
-    }
-    done = true;
-  }
-  return true;
+    if (!all) cudaGetLastError();
+    return all;
+  });
 }
 
 int attn_tc_max_active_clusters(int D, int cluster) {
-  static int cache[2][TC_MAX_CLUSTER + 1];
-  static bool have[2][TC_MAX_CLUSTER + 1];
+  static PerDeviceInt cache[2][TC_MAX_CLUSTER + 1];
   const int di = D == 64 ? 0 : 1;
   if (cluster < 1 || cluster > TC_MAX_CLUSTER) return 0;
-  if (!have[di][cluster]) {
+  return cache[di][cluster].get([&]() {
     int n = 0;
     cudaLaunchAttribute attr[2];
     cudaError_t e = cudaErrorUnknown;
@@ -702,10 +701,8 @@ int attn_tc_max_active_clusters(int D, int cluster) {
       e = cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<128, 0>, &cfg);
     }
     if (e != cudaSuccess) { cudaGetLastError(); n = 0; }
-    cache[di][cluster] = n;
-    have[di][cluster] = true;
-  }
-  return cache[di][cluster];
+    return n;
+  }, 0);
 }
 
 template <int D>
@@ -713,7 +710,7 @@ static sb_status launch_tc(const AttnParams& p, dim3 grid, int cluster, cudaStre
   if (!tc_prepare<D>()) return SB_ERR_CUDA;
   cudaLaunchAttribute attr[2];
   cudaLaunchConfig_t cfg = tc_config<D>(grid, cluster, cs, attr);
-  if (getenv("SB_DEBUG"))
+  if (test_knob("SB_DEBUG"))
     fprintf(stderr, "[sb] attn_tc<%d> grid (%u,%u,%u) cluster %d outer %d: max active clusters %d\n", D, grid.x, grid.y,
             grid.z, cluster, p.outer, attn_tc_max_active_clusters(D, cluster));
   const int box_rows = p.tb.page_size == 0 ? TC_BN : (p.tb.page_size < TC_BN ? p.tb.page_size : TC_BN);

@@ -128,7 +128,10 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
     const int pieces = ceil_div(nj, box_rows);
 #pragma unroll 1
     for (int i = 0; i < MAX_PIECES; ++i)
-      if (i < pieces) pg[i] = p.tb.page_table[(long long)b * p.tb.max_pages + (k0 + i * box_rows) / p.tb.page_size];
+      if (i < pieces) {
+        const int lp = (k0 + i * box_rows) / p.tb.page_size;
+        pg[i] = SB_CHECKED_ACCESS(lp, p.tb.max_pages, &p.status[b]) ? p.tb.page_table[(long long)b * p.tb.max_pages + lp] : 0;
+      }
   };
   auto issue_pieces = [&](int j, const int (&pg)[MAX_PIECES], const CUtensorMap* map, uint32_t stage_addr,
                           uint64_t* bar) {
@@ -199,8 +202,9 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
         const int node_l = valid ? R / G : 0;
         const int hh = valid ? R - node_l * G : 0;
         const long long off = ((long long)(si.q_off + node_l) * Hq + g * G + hh) * D + ch * 8;
-        cp_async_16_tc(qd + (r / TC_BM) * QT_BYTES + sw128_chunk_off(r % TC_BM, ch, TC_BM), p.q + (valid ? off : 0),
-                       valid ? 16 : 0);
+        const bool q_ok = valid && SB_CHECKED_ACCESS(off + 7, (long long)p.total_q * Hq * D, &p.status[b]);
+        cp_async_16_tc(qd + (r / TC_BM) * QT_BYTES + sw128_chunk_off(r % TC_BM, ch, TC_BM), p.q + (q_ok ? off : 0),
+                       q_ok ? 16 : 0);
       }
       asm volatile("cp.async.commit_group;\n" ::);
       asm volatile("cp.async.wait_group 0;\n" ::: "memory");
@@ -479,6 +483,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
       const int node_l = Rr / G, hh = Rr - node_l * G;
       const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
       const float lse2 = l > 0.f ? m + log2f(l) : -INFINITY;
+      if (!SB_CHECKED_ACCESS(grow, rows_all, &p.status[b])) continue;
       if (p.outer == 1) {
         *reinterpret_cast<uint4*>(p.out + grow * D + col8 * 8) = raw;
         if (p.lse && col8 == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
@@ -504,15 +509,14 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
 
 template <int D>
 static sb_status launch_tc2(const AttnParams& p, dim3 grid, cudaStream_t cs) {
-  static bool prepared = false;
-  if (!prepared) {
-    if (cudaFuncSetAttribute(attn_tc2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_tc2_smem_bytes<D>()) != cudaSuccess) {
-      cudaGetLastError();
-      return SB_ERR_CUDA;
-    }
-    prepared = true;
-  }
+  static PerDeviceOnce once;
+  if (!once.run([]() {
+        const bool ok = cudaFuncSetAttribute(attn_tc2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)attn_tc2_smem_bytes<D>()) == cudaSuccess;
+        if (!ok) cudaGetLastError();
+        return ok;
+      }))
+    return SB_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(T2_THREADS);
@@ -523,8 +527,8 @@ static sb_status launch_tc2(const AttnParams& p, dim3 grid, cudaStream_t cs) {
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = getenv("SB_NO_PDL") ? 0 : 1;
-  if (getenv("SB_DEBUG"))
+  cfg.numAttrs = test_knob("SB_NO_PDL") ? 0 : 1;
+  if (test_knob("SB_DEBUG"))
     fprintf(stderr, "[sb] attn_tc2<%d> grid (%u,%u,%u) outer %d\n", D, grid.x, grid.y, grid.z, p.outer);
   const int box_rows = p.tb.page_size == 0 ? TC_BN : (p.tb.page_size < TC_BN ? p.tb.page_size : TC_BN);
   CUtensorMap kmap, vmap, qmap;

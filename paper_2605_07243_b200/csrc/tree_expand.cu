@@ -558,13 +558,15 @@ __global__ void __launch_bounds__(FINISH_THREADS) expand_finish_kernel(
       const int base_depth = start == -1 ? 0 : (slab == 0 ? pre_depth : depth[start]) + 1;
       for (int j = 0; j < width && first + j < node_budget; ++j) {
         const int n = first + j;
+        if (!SB_CHECKED_ACCESS(n, node_budget, status)) break;
         tok[n] = topk_tok[r * SB_KMAX + j];
         parent[n] = par;
         depth[n] = base_depth + kpos;
         node_row[n] = row_base + r;
         node_rank[n] = j;
       }
-      if (child_row && par >= 0 && first < node_budget) child_row[par] = row_base + r;  // this row proposed par's children
+      if (child_row && par >= 0 && first < node_budget && SB_CHECKED_ACCESS(par, node_budget, status))
+        child_row[par] = row_base + r;  // this row proposed par's children
     }
     __syncthreads();
     if (tid == 0) s_carry = carry + s_warp_sum[FINISH_THREADS / 32 - 1];
@@ -708,7 +710,7 @@ __global__ void __launch_bounds__(ROWS_THREADS) expand_rows_kernel(
     const int id = low < 0x80000000u ? -1 : (int)(0xffffffffu - low);
     topk_tok[rr * SB_KMAX + rank] = id;
     topk_val[rr * SB_KMAX + rank] = s_val[c];
-    if (!any_bad && rank < width && first + rank < node_budget) {
+    if (!any_bad && rank < width && first + rank < node_budget && SB_CHECKED_ACCESS(first + rank, node_budget, status)) {
       const int n = first + rank;
       tok[n] = id;
       parent[n] = par;
@@ -718,7 +720,9 @@ __global__ void __launch_bounds__(ROWS_THREADS) expand_rows_kernel(
     }
   }
   // this row proposed the children of `par`: recorded for the calls that need the draft distribution of a node
-  if (tid == 0 && child_row && !any_bad && width > 0 && first < node_budget && par >= 0) child_row[par] = row_base + rr;
+  if (tid == 0 && child_row && !any_bad && width > 0 && first < node_budget && par >= 0 &&
+      SB_CHECKED_ACCESS(par, node_budget, status))
+    child_row[par] = row_base + rr;
   if (rr == 0 && tid == 0) {
     if (any_bad) {
       *status = SB_ERR_INVALID_ARG;
@@ -830,13 +834,14 @@ static size_t topk_list_bytes(int n_rows, int vocab) {
 // Dynamic shared memory of topk_partial_reg_kernel: the staged chunk.  Both instantiations are told
 // once that they may exceed the default 48 KB together with their static arrays.
 static size_t topk_stage_bytes(int chunk) {
-  static bool prepared = false;
-  if (!prepared) {
-    cudaFuncSetAttribute(topk_partial_reg_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TOPK_STAGE_BYTES);
-    cudaFuncSetAttribute(topk_partial_reg_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TOPK_STAGE_BYTES);
-    cudaGetLastError();
-    prepared = true;
-  }
+  static PerDeviceOnce once;
+  once.run([]() {
+    const bool ok =
+        cudaFuncSetAttribute(topk_partial_reg_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TOPK_STAGE_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(topk_partial_reg_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TOPK_STAGE_BYTES) == cudaSuccess;
+    if (!ok) cudaGetLastError();
+    return ok;  // a failure shows as a launch error of the scan
+  });
   return (size_t)chunk * sizeof(float);
 }
 

@@ -99,8 +99,11 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) row_argmax_kernel(const T* __r
       // Every thread keeps the first of its maxima by strict compares over ascending ids, so a chunk
       // that holds nothing above -inf (NaN counts as -inf) records no id at all: its first element wins.
       if (x.i == 0x7fffffff && begin < end) x.i = begin;
-      part_val[(long long)row * n_chunks + c] = x.v;
-      part_idx[(long long)row * n_chunks + c] = x.i;
+      // (checked build: gridDim.y rows of n_chunks partials each were sized by the host)
+      if (SB_CHECKED_ACCESS((long long)row * n_chunks + c, (long long)gridDim.y * n_chunks, nullptr)) {
+        part_val[(long long)row * n_chunks + c] = x.v;
+        part_idx[(long long)row * n_chunks + c] = x.i;
+      }
     }
   }
 }
@@ -140,7 +143,7 @@ __global__ void __launch_bounds__(SB_MAX_NODES) accept_kernel(int n_chunks, cons
       if (better(v, id, bv, bi)) { bv = v; bi = id; }
     }
     s_amax[i] = bi;
-    amax[o + i] = bi;
+    if (SB_CHECKED_ACCESS(o + i, total_nodes, &status[b])) amax[o + i] = bi;
     const int p = parent[o + i];
     s_parent[i] = p;
     s_tok[i] = tok[o + i];
@@ -169,6 +172,7 @@ __global__ void __launch_bounds__(SB_MAX_NODES) accept_kernel(int n_chunks, cons
     bonus[b] = s_amax[node];
     otok[depth] = s_amax[node];
     for (int t = depth; t >= 0; --t) {
+      if (!SB_CHECKED_ACCESS(t, max_depth + 1, &status[b]) || !SB_CHECKED_ACCESS(node, n, &status[b])) break;
       path[t] = node;
       if (t > 0) otok[t - 1] = s_tok[node];
       node = s_parent[node];
@@ -258,20 +262,21 @@ extern "C" sb_status sb_verify_accept_static(const void* logits, sb_dtype dtype,
   if (need > (size_t)SB_STATIC_SCRATCH_BYTES) return SB_ERR_WORKSPACE;  // larger than the fixed array
 
   // Device address of the array, looked up once per device with that device current.
-  constexpr int kMaxDevices = 64;
-  static void* scratch_of_device[kMaxDevices] = {};
+  // (Atomic slots: two host threads may make a device's first call at once; both then store the same
+  // address.  The address holds for the life of the device's primary context.)
+  static std::atomic<void*> scratch_of_device[kMaxDevices];
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return SB_ERR_CUDA;
   if (dev >= kMaxDevices) return SB_ERR_UNSUPPORTED;
-  if (!scratch_of_device[dev]) {
-    void* ptr = nullptr;
+  void* ptr = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!ptr) {
     if (cudaGetSymbolAddress(&ptr, g_accept_scratch) != cudaSuccess || !ptr) {
       cudaGetLastError();
       return SB_ERR_CUDA;
     }
-    scratch_of_device[dev] = ptr;
+    scratch_of_device[dev].store(ptr, std::memory_order_release);
   }
-  char* scratch = static_cast<char*>(scratch_of_device[dev]);
+  char* scratch = static_cast<char*>(ptr);
 
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   const int esz = dtype == SB_BF16 ? 2 : 4;

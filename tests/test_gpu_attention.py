@@ -182,9 +182,10 @@ def test_chunk_without_visible_key():
 
 
 @pytest.mark.parametrize("impl", ["mma", "tc"])
-def test_both_tensor_core_paths(monkeypatch, impl):
-    """The tcgen05 kernel is the default; the mma.sync kernel stays selectable and correct."""
-    monkeypatch.setenv("SB_ATTN_IMPL", impl)
+def test_both_tensor_core_paths(test_build, impl):
+    """The tcgen05 kernel is the library's only backend; the test build also holds an mma.sync kernel,
+    an independent implementation that must agree with the oracle on the same cases."""
+    test_build.setenv("SB_ATTN_IMPL", impl)
     attn, _ = W.config1_tiny()
     check_attention(attn, f"{impl}: config 1", num_splits=2)
     check_attention(W.config2_verify_layer(prefix=777), f"{impl}: 8B-shaped, P=777")
@@ -195,8 +196,8 @@ def test_both_tensor_core_paths(monkeypatch, impl):
     check_attention(case, f"{impl}: ragged paged G=8", num_splits=5)
 
 
-def test_simple_kernel_path(monkeypatch):
-    monkeypatch.setenv("SB_ATTN_IMPL", "simple")
+def test_simple_kernel_path(test_build):
+    test_build.setenv("SB_ATTN_IMPL", "simple")
     attn, _ = W.config1_tiny()
     check_attention(attn, "simple kernel, config 1")
     rng = W.rng_for(47)
@@ -269,10 +270,10 @@ def test_config5_long_context_full_size_sampled():
     check_attention(attn, "config 5 sampled, 16 chunks", sel=sel, num_splits=16)
 
 
-def test_two_tiles_per_cta_kernel(monkeypatch):
+def test_two_tiles_per_cta_kernel(test_build):
     """The throughput kernel (two row tiles per CTA, P written over S in tensor memory, chunks merged
     from fp32 partials), forced on shapes that would otherwise take the one-tile kernel."""
-    monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
+    test_build.setenv("SB_ATTN_TWO_TILES", "1")
     check_attention(W.config2_verify_layer(prefix=777), "two tiles: 8B-shaped, P=777, 1 chunk", num_splits=1)
     check_attention(W.config2_verify_layer(prefix=777), "two tiles: 8B-shaped, P=777, 3 chunks", num_splits=3)
     check_attention(W.config2_verify_layer(prefix=2048), "two tiles: 8B-shaped, library's chunks")
@@ -294,10 +295,10 @@ def test_two_tiles_per_cta_kernel(monkeypatch):
     check_attention(case, "two tiles: P=0")
 
 
-def test_two_tiles_per_cta_long_chunks(monkeypatch):
+def test_two_tiles_per_cta_long_chunks(test_build):
     """Many blocks per CTA (the steady state of the two-tile pipeline), peaky scores so that the
     reference maximum moves and accumulators are rescaled."""
-    monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
+    test_build.setenv("SB_ATTN_TWO_TILES", "1")
     rng = W.rng_for(71)
     case = W.make_attn_case(rng, parents=[W.random_tree(rng, 96, 10), W.random_tree(rng, 33, 10)],
                             prefix_lens=[6000, 3001], n_q_heads=32, n_kv_heads=8, head_dim=128, page_size=64, q_std=4.0)
@@ -306,7 +307,7 @@ def test_two_tiles_per_cta_long_chunks(monkeypatch):
 
 
 @pytest.mark.parametrize("seed", range(12))
-def test_random_shapes_against_oracle(seed, monkeypatch):
+def test_random_shapes_against_oracle(seed, test_build):
     """Seeded random shapes: batch, head layout, head_dim, page size, tree sizes, prefix lengths, query
     range, chunk count and kernel variant all drawn at random; element-wise parity on every one."""
     rng = W.rng_for(9000 + seed)
@@ -327,7 +328,7 @@ def test_random_shapes_against_oracle(seed, monkeypatch):
                             q_std=float(rng.choice([1.0, 1.0, 4.0])), capacity_pad=int(rng.integers(0, 40)))
     splits = int(rng.choice([0, 0, 1, 2, 3, 5, 8, 16]))
     if rng.random() < 0.4:
-        monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
+        test_build.setenv("SB_ATTN_TWO_TILES", "1")
     check_attention(case, f"random shape {seed}: B={B} Hkv={hkv} G={G} D={D} page={page} splits={splits}",
                     num_splits=splits)
 
@@ -353,7 +354,7 @@ def test_settled_flags_give_the_same_bits():
 
 @pytest.mark.parametrize("page_size", [0, 64])
 @pytest.mark.parametrize("num_splits", [0, 1, 3])
-def test_empty_sequences_inside_a_batch(page_size, num_splits, monkeypatch):
+def test_empty_sequences_inside_a_batch(page_size, num_splits, test_build):
     """Sequences without any tree node (and one whose query range is empty) between ordinary ones: they own no
     output row, report status 0 and leave their neighbours' rows alone -- on the one-tile and the two-tile kernel."""
     rng = W.rng_for(77 + page_size + num_splits)
@@ -362,5 +363,5 @@ def test_empty_sequences_inside_a_batch(page_size, num_splits, monkeypatch):
     case = W.make_attn_case(rng, parents=parents, prefix_lens=[40, 300, 0, 0, 129, 5], n_q_heads=8, n_kv_heads=2,
                             head_dim=128, page_size=page_size, q_node_begin=[0, 0, 0, 3, 20, 0])
     for two in ("0", "1"):
-        monkeypatch.setenv("SB_ATTN_TWO_TILES", two)
+        test_build.setenv("SB_ATTN_TWO_TILES", two)
         check_attention(case, f"empty sequences, page {page_size}, splits {num_splits}, two tiles {two}", num_splits=num_splits)

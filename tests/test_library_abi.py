@@ -64,3 +64,33 @@ def test_binding_struct_matches_header_layout():
     assert s.k_cache.offset == 16 and s.kv_capacity.offset == 40 and s.page_table.offset == 56
     assert s.max_nodes.offset == 88 and s.index_arrays_settled.offset == 96
     assert ctypes.sizeof(s) == 104
+
+
+def _test_header_symbols():
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    text = open(os.path.join(root, "include", "specblock_test.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sb_[a-z_]+)\s*\(", text)))
+
+
+def test_build_variants_export_their_hooks_and_the_library_proper_does_not():
+    """libspecblock_test.so / libspecblock_checked.so: the same ABI plus the hooks of specblock_test.h.
+    The library proper exports none of the hooks, holds no check kernel and reads no environment."""
+    hooks = _test_header_symbols()
+    assert hooks == ["sb_checked_selftest", "sb_checked_violations", "sb_test_wait_expires"]
+    proper = ctypes.CDLL(build.build())
+    test = ctypes.CDLL(build.build(variant="test"))
+    checked = ctypes.CDLL(build.build(variant="checked"))
+    for name in _declared_symbols():
+        assert hasattr(test, name) and hasattr(checked, name), name
+    for name in hooks:
+        assert not hasattr(proper, name), f"{name} must not be in the library proper"
+    assert hasattr(test, "sb_test_wait_expires") and not hasattr(test, "sb_checked_violations")
+    assert hasattr(checked, "sb_checked_violations") and hasattr(checked, "sb_checked_selftest")
+    # the only getenv of the sources is the test build's switch reader
+    csrc = os.path.join(os.path.dirname(build.__file__), "csrc")
+    uses = [(f, i + 1) for f in sorted(os.listdir(csrc)) for i, line in enumerate(open(os.path.join(csrc, f)))
+            if "getenv" in line]
+    assert uses == [("common.cuh", uses[0][1])], uses
+    common = open(os.path.join(csrc, "common.cuh")).read()
+    assert common.index("#ifdef SB_TEST_KERNELS") < common.index("getenv") < common.index("#else", common.index("getenv") - 200)
