@@ -173,6 +173,60 @@ def test_mask_leaks_are_order_one(prefix):
                         value_scale=100.0)
 
 
+def _dominant_tree_keys(rng, parents, prefix_lens, **shape):
+    """Every tree key overwhelms the whole prefix for every query row (one shared query component of 8
+    against a key component of 32: a score of +22 before the usual N(0,1) part, against at most 33k prefix
+    keys of weight ~1) and carries V = +-100 with random signs: an output row is then a short weighted
+    average of +-100 over the row's own ancestors.  One leaked off-path key, or one missing on-path key,
+    moves it by O(10); the tolerance's absolute term is 1.0 here (value_scale = 100)."""
+    case = W.make_attn_case(rng, parents=parents, prefix_lens=prefix_lens, **shape)
+    q = W.bf16_bits_to_f32(case.q)
+    q[:, :, 0] = 8.0
+    case.q = W.f32_to_bf16_bits(q)
+    k, v = W.bf16_bits_to_f32(case.k), W.bf16_bits_to_f32(case.v)
+    for b, par in enumerate(parents):
+        for i in range(len(par)):
+            slot = W.kv_slot(case, b, int(prefix_lens[b]) + i)
+            k[slot][:, 0] = 32.0
+            v[slot] = 100.0 * rng.choice([-1.0, 1.0], size=v[slot].shape)
+    case.k, case.v = W.f32_to_bf16_bits(k), W.f32_to_bf16_bits(v)
+    return case
+
+
+@pytest.mark.parametrize("page_size", [0, 16, 64])
+@pytest.mark.parametrize("two_tiles", [False, True])
+def test_mask_leaks_are_order_one_across_tiles_pages_and_blocks(page_size, two_tiles, request):
+    """The tree's cache slots straddle a page boundary, a 128-key block boundary and a chunk boundary,
+    on the one-tile and on the two-tile kernel (whose window-application code is its own), contiguous
+    and paged.  G = 8 with up to 60 nodes gives one to four row tiles per KV head."""
+    if two_tiles:
+        request.getfixturevalue("test_build").setenv("SB_ATTN_TWO_TILES", "1")
+    rng = W.rng_for(4600 + page_size + (1 if two_tiles else 0))
+    shape = dict(n_q_heads=16, n_kv_heads=2, head_dim=128, page_size=page_size)
+    for prefix in ([13, 120], [60, 250], [127, 1000], [128, 5]):
+        parents = [W.random_tree(rng, 60, 7), W.block_tree(rng, 40)]
+        case = _dominant_tree_keys(rng, parents, prefix, **shape)
+        for splits in (1, 2, 3):
+            check_attention(case, f"dominant tree keys, page {page_size}, two tiles {two_tiles}, P={prefix}, splits={splits}",
+                            num_splits=splits, value_scale=100.0)
+
+
+@pytest.mark.parametrize("prefix", [8000, 33000])
+@pytest.mark.parametrize("two_tiles", [False, True])
+def test_mask_leaks_are_order_one_behind_a_long_prefix(prefix, two_tiles, request):
+    """Long prefixes are where the float tolerance alone cannot see a leaked key (one key among 33k moves
+    the output by 3e-5): here the tree sits in the last of 16 chunks behind 8k / 33k prefix keys, with the
+    128-node trees and eight heads per KV head of the long-context configuration, paged as it is."""
+    if two_tiles:
+        request.getfixturevalue("test_build").setenv("SB_ATTN_TWO_TILES", "1")
+    rng = W.rng_for(4700 + prefix // 1000 + (1 if two_tiles else 0))
+    case = _dominant_tree_keys(rng, [W.random_tree(rng, 128, 12)], [prefix], n_q_heads=16, n_kv_heads=2,
+                               head_dim=128, page_size=64)
+    for splits in (16, 0):
+        check_attention(case, f"dominant tree keys behind P={prefix}, two tiles {two_tiles}, splits={splits}",
+                        num_splits=splits, value_scale=100.0)
+
+
 def test_chunk_without_visible_key():
     """P = 0 and many chunks: most chunks hold no key a given row may see."""
     rng = W.rng_for(46)
@@ -256,18 +310,28 @@ def test_host_argument_errors():
     assert e.value.code == 1
 
 
-# ---- full-size configurations: sampled rows (the oracle computes each row on its own) ---------
+# ---- full-size configurations, every output element (the oracle takes seconds on them) ----------
 
-def test_config4_batched_full_size_sampled():
+def test_config4_batched_full_size():
+    """All 16 ragged paged sequences, every row: the launch configuration the bench times (the library's
+    own choice of chunks) and an explicit split."""
     attn, _ = W.config4_batched(with_logits=False)
-    sel = sample_rows(attn, 160, seed=4)
-    check_attention(attn, "config 4 sampled", sel=sel)
+    ref = oracle.tree_attention(**attn.oracle_kwargs())
+    for what, kw in (("config 4, library's chunks", {}), ("config 4, 3 chunks", dict(num_splits=3))):
+        out, lse, status = gpu_attention(attn, **kw)
+        np.testing.assert_array_equal(status, ref[2])
+        assert_attention_close(out, lse, ref[0], ref[1], what)
 
 
-def test_config5_long_context_full_size_sampled():
+def test_config5_long_context_full_size():
+    """All four 32k-token sequences, every row, with the 16 chunks the configuration prescribes and with
+    the chunk count the library chooses (one chunk: 257 key blocks per CTA)."""
     attn, _ = W.config5_long(with_logits=False)
-    sel = sample_rows(attn, 96, seed=5)
-    check_attention(attn, "config 5 sampled, 16 chunks", sel=sel, num_splits=16)
+    ref = oracle.tree_attention(**attn.oracle_kwargs())
+    for what, kw in (("config 5, 16 chunks", dict(num_splits=16)), ("config 5, library's chunks", {})):
+        out, lse, status = gpu_attention(attn, **kw)
+        np.testing.assert_array_equal(status, ref[2])
+        assert_attention_close(out, lse, ref[0], ref[1], what)
 
 
 def test_two_tiles_per_cta_kernel(test_build):
@@ -307,7 +371,7 @@ def test_two_tiles_per_cta_long_chunks(test_build):
 
 
 @pytest.mark.parametrize("seed", range(12))
-def test_random_shapes_against_oracle(seed, test_build):
+def test_random_shapes_against_oracle(seed, request):
     """Seeded random shapes: batch, head layout, head_dim, page size, tree sizes, prefix lengths, query
     range, chunk count and kernel variant all drawn at random; element-wise parity on every one."""
     rng = W.rng_for(9000 + seed)
@@ -327,8 +391,8 @@ def test_random_shapes_against_oracle(seed, test_build):
                             page_size=page, q_node_begin=qbegin if use_qbegin else None,
                             q_std=float(rng.choice([1.0, 1.0, 4.0])), capacity_pad=int(rng.integers(0, 40)))
     splits = int(rng.choice([0, 0, 1, 2, 3, 5, 8, 16]))
-    if rng.random() < 0.4:
-        test_build.setenv("SB_ATTN_TWO_TILES", "1")
+    if rng.random() < 0.4:   # the forced two-tile kernel lives in the test build; the rest runs on the library proper
+        request.getfixturevalue("test_build").setenv("SB_ATTN_TWO_TILES", "1")
     check_attention(case, f"random shape {seed}: B={B} Hkv={hkv} G={G} D={D} page={page} splits={splits}",
                     num_splits=splits)
 
@@ -354,7 +418,7 @@ def test_settled_flags_give_the_same_bits():
 
 @pytest.mark.parametrize("page_size", [0, 64])
 @pytest.mark.parametrize("num_splits", [0, 1, 3])
-def test_empty_sequences_inside_a_batch(page_size, num_splits, test_build):
+def test_empty_sequences_inside_a_batch(page_size, num_splits, monkeypatch):
     """Sequences without any tree node (and one whose query range is empty) between ordinary ones: they own no
     output row, report status 0 and leave their neighbours' rows alone -- on the one-tile and the two-tile kernel."""
     rng = W.rng_for(77 + page_size + num_splits)
@@ -362,6 +426,7 @@ def test_empty_sequences_inside_a_batch(page_size, num_splits, test_build):
     parents = [none, W.random_tree(rng, 70, 6), none, W.chain_tree(9), W.random_tree(rng, 20, 4), none]
     case = W.make_attn_case(rng, parents=parents, prefix_lens=[40, 300, 0, 0, 129, 5], n_q_heads=8, n_kv_heads=2,
                             head_dim=128, page_size=page_size, q_node_begin=[0, 0, 0, 3, 20, 0])
-    for two in ("0", "1"):
-        test_build.setenv("SB_ATTN_TWO_TILES", two)
-        check_attention(case, f"empty sequences, page {page_size}, splits {num_splits}, two tiles {two}", num_splits=num_splits)
+    check_attention(case, f"empty sequences, page {page_size}, splits {num_splits}", num_splits=num_splits)
+    with sb.build_variant("test"):
+        monkeypatch.setenv("SB_ATTN_TWO_TILES", "1")
+        check_attention(case, f"empty sequences, page {page_size}, splits {num_splits}, two tiles", num_splits=num_splits)

@@ -299,6 +299,51 @@ def test_accept_then_compact_chain_on_device():
         np.testing.assert_array_equal(got_k[0, 200 + j], case.k[0, 200 + node])
 
 
+@pytest.mark.parametrize("which", [4, 5])
+def test_accept_then_compact_on_the_batched_and_long_configurations(which):
+    """Configurations 4 (16 ragged paged sequences, accept lengths drawn with the paper's per-position
+    acceptance rates) and 5 (four 32k-token sequences) at full size: acceptance on the planted logits, then
+    the in-place compaction of two layers of the real paged caches, chained on the device; paths, tokens,
+    new lengths and every live cache row against the oracle."""
+    attn, ver = W.config4_batched() if which == 4 else W.config5_long()
+    L = 2
+    layer_elems = int(attn.k.size)
+    rng = W.rng_for(8800 + which)
+    k_all = np.stack([attn.k, attn.v])                         # two "layers" with distinct contents
+    v_all = np.stack([attn.v, attn.k])
+    logits = dev.bf16_tensor(ver.logits) if ver.logits.dtype == np.uint16 else torch.from_numpy(ver.logits).cuda()
+    r = sb.sb_verify_accept(logits, dev.i32_tensor(ver.node_offsets), dev.i32_tensor(ver.parent),
+                            dev.i32_tensor(ver.tok), ver.max_depth)
+    tb = dev.tree_batch(attn, k=dev.bf16_tensor(k_all), v=dev.bf16_tensor(v_all))
+    new_len, status = sb.sb_kv_compact(tb, L, layer_elems, r["path_nodes"], r["accept_len"], ver.max_depth)
+    torch.cuda.synchronize()
+    ref = oracle.verify_accept(ver.logits, ver.node_offsets, ver.parent, ver.tok, ver.max_depth)
+    for key in ("amax", "accept_len", "path_nodes", "out_tokens", "bonus", "status"):
+        np.testing.assert_array_equal(r[key].cpu().numpy(), ref[key], err_msg=key)
+    np.testing.assert_array_equal(ref["accept_len"], ver.planted_len)
+    kw = dict(n_kv_heads=attn.n_kv_heads, head_dim=attn.head_dim, n_layers=L, layer_stride_elems=layer_elems,
+              page_size=attn.page_size, max_pages=attn.max_pages, num_pages=attn.num_pages, kv_capacity=attn.kv_capacity,
+              page_table=attn.page_table, prefix_len=attn.prefix_len, node_offsets=attn.node_offsets,
+              path_nodes=ref["path_nodes"], accept_len=ref["accept_len"], max_depth=ver.max_depth)
+    ref_k, ref_len, ref_st = oracle.kv_compact(cache=k_all.reshape(-1), **kw)
+    ref_v, _, _ = oracle.kv_compact(cache=v_all.reshape(-1), **kw)
+    np.testing.assert_array_equal(status.cpu().numpy(), ref_st)
+    np.testing.assert_array_equal(new_len.cpu().numpy(), ref_len)
+    np.testing.assert_array_equal(ref_len, attn.prefix_len + ver.planted_len + 1)
+    got_k = tb.k_cache.view(torch.int16).cpu().numpy().view(np.uint16).reshape(k_all.shape)
+    got_v = tb.v_cache.view(torch.int16).cpu().numpy().view(np.uint16).reshape(v_all.shape)
+    ref_k, ref_v = ref_k.reshape(k_all.shape), ref_v.reshape(v_all.shape)
+    # pages belong to one sequence each, slots past new_len are written by neither side: whole caches compare
+    np.testing.assert_array_equal(got_k, ref_k)
+    np.testing.assert_array_equal(got_v, ref_v)
+    for b in range(attn.batch):                                # and the committed rows are where they belong
+        for j, node in enumerate(ref["path_nodes"][b, :ref["accept_len"][b] + 1]):
+            dst = W.kv_slot(attn, b, int(attn.prefix_len[b]) + j)
+            src = W.kv_slot(attn, b, int(attn.prefix_len[b]) + int(node))
+            np.testing.assert_array_equal(got_k[(0,) + dst], attn.k[src])
+            np.testing.assert_array_equal(got_v[(0,) + dst], attn.v[src])
+
+
 # ---- rank-head distribution summary -------------------------------------------------------------------
 
 # fp32 sums over rows of up to 128256 terms: |err| <= 2e-5 * max(1, |ref|)

@@ -3,11 +3,13 @@ memory (its argmax partials live in a fixed array inside the library).  Collecte
 
 Called through the C ABI twice in a row on different inputs; every result must equal what the
 workspace-taking entry point returns for the same inputs (integer results: exact equality), which
-also shows that the shared array needs no clearing between calls."""
+also shows that the shared array needs no clearing between calls -- and what the CPU oracle computes
+from the same host arrays."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2605_07243_b200 import binding as sb
 from paper_2605_07243_b200 import device_inputs as dev
 from paper_2605_07243_b200 import workloads as W
@@ -32,8 +34,10 @@ def _both_ways(case):
     ref = sb.sb_verify_accept(logits, offs, par, tok, case.max_depth)
     got = sb.sb_verify_accept_static(logits, offs, par, tok, case.max_depth, _empty_out(total, batch, case.max_depth))
     torch.cuda.synchronize()
+    want = oracle.verify_accept(case.logits, case.node_offsets, case.parent, case.tok, case.max_depth)
     for k in KEYS:
         np.testing.assert_array_equal(got[k].cpu().numpy(), ref[k].cpu().numpy(), err_msg=k)
+        np.testing.assert_array_equal(got[k].cpu().numpy(), want[k], err_msg=f"{k} against the oracle")
     return got
 
 
