@@ -10,6 +10,13 @@ than L2), greedy acceptance over bf16 logits [60, 128256], and KV compaction of 
 The step is captured once in a CUDA graph and replayed; time is taken with CUDA events on the
 launching stream, max over ranks.  Prints ONE JSON line (rank 0).
 
+Beside the contract's figure (exactly --steps replays between two events), the line carries
+distributions that do not depend on --steps: the step and every breakdown entry as median / p10 / p90
+over at least 200 samples, and under "configs" the tree attention of all five benchmark
+configurations (at least 200 samples for 1-3, 30 for 4-5; configuration 5 with the 16 chunks it
+prescribes and with the library's own choice), each a CUDA-graph replay that walks buffer sets larger
+than L2, with algorithmic bytes and flops and the fraction of its binding roof.
+
 With N > 1 (launched by torch.distributed.run) every rank runs its own sequence (weak scaling,
 no data-path collective); NCCL is used only for the barrier and the max over ranks.
 
@@ -32,20 +39,22 @@ if ROOT not in sys.path:
 METRIC = "tree-verify attention GB/s (% of B200 HBM peak) and us per verify step"
 N_LAYERS = 32
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on this workload, from the
-# ncu capture summarised in profiles/attn_tc_kernel_c2_verify_layer.md
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of this workload, from an ncu
+# capture of the library as committed (the summary of that capture is committed with the profiles)
 ATTN_DRAM_TRAFFIC_BYTES = 9189120
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_TFLOPS = 1400.0   # sustained dense bf16
 
 
 def measured_peaks():
+    """(HBM GB/s, sustained dense bf16 TFLOP/s, "measured" | "fallback")."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
+        return float(d["hbm_gbs"]), float(d["bf16_tflops_sustained"]), "measured"
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback"
+        return FALLBACK_HBM_GBS, FALLBACK_TFLOPS, "fallback"
 
 
 def build_workload(rank, n_layers):
@@ -200,6 +209,74 @@ def capture(torch, fn):
     return g
 
 
+def sample_graph(torch, graph, samples, replays_per_sample=1, calls_per_replay=1):
+    """`samples` event pairs on the current stream, each around `replays_per_sample` replays of `graph`
+    (which holds `calls_per_replay` calls): -> microseconds per call as median / p10 / p90."""
+    import numpy as np
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(samples)]
+    for e0, e1 in pairs:
+        e0.record()
+        for _ in range(replays_per_sample):
+            graph.replay()
+        e1.record()
+    torch.cuda.synchronize()
+    us = np.asarray([e0.elapsed_time(e1) for e0, e1 in pairs]) * 1e3 / (replays_per_sample * calls_per_replay)
+    return {"median_us": float(np.median(us)), "p10_us": float(np.percentile(us, 10)),
+            "p90_us": float(np.percentile(us, 90)), "samples": samples,
+            "calls_per_sample": replays_per_sample * calls_per_replay}
+
+
+ATTENTION_CONFIGS = (   # (key, configuration, num_splits, samples)
+    ("1_tiny", 1, 0, 200), ("2_8b_verify_layer", 2, 0, 200), ("3_drafter_blocks", 3, 0, 200),
+    ("4_batched_paged", 4, 0, 30), ("5_long_context_16_chunks", 5, 16, 30), ("5_long_context_library_chunks", 5, 0, 30))
+
+
+def time_attention_config(torch, sb, which, num_splits, samples):
+    """sb_tree_attention on one benchmark configuration, standing alone: a CUDA graph walks copies of the
+    K/V caches whose total exceeds twice the L2 size, so every call streams its keys and values from HBM."""
+    import numpy as np
+    from paper_2605_07243_b200 import device_inputs as dev
+    from paper_2605_07243_b200 import workloads as W
+    case = {1: lambda: W.config1_tiny()[0], 2: W.config2_verify_layer, 3: lambda: W.config3_drafter()[0],
+            4: lambda: W.config4_batched(with_logits=False)[0], 5: lambda: W.config5_long(with_logits=False)[0]}[which]()
+    kv_bytes = case.k.nbytes + case.v.nbytes
+    l2 = torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size
+    n_sets = max(2, min(32, int(np.ceil(2 * l2 / kv_bytes))))
+    tb, q, kw = dev.attention_args(case)
+    sets = [(tb.k_cache, tb.v_cache)] + [(tb.k_cache.clone(), tb.v_cache.clone()) for _ in range(n_sets - 1)]
+    out = torch.empty_like(q)
+    lse = torch.empty((q.shape[0], case.n_q_heads), dtype=torch.float32, device="cuda")
+    status = torch.empty(case.batch, dtype=torch.int32, device="cuda")
+    ws = torch.empty(max(256, sb.sb_tree_attention_workspace_bytes(tb, q.shape[0], num_splits)), dtype=torch.uint8,
+                     device="cuda")
+
+    def walk():
+        for k, v in sets:
+            sb.sb_tree_attention(tb, q, out, lse, num_splits=num_splits, workspace=ws, status=status, k_cache=k,
+                                 v_cache=v, **kw)
+
+    walk()
+    torch.cuda.synchronize()
+    assert int(status.max()) == 0
+    graph = capture(torch, walk)
+    st = sample_graph(torch, graph, samples, 1, n_sets)
+    hbm, tflops, kind = measured_peaks()
+    nbytes, flops = case.algorithmic_bytes(), case.flops()
+    t_hbm, t_tc = nbytes / (hbm * 1e9) * 1e6, flops / (tflops * 1e12) * 1e6
+    us = st["median_us"]
+    res = {"us": us, "p10_us": st["p10_us"], "p90_us": st["p90_us"], "samples": samples, "kv_sets_rotated": n_sets,
+           "num_splits": num_splits, "algorithmic_bytes": nbytes, "flops": flops, "GBps": nbytes / us / 1e3,
+           "TFLOPps": flops / us / 1e6, "bound": "hbm" if t_hbm >= t_tc else "tensor",
+           "roof_us": max(t_hbm, t_tc), "frac": max(t_hbm, t_tc) / us,
+           "peak": f"{kind}: " + (f"{hbm} GB/s HBM copy" if t_hbm >= t_tc else f"{tflops} TFLOP/s sustained dense bf16")}
+    del sets, graph, tb, q, out, ws
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_ours(args):
     import torch
     from paper_2605_07243_b200 import binding as sb
@@ -274,16 +351,23 @@ def run_ours(args):
         # the dominant kernel (tree attention): 32 launches on 32 distinct KV buffers per replay
         attn_iters = max(args.steps, 10)
         ms_attn = time_graph(torch, g_attn, attn_iters, dist_on)
+        # distributions that do not depend on --steps: one sample = one replay of the step / the 32 layers
+        n_samples = 20 if args.quick else 200
+        step_stats = sample_graph(torch, g_step, n_samples)
+        attn_stats = sample_graph(torch, g_attn, n_samples, 1, N_LAYERS)
         keep_busy(0.4)
         clocks = sampler.stop()
-        parts_ms = {}
+        parts_stats = {}
+        calls = {"shift_project_32x4096_not_in_step": step.SHIFT_SETS, "fuse_project_8x4x4096_not_in_step": step.FUSE_SETS}
         for name, g in [("expand", g_expand), ("accept", g_accept), ("compact", g_compact)] + extras:
-            for _ in range(3):
-                g.replay()
-            parts_ms[name] = time_graph(torch, g, 20, False) / 20
-        if "shift_project_32x4096_not_in_step" in parts_ms:   # one graph = one call per weight set
-            parts_ms["shift_project_32x4096_not_in_step"] /= step.SHIFT_SETS
-            parts_ms["fuse_project_8x4x4096_not_in_step"] /= step.FUSE_SETS
+            # short graphs: ten replays per sample keep the event pair's own cost out of the figure
+            reps = 1 if name.startswith("whole_iteration") else 10
+            parts_stats[name] = sample_graph(torch, g, n_samples, reps, calls.get(name, 1))
+        parts_ms = {k: v["median_us"] * 1e-3 for k, v in parts_stats.items()}
+        configs = None
+        if world == 1 and not args.quick and not args.step_only:
+            configs = {key: time_attention_config(torch, sb, which, splits, n)
+                       for key, which, splits, n in ATTENTION_CONFIGS}
 
         # end to end: inputs in pinned host memory, results back to pinned host memory
         e2e_steps = 1 if args.quick else max(3, min(args.steps, 5))
@@ -309,7 +393,7 @@ def run_ours(args):
     value = world * total_bytes / (ms_step * 1e-3) / 1e9
     e2e_value = world * total_bytes / (ms_e2e * 1e-3) / 1e9
     h2d, d2h = step.host_bytes()
-    peak, peak_kind = measured_peaks()
+    peak, _tflops, peak_kind = measured_peaks()
     attn_bytes = parts["attention_per_layer"]
     achieved = attn_bytes / (ms_attn_launch * 1e-3) / 1e9
 
@@ -320,6 +404,9 @@ def run_ours(args):
         "config": {"workload": "8B-shaped verify step (configs[1]): batch 1 per GPU, 32 query / 8 KV heads, "
                                "D=128, contiguous bf16 KV prefix 2048, 60-node K=4/M=2 block tree, 32 layers, "
                                "bf16 logits vocab 128256 (accept_len 3), fp32 drafter scores 32x128256",
+                   "step_contents": "ancestor masks, the drafter's top-k expansion of the next block (32 x 128256 "
+                                    "scores: part of the iteration, not of the verify forward proper), 32 attention "
+                                    "layers, greedy acceptance, compaction of 32 layers",
                    "l2": "inputs larger than L2: 32 distinct KV buffers (276 MB) stream through per step",
                    "launch": "whole step captured in one CUDA graph", "num_splits": args.num_splits},
         "us_per_verify_step": ms_step * 1e3,
@@ -328,6 +415,8 @@ def run_ours(args):
         "breakdown_us": {"attention_32_layers": ms_attn_launch * N_LAYERS * 1e3,
                          "attention_per_layer": ms_attn_launch * 1e3,
                          **{k: v * 1e3 for k, v in parts_ms.items()}},
+        "step_us_stats": step_stats,
+        "breakdown_us_stats": {"attention_per_layer": attn_stats, **parts_stats},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e},
@@ -338,6 +427,8 @@ def run_ours(args):
                      "algorithmic_bytes_per_launch": attn_bytes,
                      "pct_of_nominal_8TBps": 100.0 * achieved / NOMINAL_HBM_GBS},
     }
+    if configs is not None:
+        line["configs"] = configs
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.quick:
         import oracle
         t0 = time.perf_counter()
@@ -349,7 +440,7 @@ def run_ours(args):
                                           "compaction) on the fp64 oracle, once"}
     if rank == 0 and world == 1 and args.oracle_configs:
         # The oracle's tree attention on each of the five benchmark configurations, once, on the host
-        # cores (the counterpart of `python -m paper_2605_07243_b200.time_configs`); a baseline only.
+        # cores (the counterpart of the "configs" key); a baseline only.
         import oracle
         from paper_2605_07243_b200 import workloads as W
         makers = {1: lambda: W.config1_tiny()[0], 2: W.config2_verify_layer, 3: lambda: W.config3_drafter()[0],

@@ -8,9 +8,20 @@
 
 #include <atomic>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/specblock.h"
 
 namespace sb {
+
+// NVTX range around an entry point: a profiler's timeline shows which call enqueued which kernels
+// (header-only NVTX; costs a few nanoseconds when no tool is attached).
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 // Host-side count of kernel launches made by this library (read by benchmarks).
 extern long long g_launch_count;

@@ -133,6 +133,7 @@ __global__ void __launch_bounds__(64) path_rows_kernel(const int* __restrict__ n
 extern "C" sb_status sb_path_rows(int32_t batch, const int32_t* node_offsets, const int32_t* node_row,
                                   const int32_t* row_begin, const int32_t* path_nodes, const int32_t* accept_len,
                                   int32_t max_depth, int32_t* path_rows, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_path_rows");
   using namespace sb;
   if (batch < 1 || !node_offsets || !node_row || !path_nodes || !accept_len || !path_rows || !status)
     return SB_ERR_INVALID_ARG;
@@ -145,6 +146,7 @@ extern "C" sb_status sb_path_rows(int32_t batch, const int32_t* node_offsets, co
 extern "C" sb_status sb_kv_compact(const sb_tree_batch* tb, int32_t n_layers, int64_t layer_stride_elems,
                                    const int32_t* path_nodes, const int32_t* accept_len, int32_t max_depth,
                                    int32_t* new_len, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_kv_compact");
   using namespace sb;
   if (!tb || tb->batch < 1 || !tb->k_cache || !tb->v_cache || !tb->prefix_len || !tb->node_offsets ||
       !path_nodes || !accept_len || !new_len || !status || n_layers < 1 || tb->n_kv_heads < 1)

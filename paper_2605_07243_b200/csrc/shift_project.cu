@@ -409,6 +409,7 @@ extern "C" size_t sb_shift_project_workspace_bytes(int32_t n_rows, int32_t d, in
 extern "C" sb_status sb_shift_project(const void* h, const void* w, int32_t n_rows, int32_t d, int32_t d_out,
                                       int32_t block_k, void* out, void* workspace, size_t workspace_bytes,
                                       int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_shift_project");
   using namespace sb;
   if (!h || !w || !out || !status) return SB_ERR_INVALID_ARG;
   ShiftPlan pl;
@@ -443,6 +444,7 @@ extern "C" sb_status sb_fuse_project(const void* c, const void* e, const void* q
                                      int32_t n_starts, int32_t block_k, int32_t d, int32_t d_out, float* q_term,
                                      int32_t q_term_valid, void* out, void* workspace, size_t workspace_bytes,
                                      int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_fuse_project");
   using namespace sb;
   if (!c || !e || !q || !w || !out || !status || (q_term_valid && !q_term) || !(eps >= 0.f)) return SB_ERR_INVALID_ARG;
   FusePlan fp;

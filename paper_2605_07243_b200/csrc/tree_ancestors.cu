@@ -36,6 +36,7 @@ __global__ void __launch_bounds__(128) tree_ancestors_kernel(int batch, const in
 extern "C" sb_status sb_tree_ancestors(int32_t batch, const int32_t* node_offsets, const int32_t* parent,
                                        int32_t max_nodes, uint32_t* anc_mask, int32_t* depth,
                                        int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_tree_ancestors");
   if (batch < 1 || !node_offsets || !parent || !status) return SB_ERR_INVALID_ARG;
   if (max_nodes < 1 || max_nodes > SB_MAX_NODES) return SB_ERR_UNSUPPORTED;
   if (anc_mask && (reinterpret_cast<uintptr_t>(anc_mask) & 15)) return SB_ERR_INVALID_ARG;

@@ -728,6 +728,7 @@ extern "C" sb_status sb_tree_attention(const sb_tree_batch* tb, const int32_t* q
                                        const int32_t* q_offsets, int32_t total_q, const void* q, void* out,
                                        float* lse, float scale, int32_t num_splits, void* workspace,
                                        size_t workspace_bytes, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_tree_attention");
   using namespace sb;
   sb_status st = check_batch(tb);
   if (st != SB_OK) return st;

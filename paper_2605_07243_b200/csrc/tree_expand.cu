@@ -922,6 +922,7 @@ extern "C" sb_status sb_tree_expand(const float* scores, int64_t row_stride, int
                                     int32_t* tok, int32_t* parent, int32_t* depth, int32_t* node_row,
                                     int32_t* node_rank, int32_t* topk_tok, float* topk_val, void* workspace,
                                     size_t workspace_bytes, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_tree_expand");
   return expand_impl(scores, row_stride, n_rows, vocab, block_k, bucket, bmap, start_parent, node_budget, n_nodes, tok,
                      parent, depth, node_row, node_rank, topk_tok, topk_val, nullptr, nullptr, 0, workspace,
                      workspace_bytes, status, stream);
@@ -934,6 +935,7 @@ extern "C" sb_status sb_tree_expand_features(const float* scores, int64_t row_st
                                              int32_t* node_rank, int32_t* topk_tok, float* topk_val, float* features,
                                              int32_t* child_row, int32_t row_base, void* workspace,
                                              size_t workspace_bytes, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_tree_expand_features");
   if (!features || row_base < 0) return SB_ERR_INVALID_ARG;
   return expand_impl(scores, row_stride, n_rows, vocab, block_k, bucket, bmap, start_parent, node_budget, n_nodes, tok,
                      parent, depth, node_row, node_rank, topk_tok, topk_val, features, child_row, row_base, workspace,
@@ -948,6 +950,7 @@ extern "C" size_t sb_rank_features_workspace_bytes(int32_t n_rows, int32_t vocab
 
 extern "C" sb_status sb_rank_features(const float* scores, int64_t row_stride, int32_t n_rows, int32_t vocab,
                                       float* features, void* workspace, size_t workspace_bytes, void* stream) {
+  sb::TraceRange trace_range("sb_rank_features");
   using namespace sb;
   if (!scores || !features || n_rows < 1 || vocab < 1 || row_stride < vocab) return SB_ERR_INVALID_ARG;
   if (n_rows > 65535) return SB_ERR_UNSUPPORTED;

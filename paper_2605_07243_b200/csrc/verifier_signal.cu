@@ -138,6 +138,7 @@ extern "C" sb_status sb_verifier_signal(const float* scores, int64_t row_stride,
                                         const int32_t* child_row, const int32_t* path_nodes,
                                         const int32_t* accept_len, const int32_t* bonus, int32_t max_depth,
                                         float* r_prob, float* signal, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_verifier_signal");
   using namespace sb;
   if (!scores || !node_offsets || !child_row || !path_nodes || !accept_len || !bonus || !r_prob || !signal ||
       !status || n_rows < 1 || vocab < 1 || batch < 1 || total_nodes < 1 || row_stride < vocab)

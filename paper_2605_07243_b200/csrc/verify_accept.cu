@@ -204,6 +204,7 @@ extern "C" sb_status sb_verify_accept(const void* logits, sb_dtype dtype, int64_
                                       int32_t* amax, int32_t* accept_len, int32_t* path_nodes,
                                       int32_t* out_tokens, int32_t* bonus, void* workspace,
                                       size_t workspace_bytes, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_verify_accept");
   using namespace sb;
   if (!logits || !node_offsets || !parent || !tok || !amax || !accept_len || !path_nodes || !out_tokens ||
       !bonus || !status || batch < 1 || total_nodes < 1 || vocab < 1 || row_stride < vocab)
@@ -252,6 +253,7 @@ extern "C" sb_status sb_verify_accept_static(const void* logits, sb_dtype dtype,
                                              const int32_t* parent, const int32_t* tok, int32_t max_depth,
                                              int32_t* amax, int32_t* accept_len, int32_t* path_nodes,
                                              int32_t* out_tokens, int32_t* bonus, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_verify_accept_static");
   using namespace sb;
   if (!logits || !node_offsets || !parent || !tok || !amax || !accept_len || !path_nodes || !out_tokens ||
       !bonus || !status || batch < 1 || total_nodes < 1 || vocab < 1 || row_stride < vocab)

@@ -559,6 +559,7 @@ extern "C" sb_status sb_verify_sample(const void* logits, sb_dtype dtype, int64_
                                       const float* u_accept, const float* u_bonus, int32_t max_depth,
                                       int32_t* accept_len, int32_t* path_nodes, int32_t* out_tokens, int32_t* bonus,
                                       void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+  sb::TraceRange trace_range("sb_verify_sample");
   using namespace sb;
   if (!logits || !scores || !node_offsets || !parent || !tok || !child_row || !u_accept || !u_bonus || !accept_len ||
       !path_nodes || !out_tokens || !bonus || !status || batch < 1 || total_nodes < 1 || vocab < 1 || n_rows < 1 ||
