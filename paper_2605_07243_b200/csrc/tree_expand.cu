@@ -26,6 +26,7 @@ namespace sb {
 constexpr int TOPK_THREADS = 256;
 constexpr int kNoId = 0x7fffffff;
 
+
 __device__ inline bool ranks_before(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
 
 // Softmax statistics of a chunk for the rank head's distribution summary (App. B): with m the
@@ -208,13 +209,14 @@ constexpr int TOPK_REG_ELEMS = TOPK_THREADS * TOPK_VEC_PER_THREAD * 4;  // 16384
 constexpr int TOPK_CAND = 512;
 constexpr int TOPK_STAGE_BYTES = TOPK_REG_ELEMS * 4;     // dynamic shared memory: the staged chunk
 
-template <bool STATS>
-__global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const float* __restrict__ scores,
-                                                                        long long row_stride, int vocab, int chunk,
-                                                                        int n_chunks, float* __restrict__ part_val,
-                                                                        int* __restrict__ part_idx,
-                                                                        float* __restrict__ part_stats, const int* __restrict__ n_nodes_in,
-    int* __restrict__ n0_snapshot) {
+// The body shared by topk_partial_reg_kernel and expand_cluster_kernel: the 16 best of one (row, chunk)
+// in order, written to out_val / out_idx (16 entries each; global memory, or a cluster peer's shared
+// memory through a generic pointer), and with STATS the chunk's (m, s, t) to stats_out.  `while_loading`
+// runs after the chunk's bulk copies have been issued and before they are awaited.  Every thread of
+// the CTA must call it (barriers inside); all threads return together.
+template <bool STATS, typename F>
+__device__ __forceinline__ void topk_reg_chunk(const float* __restrict__ base, int begin, int end,
+                                               float* out_val, int* out_idx, float* stats_out, F while_loading) {
   __shared__ float s_val[SB_KMAX][TOPK_THREADS];  // fallback lists; the candidate arrays alias them
   __shared__ int s_idx[SB_KMAX][TOPK_THREADS];
   __shared__ float s_group[16];
@@ -226,12 +228,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
   extern __shared__ float4 s_stage[];  // the chunk as it lies in memory
   float* s_cv = &s_val[0][0];
   int* s_ci = &s_idx[0][0];
-  const int row = blockIdx.y, c = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
-  const float* base = scores + (long long)row * row_stride;
-  const int begin = c * chunk;
-  const int end = min(vocab, begin + chunk);
-  pdl_release();  // the finishing kernel may start its prologue
-  if (n0_snapshot && row == 0 && c == 0 && tid == 0) *n0_snapshot = *n_nodes_in;  // the finishing kernel overwrites the counter
+  const int tid = threadIdx.x, lane = tid & 31;
   const int n_elems = max(0, end - begin);
   const int n_vec = n_elems / 4;  // whole float4s; up to 3 tail elements are handled apart
   const float4* vb = reinterpret_cast<const float4*>(base + begin);
@@ -247,6 +244,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
     for (int off = 0; off < n_vec; off += 1024)  // 16 KB pieces
       bulk_load_1d(smem_u32(s_stage + off), vb + off, (uint32_t)min(1024, n_vec - off) * 16u, &s_bar);
   }
+  while_loading();
   const bool staged = n_vec == 0 || mbar_wait(&s_bar, 0, &s_abort);  // bounded; else read global memory directly
 
   float4 x[TOPK_VEC_PER_THREAD];
@@ -285,8 +283,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
     ss = cta_reduce_sum(ss, s_red);
     tt = cta_reduce_sum(tt, s_red);
     if (tid == 0) {
-      float* o = part_stats + ((long long)row * n_chunks + c) * 3;
-      o[0] = cmax; o[1] = ss; o[2] = tt;
+      stats_out[0] = cmax; stats_out[1] = ss; stats_out[2] = tt;
     }
   }
   float gmax = tmax;
@@ -340,7 +337,6 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
   }
   __syncthreads();
   const int count = s_count;
-  const long long out0 = ((long long)row * n_chunks + c) * SB_KMAX;
   if (count <= TOPK_CAND) {
     // rank of candidate a = number of candidates that come before it; four threads share one
     // candidate (a quarter of the comparisons each, combined by shuffles)
@@ -354,9 +350,9 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
         for (int b2 = tid & 3; b2 < count; b2 += 4) r += ranks_before(s_cv[b2], s_ci[b2], v, id) ? 1 : 0;
       r += __shfl_xor_sync(0xffffffffu, r, 1);
       r += __shfl_xor_sync(0xffffffffu, r, 2);
-      if (live && (tid & 3) == 0 && r < SB_KMAX) { part_val[out0 + r] = v; part_idx[out0 + r] = id; }
+      if (live && (tid & 3) == 0 && r < SB_KMAX) { out_val[r] = v; out_idx[r] = id; }
     }
-    if (tid < SB_KMAX && tid >= count) { part_val[out0 + tid] = -INFINITY; part_idx[out0 + tid] = kNoId; }
+    if (tid < SB_KMAX && tid >= count) { out_val[tid] = -INFINITY; out_idx[tid] = kNoId; }
     return;
   }
   // ---- massive ties: per-thread sorted lists (ids ascend inside a thread), then ordered pops ----
@@ -410,13 +406,31 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const fl
       int bi = s_wi[0], bt = s_wt[0];
       for (int w = 1; w < TOPK_THREADS / 32; ++w)
         if (ranks_before(s_wv[w], s_wi[w], bv, bi)) { bv = s_wv[w]; bi = s_wi[w]; bt = s_wt[w]; }
-      part_val[out0 + round] = bv;
-      part_idx[out0 + round] = bi;
+      out_val[round] = bv;
+      out_idx[round] = bi;
       s_winner = bi == kNoId ? -1 : bt;
     }
     __syncthreads();
     if (tid == s_winner) ++pos;
   }
+}
+
+template <bool STATS>
+__global__ void __launch_bounds__(TOPK_THREADS) topk_partial_reg_kernel(const float* __restrict__ scores,
+                                                                        long long row_stride, int vocab, int chunk,
+                                                                        int n_chunks, float* __restrict__ part_val,
+                                                                        int* __restrict__ part_idx,
+                                                                        float* __restrict__ part_stats, const int* __restrict__ n_nodes_in,
+                                                                        int* __restrict__ n0_snapshot) {
+  const int row = blockIdx.y, c = blockIdx.x;
+  const float* base = scores + (long long)row * row_stride;
+  const int begin = c * chunk;
+  const int end = min(vocab, begin + chunk);
+  pdl_release();  // the finishing kernel may start its prologue
+  if (n0_snapshot && row == 0 && c == 0 && threadIdx.x == 0) *n0_snapshot = *n_nodes_in;  // the finishing kernel overwrites the counter
+  const long long out0 = ((long long)row * n_chunks + c) * SB_KMAX;
+  topk_reg_chunk<STATS>(base, begin, end, part_val + out0, part_idx + out0,
+                        STATS ? part_stats + ((long long)row * n_chunks + c) * 3 : nullptr, []() {});
 }
 
 constexpr int FINISH_THREADS = 1024;
@@ -734,6 +748,181 @@ __global__ void __launch_bounds__(ROWS_THREADS) expand_rows_kernel(
   }
 }
 
+// ---- scan and finish in ONE kernel: the chunk CTAs of a row are a thread-block cluster -------------------
+// For rows whose chunks fit the register-resident scan and one cluster (at most 16 chunks): every CTA takes
+// the 16 best of its chunk exactly as topk_partial_reg_kernel does, but writes them into the shared memory of
+// the cluster's first CTA (distributed shared memory) instead of a workspace; after one cluster barrier that
+// CTA ranks the row's candidates and writes the row's top-16 and its own nodes, as expand_rows_kernel does.
+// No chunk lists travel through global memory and no second grid has to start before a row is finished.
+// The branching structure (which rows are alive, where their nodes go) depends on the inputs alone and is
+// derived by the first CTA while its chunk is in flight.  The node counter is only READ here (by every
+// finishing CTA, whenever it starts): the new count and the status word are written by expand_commit_kernel,
+// a one-warp programmatic dependent that starts after this whole grid has completed, so no CTA of this grid
+// can ever see the counter already advanced.
+constexpr int XC_MAX_CHUNKS = 16;
+
+__global__ void __launch_bounds__(TOPK_THREADS) expand_cluster_kernel(
+    const float* __restrict__ scores, long long row_stride, int vocab, int chunk, int n_rows, int block_k,
+    const uint8_t* __restrict__ bucket, int4 bmap, const int* __restrict__ start_parent, int node_budget,
+    const int* __restrict__ n_nodes, int* __restrict__ tok, int* __restrict__ parent, int* __restrict__ depth,
+    int* __restrict__ node_row, int* __restrict__ node_rank, int* __restrict__ topk_tok, float* __restrict__ topk_val,
+    int* __restrict__ child_row, int row_base, int* __restrict__ commit, int* __restrict__ status) {
+  static_assert(ROWS_THREADS == TOPK_THREADS, "the row structure is derived with the scan's block size");
+  __shared__ float s_cand_val[XC_MAX_CHUNKS * SB_KMAX];  // the row's chunk lists: written by the cluster's CTAs
+  __shared__ int s_cand_idx[XC_MAX_CHUNKS * SB_KMAX];
+  __shared__ __align__(16) unsigned long long s_key[XC_MAX_CHUNKS * SB_KMAX];
+  __shared__ int s_rank[XC_MAX_CHUNKS * SB_KMAX];
+  __shared__ int s_warp_sum[ROWS_THREADS / 32];
+  __shared__ int s_my[3];  // this row: first id (relative), width, the previous row's first id (relative)
+  cg::cluster_group cluster = cg::this_cluster();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int c = blockIdx.x, rr = blockIdx.y;  // the cluster spans x: c is also the rank in the cluster
+  const int n_chunks = gridDim.x;
+  const int n_cand = n_chunks * SB_KMAX;
+  const float* base = scores + (long long)rr * row_stride;
+  const int begin = c * chunk;
+  const int end = min(vocab, begin + chunk);
+  pdl_release();  // expand_commit_kernel may take its place; it waits for this grid before it reads or writes
+
+  auto width_of_bucket = [&](int bk) {
+    const int w = bk == 0 ? bmap.x : bk == 1 ? bmap.y : bk == 2 ? bmap.z : bmap.w;
+    return w < vocab ? w : vocab;
+  };
+  bool bad = false;
+  int total = 0, n0 = 0, start = -1, start_depth = 0;
+  auto structure = [&]() {
+    if (c != 0) return;
+    // inputs only: widths of all rows, their prefix sums, this row's share (as in expand_rows_kernel)
+    const int rpt = ceil_div(n_rows, ROWS_THREADS);  // consecutive rows per thread (<= 4)
+    int w_loc[4] = {0, 0, 0, 0};
+    int wsum = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = tid * rpt + i;
+      if (i < rpt && r < n_rows) {
+        const int kpos = r % block_k;
+        const int bk = bucket[r];
+        bad = bad || bk > 3;
+        bool alive = true;
+        for (int k = 1; k <= kpos; ++k) alive = alive && width_of_bucket(bucket[r - k]) >= 1;
+        w_loc[i] = alive ? width_of_bucket(bk) : 0;
+        wsum += w_loc[i];
+      }
+    }
+    n0 = *n_nodes;  // the count before this call: nothing in this grid writes it
+    bad = bad || n0 < 0 || n0 > node_budget;
+    const int n_starts = n_rows / block_k;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (tid + i * ROWS_THREADS < n_starts) {
+        const int sp = start_parent[tid + i * ROWS_THREADS];
+        bad = bad || sp < -1 || sp >= n0;
+      }
+    start = start_parent[rr / block_k];
+    start_depth = (start >= 0 && start < node_budget) ? depth[start] : 0;  // an existing node: never rewritten
+    int incl = wsum;
+#pragma unroll
+    for (int sft = 1; sft < 32; sft <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, sft);
+      if (lane >= sft) incl += o;
+    }
+    if (lane == 31) s_warp_sum[warp] = incl;
+    for (int k = tid; k < n_cand; k += ROWS_THREADS) s_rank[k] = 0;
+    __syncthreads();
+    int run = incl - wsum;
+    for (int w = 0; w < warp; ++w) run += s_warp_sum[w];
+    for (int w = 0; w < ROWS_THREADS / 32; ++w) total += s_warp_sum[w];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = tid * rpt + i;
+      if (i < rpt) {
+        if (r == rr) { s_my[0] = run; s_my[1] = w_loc[i]; }
+        if (r == rr - 1) s_my[2] = run;
+        run += w_loc[i];
+      }
+    }
+  };
+  // the 16 best of this chunk, straight into the first CTA's candidate arrays
+  float* out_val = cluster.map_shared_rank(s_cand_val, 0) + c * SB_KMAX;
+  int* out_idx = cluster.map_shared_rank(s_cand_idx, 0) + c * SB_KMAX;
+  topk_reg_chunk<false>(base, begin, end, out_val, out_idx, nullptr, structure);
+  cluster.sync();  // every chunk's list has landed in the first CTA
+  if (c != 0) return;
+
+  // ---- merge this row's chunk lists (as expand_rows_kernel) -------------------------------------------------
+  for (int k = tid; k < n_cand; k += ROWS_THREADS) {
+    float v = s_cand_val[k];
+    const int id = s_cand_idx[k];
+    if (!(v == v)) v = -INFINITY;
+    uint32_t u = __float_as_uint(v == 0.f ? 0.f : v);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    const uint32_t low = id == kNoId ? 0x7fffffffu - (uint32_t)k : 0xffffffffu - (uint32_t)id;
+    s_key[k] = ((unsigned long long)u << 32) | low;
+  }
+  const int any_bad = __syncthreads_or(bad ? 1 : 0);  // also publishes the keys
+  {
+    const int parts = n_cand <= ROWS_THREADS ? ROWS_THREADS / n_cand : 1;
+    const int n_pairs = n_cand / 2;
+    const int per = ceil_div(n_pairs, parts);
+    const ulonglong2* kp = reinterpret_cast<const ulonglong2*>(s_key);
+    for (int w = tid; w < n_cand * parts; w += ROWS_THREADS) {
+      const int k = w % n_cand, part = w / n_cand;
+      const unsigned long long key = s_key[k];
+      const int hi = min(n_pairs, (part + 1) * per);
+      int cnt = 0;
+#pragma unroll 2
+      for (int o = part * per; o < hi; ++o) {
+        const ulonglong2 k2 = kp[o];
+        cnt += (k2.x > key ? 1 : 0) + (k2.y > key ? 1 : 0);
+      }
+      if (cnt) atomicAdd(&s_rank[k], cnt);
+    }
+  }
+  __syncthreads();
+  const int first = n0 + s_my[0], width = s_my[1];
+  const int kpos = rr % block_k;
+  const int par = kpos == 0 ? start : n0 + s_my[2];  // the rank-0 node of the previous position
+  const int node_depth = (start == -1 ? 0 : start_depth + 1) + kpos;
+  for (int k = tid; k < n_cand; k += ROWS_THREADS) {
+    const int rank = s_rank[k];
+    if (rank >= SB_KMAX) continue;
+    const uint32_t low = (uint32_t)s_key[k];
+    const int id = low < 0x80000000u ? -1 : (int)(0xffffffffu - low);
+    topk_tok[rr * SB_KMAX + rank] = id;
+    topk_val[rr * SB_KMAX + rank] = s_cand_val[k];
+    if (!any_bad && rank < width && first + rank < node_budget && SB_CHECKED_ACCESS(first + rank, node_budget, status)) {
+      const int n = first + rank;
+      tok[n] = id;
+      parent[n] = par;
+      depth[n] = node_depth;
+      node_row[n] = row_base + rr;
+      node_rank[n] = rank;
+    }
+  }
+  if (tid == 0 && child_row && !any_bad && width > 0 && first < node_budget && par >= 0 &&
+      SB_CHECKED_ACCESS(par, node_budget, status))
+    child_row[par] = row_base + rr;
+  if (rr == 0 && tid == 0) {  // what expand_commit_kernel publishes once the whole grid is done
+    const int n_new = n0 + total;
+    commit[0] = any_bad ? -1 : (n_new < node_budget ? n_new : node_budget);
+  }
+}
+
+// One warp, a programmatic dependent of expand_cluster_kernel: the new node count and the status word.
+__global__ void expand_commit_kernel(const int* __restrict__ commit, int* __restrict__ n_nodes, int* __restrict__ status) {
+  pdl_release();
+  pdl_wait();  // every CTA of the expansion grid has completed (and has read the old count)
+  if (threadIdx.x == 0) {
+    const int n_new = commit[0];
+    if (n_new < 0) {
+      *status = SB_ERR_INVALID_ARG;
+    } else {
+      *n_nodes = n_new;
+      *status = SB_OK;
+    }
+  }
+}
+
 // psi(p) of every row from the chunk partials: a warp per row merges the chunk lists (value
 // descending, id ascending) and the chunk statistics (m, s, t):  M = max m_c,
 // S = sum s_c e^(m_c - M), T = sum t_c e^(m_c - M); ln Z = M + ln S; entropy = ln Z - T / S.
@@ -837,12 +1026,57 @@ static size_t topk_stage_bytes(int chunk) {
   static PerDeviceOnce once;
   once.run([]() {
     const bool ok =
+        cudaFuncSetAttribute(expand_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TOPK_STAGE_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(expand_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
         cudaFuncSetAttribute(topk_partial_reg_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TOPK_STAGE_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(topk_partial_reg_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TOPK_STAGE_BYTES) == cudaSuccess;
     if (!ok) cudaGetLastError();
     return ok;  // a failure shows as a launch error of the scan
   });
   return (size_t)chunk * sizeof(float);
+}
+
+// Launch configuration of expand_cluster_kernel for `nc` chunks per row.
+static cudaLaunchConfig_t expand_cluster_config(dim3 grid, int nc, size_t smem, cudaStream_t cs, cudaLaunchAttribute* attr) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(TOPK_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = cs;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = nc;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cfg;
+}
+
+// Clusters of `nc` CTAs of expand_cluster_kernel that can be resident at once on the current device.
+static int expand_cluster_fit(int nc) {
+  static PerDeviceInt cache[XC_MAX_CHUNKS + 1];
+  if (nc < 1 || nc > XC_MAX_CHUNKS) return 0;
+  return cache[nc].get([&]() {
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = expand_cluster_config(dim3(nc, 64), nc, topk_stage_bytes(TOPK_REG_ELEMS), nullptr, attr);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, expand_cluster_kernel, &cfg) != cudaSuccess) {
+      cudaGetLastError();
+      n = 0;
+    }
+    return n;
+  }, 0);
+}
+
+// Chunks per row for expand_cluster_kernel: as many as topk_chunks() wants while all rows' clusters are
+// resident together (288 CTAs in clusters of 9 do not fit a B200, 256 in clusters of 8 do), never fewer
+// than the register-resident scan needs.
+static int expand_cluster_chunks(int n_rows, int vocab) {
+  const int reg_nc = ceil_div(vocab, TOPK_REG_ELEMS);
+  int nc = topk_chunks(n_rows, vocab);
+  if (nc > XC_MAX_CHUNKS) nc = XC_MAX_CHUNKS;
+  while (nc > reg_nc && expand_cluster_fit(nc) < n_rows) --nc;
+  return nc;
 }
 
 }  // namespace sb
@@ -885,6 +1119,23 @@ static sb_status expand_impl(const float* scores, int64_t row_stride, int32_t n_
   int* snap = by_rows ? n0_snapshot : nullptr;
   dim3 grid(nc, n_rows);
   const bool reg = vec_ok && chunk <= TOPK_REG_ELEMS;
+  if (vec_ok && !features && by_rows && ceil_div(vocab, TOPK_REG_ELEMS) <= XC_MAX_CHUNKS) {
+    // scan and finish in one grid: the chunks of a row are a cluster (expand_cluster_kernel), then a one-warp commit
+    const int ncc = expand_cluster_chunks(n_rows, vocab);
+    const int cchunk = ceil_div(ceil_div(vocab, ncc), 4) * 4;
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = expand_cluster_config(dim3(ncc, n_rows), ncc, topk_stage_bytes(cchunk), cs, attr);
+    if (cudaLaunchKernelEx(&cfg, expand_cluster_kernel, scores, (long long)row_stride, (int)vocab, cchunk, (int)n_rows,
+                           (int)block_k, bucket, make_int4(bmap[0], bmap[1], bmap[2], bmap[3]), start_parent,
+                           (int)node_budget, (const int*)n_nodes, tok, parent, depth, node_row, node_rank, topk_tok,
+                           topk_val, child_row, (int)row_base, n0_snapshot, status) != cudaSuccess) {
+      cudaGetLastError();
+      return SB_ERR_CUDA;
+    }
+    sb_status st1 = launch_check();
+    if (st1 != SB_OK) return st1;
+    return launch_dependent(expand_commit_kernel, dim3(1), dim3(32), cs, (const int*)n0_snapshot, n_nodes, status);
+  }
   if (reg && features)
     topk_partial_reg_kernel<true><<<grid, TOPK_THREADS, topk_stage_bytes(chunk), cs>>>(scores, row_stride, vocab, chunk, nc,
                                                                                     part_val, part_idx, part_stats, n_nodes, snap);

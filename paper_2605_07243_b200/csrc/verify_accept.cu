@@ -52,6 +52,9 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) row_argmax_kernel(const T* __r
   pdl_release();  // the path kernel may start its prologue
   Best best = {-INFINITY, 0x7fffffff};
   if (vec_ok) {
+    // four independent running maxima (one per load slot modulo 4): the compare-select chain of a single
+    // maximum is a serial dependency of 64 steps per sweep; ids still ascend inside each of the four
+    Best acc[4] = {{-INFINITY, 0x7fffffff}, {-INFINITY, 0x7fffffff}, {-INFINITY, 0x7fffffff}, {-INFINITY, 0x7fffffff}};
     // chunk is a multiple of VEC and rows are 16-byte aligned
     const int n_vec = max(0, (end - begin) / VEC);
     const uint4* vb = reinterpret_cast<const uint4*>(base + begin);
@@ -71,11 +74,14 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) row_argmax_kernel(const T* __r
           for (int u = 0; u < VEC; ++u) {
             const float x = logit_to_float<T>(e[u]);
             const int id = begin + (t0 + q * ARGMAX_THREADS) * VEC + u;
-            if (x > best.v) { best.v = x; best.i = id; }  // ids ascend inside a thread: strict keeps the first
+            if (x > acc[q & 3].v) { acc[q & 3].v = x; acc[q & 3].i = id; }  // ids ascend inside a slot: strict keeps the first
           }
         }
       }
     }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+      if (better(acc[a].v, acc[a].i, best.v, best.i)) best = acc[a];
     for (int id = begin + n_vec * VEC + threadIdx.x; id < end; id += ARGMAX_THREADS) {
       const float x = logit_to_float<T>(base[id]);
       if (x > best.v) { best.v = x; best.i = id; }

@@ -115,6 +115,35 @@ class VerifyStep:
                           tree, workspace=e["ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"],
                           status=e["status"])
 
+    COLD_SETS = 17   # copies of the 15-16 MB score / logit matrices walked by the *_cold runs: > 2 x L2 in total
+
+    def run_expand_cold(self):
+        """sb_tree_expand once per copy of the score matrix (COLD_SETS copies, more than twice the L2 size
+        together), each call on its own tree arrays: every call streams its scores from HBM, as it does in
+        a real iteration where the scores were just produced by another kernel's pass over other data."""
+        e = self.expand
+        if e is None:
+            return
+        if "cold" not in e:
+            e["cold"] = [dict(scores=e["scores"].clone(), tree={k: t.clone() for k, t in e["tree0"].items()})
+                         for _ in range(self.COLD_SETS)]
+            e["cold_n_nodes"] = torch.full((self.COLD_SETS,), e["n0"], dtype=torch.int32, device=self.device)
+            e["cold_n_nodes0"] = e["cold_n_nodes"].clone()
+        e["cold_n_nodes"].copy_(e["cold_n_nodes0"])      # one reset for the whole walk
+        for i, c in enumerate(e["cold"]):
+            tree = dict(c["tree"], n_nodes=e["cold_n_nodes"][i:i + 1])
+            sb.sb_tree_expand(c["scores"], e["block_k"], e["bucket"], e["bmap"], e["start_parent"], e["budget"],
+                              tree, workspace=e["ws"], topk_tok=e["topk_tok"], topk_val=e["topk_val"],
+                              status=e["status"])
+
+    def run_accept_cold(self):
+        """sb_verify_accept once per copy of the logits (COLD_SETS copies, more than twice the L2 size)."""
+        if not hasattr(self, "logits_cold"):
+            self.logits_cold = [self.logits.clone() for _ in range(self.COLD_SETS)]
+        for lg in self.logits_cold:
+            sb.sb_verify_accept(lg, self.tb.node_offsets, self.tb.parent, self.tok, self.max_depth,
+                                workspace=self.accept_ws, out=self.accept)
+
     def run_rank_features(self):
         """psi(p) of every drafter row (not part of run_device(): a 'next' row, timed on its own)."""
         e = self.expand
