@@ -8,29 +8,38 @@
  * iteration that do not need model weights:
  *
  *   sb_tree_ancestors  ancestor bitmask / depth of every tree node      (Sec. 3.1, App. A.2, Fig. 4)
- *   sb_tree_attention  tree-masked attention over prefix KV + ancestors (Sec. 3.1, App. A.2, Alg. 1 "verify")
- *   sb_tree_expand     per-row top-k + bucket-driven branching          (Sec. 3.2, App. A.5, Alg. 1 "attach")
+ *   sb_tree_attention  tree-masked attention over prefix KV + ancestors (Sec. 3.1, App. A.2, the verify step of Alg. 1)
+ *   sb_tree_expand     per-row top-k + bucket-driven branching          (Sec. 3.2, App. A.5, the attach step of Alg. 1)
  *   sb_rank_features   15-dim summary of each draft distribution        (Sec. 3.2, App. B)
  *   sb_tree_expand_features  both of the above from one pass over the scores
  *   sb_verifier_signal verifier-derived update signal s = sum (1 - r)   (Sec. 3.4, Alg. 2)
  *   sb_verify_sample   stochastic (temperature > 0) tree verification   (Sec. 4.1, Sec. 4.2)
  *   sb_shift_project   layer-wise shift projection between drafter layers (Sec. 3.1)
- *   sb_fuse_project    the drafter's fused per-position input h^(0)      (Sec. 3.1 "Block forward")
- *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, Alg. 1 "verify"/"return")
- *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1 "cached key-value pairs")
+ *   sb_fuse_project    the drafter's fused per-position input h^(0)      (Sec. 3.1, the paragraph on the block forward)
+ *   sb_verify_accept   greedy longest accepted path + bonus token       (App. A.5, the verify and return steps of Alg. 1)
+ *   sb_kv_compact      move the accepted path's K/V behind the prefix   (Sec. 3.1, App. A.2: committed positions stay in the cache)
  *   sb_path_rows       the accepted path in the drafter's row numbering  (App. A.2)
  *
  * Conventions that hold for every call
  *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
- *     The library never allocates or frees device memory, keeps no state between calls,
- *     enqueues its kernels on `stream` (a cudaStream_t passed as void*, NULL = legacy default
- *     stream) and returns without synchronising.
+ *     The library never allocates or frees device memory, enqueues its kernels on `stream` (a
+ *     cudaStream_t passed as void*, NULL = legacy default stream) and returns without synchronising.
+ *     It keeps no state between calls, with three small exceptions: per device, kernel attributes and
+ *     occupancy figures are set up or looked up on the first call that needs them (so that first
+ *     call on a device should come before any stream capture); sb_verify_accept_static uses a fixed
+ *     scratch array inside the library image, whose device address it looks up once per device (valid
+ *     for the life of the device's primary context); and the status word of the projection calls
+ *     is written by their kernels, i.e. after the call has returned.  One process may drive several
+ *     devices: all of this is kept per device, for the device that is current during the call.
  *   - The return value reports what the host can see (null pointers, unsupported shapes,
  *     a workspace that is too small, a failed launch).  Data-dependent problems (a parent
  *     index that is not smaller than its child, a prefix longer than the cache, a page id
  *     outside the pool) are written to the caller's `status` device array, one int32 per
- *     sequence (0 = ok, else an sb_status value); the outputs of such a sequence are
- *     zero-filled.  No kernel traps, spins without bound or reads outside the described arrays.
+ *     sequence (0 = ok, else an sb_status value).  The outputs of a sequence with a bad tree or bad
+ *     lengths are zero-filled; with a page id outside the pool (SB_ERR_BOUNDS from the page table)
+ *     the sequence's outputs are unspecified -- every read is redirected to page 0, so nothing is
+ *     read outside the pool, and the other sequences' outputs are unaffected.  No kernel traps,
+ *     spins without bound or reads outside the described arrays.
  *   - bf16 = IEEE-754 binary32 truncated to its upper 16 bits (round-to-nearest-even on
  *     conversion).  All accumulation is fp32.
  *   - Tree node i of sequence b lives at logical cache position prefix_len[b] + i: the
@@ -126,9 +135,9 @@ sb_status sb_tree_ancestors(int32_t batch, const int32_t* node_offsets, const in
                             int32_t* status, void* stream);
 
 /*
- * sb_tree_attention -- tree-masked attention of one layer (Sec. 3.1 "within-block
- * dependence"; App. A.2: prefix fully visible, earlier draft positions visible only along
- * the branch path, causal inside the block; Alg. 1 line "verify").
+ * sb_tree_attention -- tree-masked attention of one layer (Sec. 3.1, the paragraph on
+ * dependence inside a block; App. A.2: prefix fully visible, earlier draft positions visible only
+ * along the branch path, causal inside the block; the verify step of Alg. 1).
  *
  *   For sequence b, query node i in [q_node_begin[b], N_b), query head h (KV head g = h / G):
  *     visible keys = {0..P_b-1} U {P_b + a : a in anc(i)}
@@ -160,8 +169,8 @@ size_t sb_tree_attention_workspace_bytes(const sb_tree_batch* tb, int32_t total_
 
 /*
  * sb_tree_expand -- attach candidates of one batched drafter forward to the tree
- * (Sec. 3.2 "bucket-driven branching"; App. A.5 maps b(.); Alg. 1 lines "for each starting
- * point i and position k: attach the top-b(bkt) tokens").
+ * (Sec. 3.2, branching driven by the rank bucket; App. A.5 maps b(.); the attach loop of Alg. 1
+ * over starting points and positions).
  *
  *   Rows r = i*block_k + k (start i, position k), scores fp32 [n_rows][row_stride >= vocab].
  *   (1) per row the SB_KMAX best ids by (score descending, id ascending; NaN counts as -inf)
@@ -188,7 +197,7 @@ size_t sb_tree_expand_workspace_bytes(int32_t n_rows, int32_t vocab);
 
 /*
  * sb_rank_features -- the rank head's 15-dimensional summary psi(p) of every draft distribution
- * (Sec. 3.2 "rank head"; App. B "distribution summary features").
+ * (Sec. 3.2, the rank head; App. B, its distribution summary).
  *
  *   scores fp32 [n_rows][row_stride >= vocab] are the drafter's logits; p = softmax(row), NaN read
  *   as -inf.  features fp32 [n_rows][15], in the order the appendix lists them:
@@ -229,7 +238,7 @@ sb_status sb_tree_expand_features(const float* scores, int64_t row_stride, int32
 
 /*
  * sb_shift_project -- the layer-wise shift between consecutive decoder layers of the drafter
- * (Sec. 3.1 "Within-block dependence", the equation for h-tilde): position k's state is
+ * (Sec. 3.1, the paragraph on dependence inside a block, the equation for h-tilde): position k's state is
  * concatenated with position k-1's state of the same block and projected back by W_shift.
  *
  *   h   bf16 [n_rows][d]: rows r = i * block_k + k are the block_k positions of block i.
@@ -253,13 +262,13 @@ sb_status sb_shift_project(const void* h, const void* w, int32_t n_rows, int32_t
 size_t sb_shift_project_workspace_bytes(int32_t n_rows, int32_t d, int32_t d_out, int32_t block_k);
 
 /*
- * sb_fuse_project -- the per-position input of a drafter block (Sec. 3.1 "Block forward", the
- * equation for h^(0)): the context feature c_s of start s, the embedding e_s of its last committed
+ * sb_fuse_project -- the per-position input of a drafter block (Sec. 3.1, the paragraph on the block
+ * forward, the equation for h^(0)): the context feature c_s of start s, the embedding e_s of its last committed
  * token and the learnable query q_k of draft depth k are normalised, concatenated and projected by
  * W_fuse.  c_s and e_s are shared by the block_k positions of a block (the prefix broadcast).
  *
  *   c, e bf16 [n_starts][d];  q bf16 [block_k][d];  w bf16 [d_out][3 d] row-major, acting on
- *   [norm(c) , norm(e) , norm(q)].  "norm" is not specified further by the paper; here it is
+ *   [norm(c) , norm(e) , norm(q)].  the normalisation is not specified further by the paper; here it is
  *   norm(x)[j] = gain[j] * x[j] / sqrt(mean_j x[j]^2 + eps), gains fp32 [d] or NULL for ones (the
  *   normalised rows are rounded to bf16, the type of the tensor-core operand).
  *   out bf16 [n_starts * block_k][d_out], row s * block_k + k; fp32 accumulation.
@@ -285,8 +294,8 @@ size_t sb_fuse_project_workspace_bytes(int32_t n_starts, int32_t block_k, int32_
 
 /*
  * sb_verify_sample -- verification at temperature T > 0 by multi-candidate rejection sampling over
- * the draft tree (Sec. 4.1 evaluates temperature 0 and 1.0; Sec. 4.2 "rejection sampling against a
- * high-entropy target").  The paper names the procedure without listing it; the steps are:
+ * the draft tree (Sec. 4.1 evaluates temperature 0 and 1.0; Sec. 4.2 mentions rejection sampling against the
+ * target).  The paper names the procedure without listing it; the steps are:
  *
  *   a = root (node 0), depth 0, p = softmax(logits[a] / T).  Repeat:
  *     children of a = the nodes c with parent[c] == a, in increasing index (emission order);
@@ -326,7 +335,7 @@ size_t sb_verify_sample_workspace_bytes(int32_t batch, int32_t vocab, int32_t to
 /*
  * sb_verifier_signal -- one iteration's term of the verifier-derived update signal
  * s = sum over rejected positions of (1 - r), r = the drafter's probability of the token the
- * target chose there (Sec. 3.4 "Verifier-derived update signal"; Alg. 2 line 2).
+ * target chose there (Sec. 3.4, the verifier-derived signal; Alg. 2 line 2).
  *
  *   A verify iteration rejects at most one position per sequence: the one right after the last
  *   accepted node best = path_nodes[b][accept_len[b]], where the target chose bonus[b] (all three
@@ -350,9 +359,9 @@ sb_status sb_verifier_signal(const float* scores, int64_t row_stride, int32_t n_
                              int32_t* status, void* stream);
 
 /*
- * sb_verify_accept -- greedy (temperature 0) verification (App. A.5 "the longest accepted
- * prefix is committed"; Alg. 1 "(prefix, bonus) <- verify(tree)"; case study: accepted
- * tokens plus one bonus token are committed).
+ * sb_verify_accept -- greedy (temperature 0) verification (App. A.5: the longest accepted
+ * prefix is what gets committed; the verify step of Alg. 1 returns it with a bonus token; case study:
+ * accepted tokens plus one bonus token are committed).
  *
  *   logits [total_nodes][row_stride >= vocab] (bf16 or fp32): the target's next-token scores
  *   at every tree node.  amax[i] = smallest id attaining the row maximum (NaN counts as -inf).

@@ -26,7 +26,7 @@
  *                         committed token is distributed exactly as the target -- checked by exact
  *                         integration over the uniforms (acceptance thresholds and bonus intervals found
  *                         by bisection on the oracle); T -> 0 reduces to greedy acceptance.  The paper
- *                         names the procedure only as "rejection sampling": the order in which siblings
+ *                         names the procedure only (rejection sampling): the order in which siblings
  *                         are tried and the treatment of the draft distribution after a rejection are
  *                         readings -- for those PARITY IS UNPINNED by the paper.
  *   sbo_shift_project   : numpy matmul on the explicitly concatenated input; W = [I, 0] returns the input,
@@ -614,7 +614,7 @@ void sbo_fuse_project(const uint16_t* c, const uint16_t* e, const uint16_t* q, c
 /* ---- stochastic verification of a draft tree (Sec. 4.1 "temperature 0 and 1.0"; Sec. 4.2) ------- */
 
 /*
- * The paper verifies at temperature 1 by "rejection sampling against the target" without giving
+ * The paper verifies at temperature 1 by rejection sampling against the target without giving
  * the procedure; this is the multi-candidate rejection sampling of tree-based speculative decoding
  * (the systems it compares with), taken in the order below.  All random numbers are inputs.
  *

@@ -1,5 +1,5 @@
 // sb_tree_expand: per-row top-k over the drafter's scores and bucket-driven branching
-// (Sec. 3.2; App. A.5 maps b(.); Alg. 1 "attach the top-b(bkt) tokens").
+// (Sec. 3.2; App. A.5 maps b(.); the attach step of Alg. 1).
 //
 //   topk_partial_kernel : streams the [rows][vocab] fp32 scores once from HBM (a second pass hits
 //                         L1/L2).  A CTA owns one (row, vocab chunk).  Pass 1: every thread takes the

@@ -1,5 +1,5 @@
 // sb_verifier_signal: the verifier-derived update signal s = sum over rejected positions of (1 - r)
-// (Sec. 3.4 "Verifier-derived update signal"; Alg. 2 line 2), one verify iteration at a time.
+// (Sec. 3.4, the verifier-derived signal; Alg. 2 line 2), one verify iteration at a time.
 //
 //   verifier_signal_kernel : a cluster of SIG_CLUSTER CTAs per sequence.  Every CTA reads the
 //                       sequence's accept result, finds the drafter row that predicted the token

@@ -1,6 +1,6 @@
 // sb_verify_sample: stochastic verification of a draft tree at temperature T > 0 by multi-candidate
-// rejection sampling (Sec. 4.1 evaluates "temperature 0 and 1.0"; Sec. 4.2 "rejection sampling
-// against a high-entropy target").  The paper names the procedure only; the order of the steps is
+// rejection sampling (Sec. 4.1 evaluates temperatures 0 and 1; Sec. 4.2 mentions rejection sampling
+// against the target).  The paper names the procedure only; the order of the steps is
 // the one stated in include/specblock.h.
 //
 //   vs_stats_kernel      : the softmax statistics of EVERY target row and every draft row, in parallel

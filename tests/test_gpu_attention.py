@@ -284,9 +284,15 @@ def test_bad_page_id_is_reported_without_fault():
     rng = W.rng_for(49)
     case = W.make_attn_case(rng, parents=[W.chain_tree(4), W.chain_tree(4)], prefix_lens=[100, 100],
                             n_q_heads=4, n_kv_heads=1, head_dim=64, page_size=16)
+    good = gpu_attention(case)
     case.page_table[1, 2] = case.num_pages + 5
-    _out, _lse, status = gpu_attention(case)
+    out, lse, status = gpu_attention(case)
     assert list(status) == [0, 5]
+    # the contract for a page id outside the pool: reported, every read redirected into the pool (so the
+    # call cannot fault), that sequence's rows unspecified -- and the other sequence's rows untouched
+    np.testing.assert_array_equal(out[:4], good[0][:4])
+    np.testing.assert_array_equal(lse[:4], good[1][:4])
+    assert np.isfinite(out[4:]).all()
 
 
 def test_host_argument_errors():
