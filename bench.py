@@ -41,7 +41,7 @@ N_LAYERS = 32
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of this workload, from an ncu
 # capture of the library as committed (the summary of that capture is committed with the profiles)
-ATTN_DRAM_TRAFFIC_BYTES = 9189120
+ATTN_DRAM_TRAFFIC_BYTES = 9183232
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_TFLOPS = 1400.0   # sustained dense bf16
 
@@ -308,12 +308,14 @@ def run_ours(args):
         g_attn = capture(torch, step.run_attention)
         g_expand = capture(torch, step.run_expand)
         g_accept = capture(torch, step.run_accept)
-        step.run_expand_cold()
-        step.run_accept_cold()
-        side.synchronize()
-        assert int(step.expand["cold_n_nodes"].min()) == int(step.expand["n_nodes"][0])
-        g_expand_cold = capture(torch, step.run_expand_cold)
-        g_accept_cold = capture(torch, step.run_accept_cold)
+        g_expand_cold = g_accept_cold = None
+        if not args.step_only:
+            step.run_expand_cold()
+            step.run_accept_cold()
+            side.synchronize()
+            assert int(step.expand["cold_n_nodes"].min()) == int(step.expand["n_nodes"][0])
+            g_expand_cold = capture(torch, step.run_expand_cold)
+            g_accept_cold = capture(torch, step.run_accept_cold)
         g_compact = capture(torch, step.run_compact)
         extras = []   # pieces outside the step (the "next" rows), timed on their own
         if not args.step_only:
@@ -370,8 +372,9 @@ def run_ours(args):
         # call each, so every call streams its matrix from HBM and the replay's own cost (about 4 us) is shared by all
         # of them -- what a call costs inside an iteration; the *_single_call_graph entries replay ONE call on the same
         # matrix (L2-warm, the whole replay cost on it), as round 1 reported them
-        for name, g in [("expand", g_expand_cold), ("accept", g_accept_cold), ("expand_single_call_graph", g_expand),
-                        ("accept_single_call_graph", g_accept), ("compact", g_compact)] + extras:
+        cold = [] if args.step_only else [("expand", g_expand_cold), ("accept", g_accept_cold)]
+        for name, g in cold + [("expand_single_call_graph", g_expand), ("accept_single_call_graph", g_accept),
+                               ("compact", g_compact)] + extras:
             # short graphs: ten replays per sample keep the event pair's own cost out of the figure
             reps = 1 if name.startswith("whole_iteration") or name in ("expand", "accept") else 10
             parts_stats[name] = sample_graph(torch, g, n_samples, reps, calls.get(name, 1))
@@ -486,11 +489,25 @@ def main():
                     help="also time the CPU oracle's tree attention on these benchmark configurations (e.g. 1,2,3,4,5)")
     ap.add_argument("--step-only", action="store_true",
                     help="profiling aid: leave out the pieces timed outside the step (their kernels then do not appear)")
+    ap.add_argument("--attention-config", default="",
+                    help="profiling aid: time sb_tree_attention on ONE benchmark configuration and print its entry of "
+                         "the \"configs\" key, e.g. 5 or 5:16 (configuration:num_splits); nothing else runs")
+    ap.add_argument("--samples", type=int, default=30, help="samples for --attention-config")
     ap.add_argument("--quick", action="store_true",
                     help="profiling aid: no clock-sampling busy loops, a single end-to-end step, no CPU baseline")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.attention_config:
+        import torch
+        from paper_2605_07243_b200 import binding as sb
+        if not torch.cuda.is_available():
+            raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+        sb.load()
+        which, _, splits = args.attention_config.partition(":")
+        with torch.cuda.stream(torch.cuda.Stream()):
+            print(json.dumps(time_attention_config(torch, sb, int(which), int(splits or 0), args.samples)))
+        return 0
     return run_ours(args)
 
 
