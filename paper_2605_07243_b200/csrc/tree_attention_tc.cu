@@ -522,12 +522,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
   const int rows_per = ceil_div(TC_BM, S);
   const int my_first = crank * rows_per;
   const int my_rows = max(0, min(TC_BM, my_first + rows_per) - my_first);
-  tc_fence_before();
-  __syncthreads();  // every role is done: no async access to Q/K/V stages is in flight any more
-  if (warp == TC_MMA_WARP) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS));
-  }
+  // No CTA-wide barrier here: a softmax thread has seen the last PV complete, and the tensor pipe runs a
+  // thread's MMAs in order, so every MMA has read its operands and every K/V/Q load (each landed before the
+  // MMA that used it) is done -- the staging area below (the Q tile and the head of K stage 0) is free.
   if (tid < TC_SOFTMAX_THREADS) {
     const bool have = nb > 0 && sp.compute;
     softmax_group_sync();  // both halves' running sums are in s_xl
@@ -549,9 +546,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     }
   }
   bool merge_ok = true;
+  tc_fence_before();
   if (S > 1) {
     fence_async_smem();  // the staged rows are read by the bulk-copy engine
-    __syncthreads();
+    __syncthreads();     // rows staged; every role is done and every read of tensor memory is over
+    if (warp == TC_MMA_WARP) {
+      tc_fence_after();
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS));
+    }
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // every peer's barriers exist (long since)
     if (tid < S) {       // thread c sends owner c its slice
       const int c = tid;
@@ -568,6 +570,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
     if (warp == TC_THREADS / 32 - 1 && lane < S) mbar_arrive_remote_relaxed(mapa_u32(smem_u32(&s_bar[ACK_BAR]), lane));
   } else {
     __syncthreads();
+    if (warp == TC_MMA_WARP) {
+      tc_fence_after();
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TC_TMEM_COLS));
+    }
   }
   {
     // One row per half-warp, eight columns per lane (D <= 128).  Every lane reads all S (m, l)
