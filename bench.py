@@ -371,7 +371,7 @@ def run_ours(args):
         # expand / accept: one graph walks COLD_SETS copies of the scores / logits (more than twice the L2 size), one
         # call each, so every call streams its matrix from HBM and the replay's own cost (about 4 us) is shared by all
         # of them -- what a call costs inside an iteration; the *_single_call_graph entries replay ONE call on the same
-        # matrix (L2-warm, the whole replay cost on it), as round 1 reported them
+        # matrix (L2-warm, the whole replay cost on it)
         cold = [] if args.step_only else [("expand", g_expand_cold), ("accept", g_accept_cold)]
         for name, g in cold + [("expand_single_call_graph", g_expand), ("accept_single_call_graph", g_accept),
                                ("compact", g_compact)] + extras:
