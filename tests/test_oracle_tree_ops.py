@@ -105,6 +105,26 @@ def test_accept_exhaustive_small_trees():
     assert checked > 5000
 
 
+def test_accept_exhaustive_three_letter_alphabet():
+    """All trees with up to 4 nodes x every token / choice assignment over a THREE-letter alphabet (a third
+    letter lets a sibling match while another one mismatches under the same parent): path enumeration equals
+    the recurrence, also with the depth cut at 1 and 2."""
+    checked = 0
+    for n in range(1, 5):
+        for parent in _all_trees(n):
+            for a in itertools.product(range(3), repeat=2 * n - 1):
+                tok = [7] + list(a[: n - 1])
+                amax = list(a[n - 1:])
+                for md in (1, 2, 8):
+                    r = oracle.accept_from_amax(parent, tok, amax, max_depth=md)
+                    ln, path, toks = _accept_by_recurrence(parent, tok, amax, md)
+                    assert r["status"] == 0 and r["accept_len"] == ln
+                    assert list(r["path_nodes"][: ln + 1]) == path
+                    assert list(r["out_tokens"][: ln + 1]) == toks
+                    checked += 1
+    assert checked > 40000
+
+
 def test_accept_random_trees_with_duplicates_and_depth_cut():
     rng = W.rng_for(24)
     for _ in range(300):
