@@ -92,20 +92,21 @@ __device__ inline SeqPre plan_lengths(const AttnParams& p, int b) {
 }
 
 // Second half: ancestor sets into shared memory, tree validity, status word.  Must be called by
-// every thread of the CTA (contains barriers).  `designated` CTAs (one per sequence) also scan
+// every thread of the group (contains its barriers).  `designated` CTAs (one per sequence) also scan
 // the page table and publish the sequence's status word.
 __device__ inline SeqPlan plan_tree(const AttnParams& p, int b, bool designated, const SeqPre& pre, int* s_parent,
-                                    uint32_t* s_anc) {
+                                    uint32_t* s_anc, const ThreadGroup grp = whole_cta()) {
   SeqPlan sp;
   sp.info = pre.info;
   sp.can_write = pre.can_write;
   int err = sp.info.err;
-  const bool tree_ok = build_ancestors_smem(p.tb.parent + pre.node_base, err ? 0 : sp.info.n, s_parent, s_anc, nullptr);
+  const bool tree_ok =
+      build_ancestors_smem(p.tb.parent + pre.node_base, err ? 0 : sp.info.n, s_parent, s_anc, nullptr, grp);
   if (!err && !tree_ok) err = SB_ERR_INVALID_TREE;
   if (designated) {
-    const bool pages_ok = err ? true : pages_in_pool(p.tb, b, sp.info.P + sp.info.n);
+    const bool pages_ok = err ? true : pages_in_pool(p.tb, b, sp.info.P + sp.info.n, grp);
     if (!err && !pages_ok) err = SB_ERR_BOUNDS;  // reported; reads were clamped into the pool
-    if (threadIdx.x == 0) p.status[b] = err;
+    if (grp.tid == 0) p.status[b] = err;
     if (!pages_ok) err = 0;  // other CTAs cannot see this; stay consistent with them
   }
   sp.compute = err == 0;

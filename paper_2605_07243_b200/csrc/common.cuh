@@ -166,22 +166,35 @@ __device__ inline SeqInfo load_seq_info(const sb_tree_batch& tb, const int* q_no
   return s;
 }
 
+// The threads that run a planning helper together: the whole CTA, or its first `n` threads (a multiple
+// of 32) meeting at named barrier 1 while the CTA's other warps do something else.
+struct ThreadGroup {
+  int tid, n;
+  bool whole_cta;
+  __device__ void sync() const {
+    if (whole_cta) __syncthreads();
+    else asm volatile("bar.sync 1, %0;" ::"r"(n) : "memory");
+  }
+};
+__device__ inline ThreadGroup whole_cta() { return ThreadGroup{(int)threadIdx.x, (int)blockDim.x, true}; }
+__device__ inline ThreadGroup first_threads(int n) { return ThreadGroup{(int)threadIdx.x, n, false}; }
+
 // Builds anc[i] = {i} U anc[parent[i]] for one tree into shared memory (4 words per node) and
 // returns false for an invalid tree.  `s_parent` is scratch of n ints.  Every thread of the
-// CTA must call it; it contains __syncthreads().
-__device__ inline bool build_ancestors_smem(const int* __restrict__ parent_g, int n,
-                                            int* s_parent, uint32_t* s_anc, int* s_depth) {
+// group must call it; it contains barriers of the group.
+__device__ inline bool build_ancestors_smem(const int* __restrict__ parent_g, int n, int* s_parent, uint32_t* s_anc,
+                                            int* s_depth, const ThreadGroup grp = whole_cta()) {
   __shared__ int s_bad;
-  if (threadIdx.x == 0) s_bad = 0;
-  __syncthreads();
-  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+  if (grp.tid == 0) s_bad = 0;
+  grp.sync();
+  for (int i = grp.tid; i < n; i += grp.n) {
     const int p = parent_g[i];
     s_parent[i] = p;
     if (p < -1 || p >= i) s_bad = 1;
   }
-  __syncthreads();
+  grp.sync();
   const bool ok = s_bad == 0;
-  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+  for (int i = grp.tid; i < n; i += grp.n) {
     uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;
     int d = -1;
     if (ok) {
@@ -202,7 +215,7 @@ __device__ inline bool build_ancestors_smem(const int* __restrict__ parent_g, in
     s_anc[4 * i + 3] = m3;
     if (s_depth) s_depth[i] = d < 0 ? 0 : d;
   }
-  __syncthreads();
+  grp.sync();
   return ok;
 }
 
@@ -223,17 +236,17 @@ __device__ inline long long kv_row_elem_offset(const sb_tree_batch& tb, int b, i
 }
 
 // True when every page the sequence's [0, len) positions need is inside the pool.
-__device__ inline bool pages_in_pool(const sb_tree_batch& tb, int b, int len) {
+__device__ inline bool pages_in_pool(const sb_tree_batch& tb, int b, int len, const ThreadGroup grp = whole_cta()) {
   if (tb.page_size == 0) return true;
   __shared__ int s_bad_page;
-  if (threadIdx.x == 0) s_bad_page = 0;
-  __syncthreads();
+  if (grp.tid == 0) s_bad_page = 0;
+  grp.sync();
   const int need = ceil_div(len, tb.page_size);
-  for (int p = threadIdx.x; p < need; p += blockDim.x) {
+  for (int p = grp.tid; p < need; p += grp.n) {
     const int page = tb.page_table[(long long)b * tb.max_pages + p];
     if (page < 0 || page >= tb.num_pages) s_bad_page = 1;
   }
-  __syncthreads();
+  grp.sync();
   return s_bad_page == 0;
 }
 

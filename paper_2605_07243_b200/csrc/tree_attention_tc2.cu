@@ -180,8 +180,13 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
     if (nb > 1) issue_block(1, &kmap, smem_u32(sK) + TILE_BYTES, &s_bar[K_FULL1]);
   }
 
-  const SeqPlan sp = plan_tree(p, b, split == 0 && blockIdx.y == 0, pre, s_parent, s_anc);
-  const SeqInfo& si = sp.info;
+  // Only the softmax threads need the tree (ancestor sets, validity): they plan it among themselves
+  // while the loaders look up pages and the first S = Q K^T is issued from the lengths alone.
+  SeqPlan sp;
+  sp.info = pre.info;
+  sp.can_write = pre.can_write;
+  sp.compute = false;
+  const SeqInfo& si = pre.info;
 
   // Row state of the softmax threads, one set per tile: row = TMEM lane, `half` selects the 64
   // columns of every block and the half of the output row this thread owns.
@@ -207,6 +212,9 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
                        q_ok ? 16 : 0);
       }
       asm volatile("cp.async.commit_group;\n" ::);
+    }
+    sp = plan_tree(p, b, split == 0 && blockIdx.y == 0, pre, s_parent, s_anc, first_threads(T2_SOFTMAX_THREADS));
+    if (!q_tma && nb > 0) {
       asm volatile("cp.async.wait_group 0;\n" ::: "memory");
       fence_async_smem();
       mbar_arrive(&s_bar[Q_FULL]);
@@ -436,18 +444,19 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
     if (!ok && lane == 0) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
   }
 
-  // ---- normalise and store, one tile after the other ------------------------------------------------
-  // The softmax threads stage the tile's rows as [O / l in bf16 (D) | m | l | pad] over the idle Q
-  // tiles; then half a warp per row writes whole rows: the output row and its log-sum-exp, or, with
-  // several KV chunks, this chunk's bf16 partial for attn_merge_kernel.
+  // ---- normalise and store ------------------------------------------------------------------------------
+  // The softmax threads stage both tiles' rows as [O / l in bf16 (D) | base-2 log-sum-exp | pad | global row]
+  // over the idle Q tiles (global row -1: the tile has no such row); then half a warp per row writes whole
+  // rows: the output row and its log-sum-exp, or, with several KV chunks, this chunk's bf16 partial for
+  // attn_merge_kernel.
+  // They start as soon as both accumulators are final: by then every MMA has completed, and with them
+  // every load into the Q tiles and K stages (each was awaited before the MMA that read it).
   constexpr int ROWB = D * 2 + 16;  // bytes per staged row (16-byte multiple)
-  tc_fence_before();
-  __syncthreads();  // every role is done: no async access to Q/K/V stages is in flight any more
-  tc_fence_after();
-  const bool have = nb > 0 && sp.compute;
-  for (int t = 0; t < ntile; ++t) {
-    uint8_t* stg = sQ + t * (TC_BM * ROWB);  // disjoint per tile; runs a little into the idle K stage
-    if (tid < T2_SOFTMAX_THREADS) {
+  if (tid < T2_SOFTMAX_THREADS) {
+    const bool have = nb > 0 && sp.compute;
+    softmax_group_sync();  // both halves' running sums are in s_xl
+    for (int t = 0; t < ntile; ++t) {
+      uint8_t* stg = sQ + t * (TC_BM * ROWB);  // disjoint per tile; runs a little into the idle K stage
       const float l_tot = s_xl[(t * 2) * TC_BM + row] + s_xl[(t * 2 + 1) * TC_BM + row];
       const float m_ref = t == 0 ? m_t[0] : m_t[1];
       const float inv_l = (have && l_tot > 0.f) ? __fdividef(1.f, l_tot) : 0.f;
@@ -467,23 +476,32 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
         }
       }
       if (half == 0) {
-        *reinterpret_cast<float*>(dst + D * 2) = (have && l_tot > 0.f) ? m_ref : -INFINITY;
-        *reinterpret_cast<float*>(dst + D * 2 + 4) = (have && l_tot > 0.f) ? l_tot : 0.f;
+        const int Rr = row0 + t * TC_BM + row;
+        const int node_l = Rr / G, hh = Rr - node_l * G;
+        const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
+        const bool row_ok = Rr < rows_total && SB_CHECKED_ACCESS(grow, rows_all, &p.status[b]);
+        *reinterpret_cast<float*>(dst + D * 2) = (have && l_tot > 0.f) ? m_ref + log2f(l_tot) : -INFINITY;
+        *reinterpret_cast<long long*>(dst + D * 2 + 8) = row_ok ? grow : -1ll;
       }
     }
-    __syncthreads();
+  }
+  tc_fence_before();
+  __syncthreads();  // the rows are staged; tensor memory has been read for the last time
+  if (warp == T2_MMA_WARP) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(T2_TMEM_COLS));
+  }
+  for (int t = 0; t < ntile; ++t) {
+    const uint8_t* stg = sQ + t * (TC_BM * ROWB);
     const int sub = lane >> 4, col8 = lane & 15;
+    if (col8 >= D / 8) continue;
+#pragma unroll 3
     for (int r = 2 * warp + sub; r < TC_BM; r += 2 * (T2_THREADS / 32)) {
-      const int Rr = row0 + t * TC_BM + r;
-      if (Rr >= rows_total || col8 >= D / 8) continue;
       const uint8_t* rowp = stg + (size_t)r * ROWB;
-      const float m = *reinterpret_cast<const float*>(rowp + D * 2);
-      const float l = *reinterpret_cast<const float*>(rowp + D * 2 + 4);
+      const long long grow = *reinterpret_cast<const long long*>(rowp + D * 2 + 8);
+      const float lse2 = *reinterpret_cast<const float*>(rowp + D * 2);
       const uint4 raw = *reinterpret_cast<const uint4*>(rowp + col8 * 16);
-      const int node_l = Rr / G, hh = Rr - node_l * G;
-      const long long grow = (long long)(si.q_off + node_l) * Hq + g * G + hh;
-      const float lse2 = l > 0.f ? m + log2f(l) : -INFINITY;
-      if (!SB_CHECKED_ACCESS(grow, rows_all, &p.status[b])) continue;
+      if (grow < 0) continue;
       if (p.outer == 1) {
         *reinterpret_cast<uint4*>(p.out + grow * D + col8 * 8) = raw;
         if (p.lse && col8 == 0) p.lse[grow] = lse2 == -INFINITY ? 0.f : lse2 * kLn2;
@@ -494,12 +512,6 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
         if (col8 == 0) p.part_lse[(long long)split * rows_all + grow] = lse2;
       }
     }
-  }
-  tc_fence_before();
-  __syncthreads();  // all reads of tensor memory are done
-  if (warp == T2_MMA_WARP) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(T2_TMEM_COLS));
   }
 }
 
