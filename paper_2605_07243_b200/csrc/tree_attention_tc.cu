@@ -337,13 +337,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const AttnParams
           if (ok) ok = mbar_wait(&s_bar[PV_FULL], (j - 1) & 1, s_abort);
           pv_waited = true;
           tc_fence_after();
+          // (rare, and 16 columns at a time: the block's 64 scores stay in registers meanwhile)
+#pragma unroll 1
+          for (int c = 0; c < DH / 16; ++c) {
+            uint32_t r[16];
+            tmem_ld16(tmem_o + lane_base + half * DH + c * 16, r);
 #pragma unroll
-          for (int c = 0; c < DH / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(tmem_o + lane_base + half * DH + c * 32, r);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
-            tmem_st32(tmem_o + lane_base + half * DH + c * 32, r);
+            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
+            tmem_st16(tmem_o + lane_base + half * DH + c * 16, r);
           }
           tmem_wait_st();
         }
