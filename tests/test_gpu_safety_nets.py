@@ -74,6 +74,13 @@ def _attention_cases():
         n_q_heads=6, n_kv_heads=2, head_dim=64, page_size=64), (0, 2)
     yield "contiguous, two row tiles, 12 chunks (partials + merge kernel)", W.make_attn_case(
         rng, parents=[W.block_tree(rng, 60)], prefix_lens=[1500], n_q_heads=16, n_kv_heads=4, head_dim=128), (0, 12)
+    # more (sequence, KV head, row tile) units than SMs and up to three row tiles per KV head: the two-tile kernel,
+    # alone (library's choice) and with bf16 partials and the merge kernel (2 chunks)
+    sizes = [70, 33, 96, 41, 64, 50, 88, 37, 72, 45]
+    yield "ragged paged batch on the two-tile kernel", W.make_attn_case(
+        rng, parents=[W.random_tree(rng, n, 8) for n in sizes],
+        prefix_lens=[130, 517, 64, 300, 0, 255, 129, 700, 31, 402], n_q_heads=32, n_kv_heads=8, head_dim=128,
+        page_size=64), (0, 2)
     attn, _ = W.config1_tiny()
     yield "tiny configuration", attn, (0, 2)
 
