@@ -196,6 +196,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
   const int row = (warp & 3) * 32 + lane;
   const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
 
+  bool softmax_ok = true;
   if (tid < T2_SOFTMAX_THREADS) {
     // ------------------------------------------------------------------ softmax warps
     if (!q_tma && nb > 0) {  // Q tiles as a gather of (node, head) rows
@@ -316,9 +317,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
     }
 #pragma unroll
     for (int t = 0; t < 2; ++t) s_xl[(t * 2 + half) * TC_BM + row] = l_t[t];
-    if (nb > 0 && ok) ok = mbar_wait(&s_bar[O_DONE], 0, s_abort);  // both accumulators are final
-    tc_fence_after();
-    if (!ok) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
+    softmax_ok = ok;
   } else if (warp == T2_MMA_WARP) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && nb > 0) {
@@ -450,13 +449,20 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
   // over the idle Q tiles (global row -1: the tile has no such row); then half a warp per row writes whole
   // rows: the output row and its log-sum-exp, or, with several KV chunks, this chunk's bf16 partial for
   // attn_merge_kernel.
-  // They start as soon as both accumulators are final: by then every MMA has completed, and with them
-  // every load into the Q tiles and K stages (each was awaited before the MMA that read it).
+  // A tile is staged as soon as its accumulator is final.  With two tiles that is PV_{nv-2} for tile 0 (the
+  // barrier is in that phase or the next, since S_{nv-1} has been consumed), so tile 0 is staged while the last
+  // PV runs.  By then every S has completed, and with the MMAs every load into the Q tiles and K stages (each
+  // was awaited before the MMA that read it).
   constexpr int ROWB = D * 2 + 16;  // bytes per staged row (16-byte multiple)
   if (tid < T2_SOFTMAX_THREADS) {
+    bool ok = softmax_ok;
     const bool have = nb > 0 && sp.compute;
     softmax_group_sync();  // both halves' running sums are in s_xl
     for (int t = 0; t < ntile; ++t) {
+      if (nb > 0 && ok) {
+        ok = t + 1 < ntile ? mbar_wait(&s_bar[PV_FULL], (nv - 2) & 1, s_abort) : mbar_wait(&s_bar[O_DONE], 0, s_abort);
+        tc_fence_after();
+      }
       uint8_t* stg = sQ + t * (TC_BM * ROWB);  // disjoint per tile; runs a little into the idle K stage
       const float l_tot = s_xl[(t * 2) * TC_BM + row] + s_xl[(t * 2 + 1) * TC_BM + row];
       const float m_ref = t == 0 ? m_t[0] : m_t[1];
@@ -485,6 +491,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) attn_tc2_kernel(const AttnParam
         *reinterpret_cast<long long*>(dst + D * 2 + 8) = row_ok ? grow : -1ll;
       }
     }
+    if (!ok) atomicMax(&p.status[b], (int)SB_ERR_CUDA);
   }
   tc_fence_before();
   __syncthreads();  // the rows are staged; tensor memory has been read for the last time
